@@ -1,0 +1,242 @@
+/*
+ * aero.h -- C ABI of the B200 (sm_100a) library for the data-parallel hot path of
+ * a GRPO / AERO training step (AERO: "Adaptive Efficient Rollout Optimization",
+ * arXiv 2602.14338).
+ *
+ * Two stages:
+ *   (a) aero_group_stats     per-prompt group statistics over ragged groups:
+ *                            group-relative advantage (Eq. 1), zero-advantage group
+ *                            masking (Sec. 3.2), selective-rejection keep-mask
+ *                            (Sec. 4.2, Strategies 2 and 3), Beta-Binomial posterior
+ *                            update (Sec. 4.2 Strategy 2; Appendix C).
+ *   (b) aero_grpo_loss_fwd   fused lm_head projection + online log-sum-exp + target
+ *       aero_grpo_loss_bwd   gather, importance ratio, clip, weighted token mean
+ *                            (Eq. 2; Appendix C "GRPO Training") and its backward to
+ *                            dH and dW (Eq. 3; Appendix A).  The [T,V] logits are
+ *                            never written to memory.
+ *
+ * Conventions
+ *   - Packed ragged batch ("padding removal", Appendix C): prompt p owns rollouts
+ *     go[p] .. go[p+1]-1, R = go[P]; rollout i owns token rows cs[i] .. cs[i+1]-1,
+ *     T = cs[R].  Rollouts of one prompt are consecutive; rows of one rollout are
+ *     consecutive.
+ *   - W is the lm_head weight, [V,d] row-major; logits z_t = W h_t.  H is [T,d]
+ *     row-major.  dtype is bf16 (tensor-core path, d % 64 == 0 and 16-byte aligned
+ *     bases required) or fp32 (plain path for small shapes).
+ *   - Unless a parameter says "host", every array pointer is a DEVICE pointer owned
+ *     by the caller and must stay valid until the stream has run the call.  The
+ *     library allocates no array memory: scratch is passed in as `workspace`.
+ *   - Calls are asynchronous on the context's stream.  Host-side checks (null
+ *     pointers, shapes, alignment, workspace size) fail with a negative return and
+ *     launch nothing.  Data-dependent faults (target id outside [0,V), non-monotone
+ *     offsets, non-binary reward, empty rollout, a pipeline wait that gave up) never
+ *     trap: they set bits in a device status word read by aero_last_status, and the
+ *     offending element is skipped or clamped.
+ *   - Sign: the paper maximises J (Eq. 2); the library returns loss = -J, so dH and
+ *     dW are descent directions.
+ *   - There is no CPU fallback: without a CUDA device every compute call fails with
+ *     AERO_ERR_CUDA.
+ */
+#ifndef AERO_H_
+#define AERO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- return codes ------------------------------------------------------------- */
+#define AERO_OK               0
+#define AERO_ERR_INVALID     -1   /* null pointer, negative size, misaligned base      */
+#define AERO_ERR_UNSUPPORTED -2   /* shape the kernels do not cover (e.g. d % 64 != 0) */
+#define AERO_ERR_WORKSPACE   -3   /* workspace smaller than aero_*_workspace_bytes     */
+#define AERO_ERR_CUDA        -4   /* a CUDA runtime/driver call failed                 */
+
+/* ---- device status bits (aero_last_status) ------------------------------------ */
+#define AERO_ST_BAD_TARGET     1u   /* y[t] outside [0,V): row treated as dropped      */
+#define AERO_ST_BAD_OFFSETS    2u   /* go[] or cs[] not non-decreasing                 */
+#define AERO_ST_BAD_REWARD     4u   /* reward not exactly 0 or 1                       */
+#define AERO_ST_EMPTY_ROLLOUT  8u   /* cs[i+1] == cs[i] for a present rollout          */
+#define AERO_ST_TIMEOUT       16u   /* a bounded wait inside a kernel ran out          */
+
+/* ---- enumerations ------------------------------------------------------------- */
+#define AERO_UNIFORM_MASK   0   /* all-correct / all-incorrect groups are dropped (Sec. 3.2)      */
+#define AERO_UNIFORM_BAYES  1   /* they use the posterior mean instead (Sec. 4.2 Strategy 2)      */
+#define AERO_STATS_KEPT     0   /* mean/std over the curated subset (Theorem 4.1: mu = c/(c+m))   */
+#define AERO_STATS_ALL      1   /* mean/std over every present rollout of the group               */
+#define AERO_TOKEN_MEAN     0   /* token-level mean (Appendix C, "GRPO Training")                 */
+#define AERO_SEQ_MEAN       1   /* 1/N sum_i 1/|o_i| sum_t (Eq. 2)                                */
+#define AERO_DENOM_SURVIVING 0  /* normalise by surviving tokens / prompts                        */
+#define AERO_DENOM_ALL      1   /* count dropped tokens / prompts too (the shrinking batch        */
+                                /* gradient described in Sec. 3.1)                                */
+#define AERO_BF16 0
+#define AERO_FP32 1
+
+#define AERO_CAT_ZERO    0      /* categories of Appendix C, threshold tau = 0.5, decided on      */
+#define AERO_CAT_PARTIAL 1      /* integers: Partial iff 0 < c and 2c < n                         */
+#define AERO_CAT_GOOD    2
+#define AERO_CAT_PERFECT 3
+#define AERO_CAT_EMPTY   4      /* no present rollout                                             */
+
+/* Indices into counters[8] written by aero_group_stats. */
+#define AERO_CNT_R_KEPT    0
+#define AERO_CNT_T_KEPT    1
+#define AERO_CNT_P_SURV    2
+#define AERO_CNT_ZERO      3
+#define AERO_CNT_PARTIAL   4
+#define AERO_CNT_GOOD      5
+#define AERO_CNT_PERFECT   6
+#define AERO_CNT_T_PRESENT 7
+
+/* Hyper-parameters (Table 9 of the paper gives the defaults noted here). */
+typedef struct aero_cfg {
+  int32_t uniform_policy;   /* AERO_UNIFORM_*                                   default MASK */
+  int32_t rejection;        /* 1: Strategy 3 (keep all correct + k*c incorrect)  default 0   */
+  int32_t k_ratio;          /* k >= 1, incorrect : correct ratio                 default 1   */
+  int32_t rescue_S;         /* Strategy 1 threshold S on correct counts          default 0   */
+  int32_t n_explore;        /* exploration budget the threshold refers to        default 8   */
+  int32_t n_keep_uniform;   /* rollouts kept from a uniform group; <= 0: all     default 4   */
+  int32_t stats_over;       /* AERO_STATS_*                                      default KEPT */
+  int32_t agg;              /* AERO_TOKEN_MEAN | AERO_SEQ_MEAN                   default TOKEN_MEAN */
+  int32_t denom;            /* AERO_DENOM_*                                      default SURVIVING */
+  float   alpha0, beta0;    /* Beta prior used when alpha_in/beta_in are NULL    default 1, 1 */
+  float   eps_std;          /* added to the standard deviation in Eq. 1          default 1e-6 */
+  float   clip_lo, clip_hi; /* clip(rho, 1-clip_lo, 1+clip_hi)                   default 0.2, 0.2 */
+  uint64_t seed;            /* seeds the default selection keys                  default 0   */
+  int32_t dtype;            /* AERO_BF16 | AERO_FP32: type of H, W and dH        default BF16 */
+  int32_t reserved;
+} aero_cfg;
+
+typedef struct aero_ctx aero_ctx;   /* opaque: device id, borrowed stream, status word */
+
+/* Library version (major*100 + minor). */
+int aero_version(void);
+
+/* Human-readable name of a return code (static string, never NULL). */
+const char* aero_error_string(int code);
+
+/* Fill *cfg with the defaults listed above. */
+void aero_cfg_default(aero_cfg* cfg);
+
+/* Create a context on CUDA device `device`.  `cuda_stream` (a cudaStream_t, may be
+ * NULL for the default stream) is borrowed, not owned.  Allocates the 4-byte device
+ * status word and nothing else. */
+int aero_create(aero_ctx** out, int device, void* cuda_stream);
+int aero_destroy(aero_ctx* ctx);
+int aero_set_stream(aero_ctx* ctx, void* cuda_stream);
+
+/* Synchronise the stream, return the OR of all status bits raised since the last
+ * call in *bits (host pointer) and clear them. */
+int aero_last_status(aero_ctx* ctx, uint32_t* bits);
+
+/* ------------------------------------------------------------------------------
+ * Stage (a).  Group statistics, curation and weights (Eq. 1; Sec. 3.2; Sec. 4.2
+ * Strategies 2-3; Appendix C categories and posterior).
+ *
+ * For every prompt p, over its PRESENT rollouts (keep_in[i] != 0, or all when
+ * keep_in is NULL): n = count, c = number with reward 1;
+ *   category  Zero (c=0) / Partial (0<c, 2c<n) / Good (2c>=n, c<n) / Perfect (c=n);
+ *   posterior alpha' = alpha + c, beta' = beta + n - c, u~ = alpha'/(alpha'+beta');
+ *   keep-mask uniform group: none (MASK) or the min(n_keep_uniform, n) rollouts of
+ *             smallest (key, index) (BAYES);  low-success mixed group with rejection:
+ *             all correct + the min(k*c, n-c) incorrect of smallest (key, index),
+ *             where low-success means Partial, or c*n_explore <= rescue_S*n when
+ *             rescue_S > 0;  any other group: all present rollouts;
+ *   advantage mixed group: (r - mean)/(std + eps_std) with the population std over
+ *             the kept subset (STATS_KEPT) or the present group (STATS_ALL);
+ *             uniform group under BAYES: (r - u~)/(sqrt(u~(1-u~)) + eps_std);
+ *             0 for every rollout that is not kept;
+ *   weight    w_i = 1/T_kept (TOKEN_MEAN) or 1/(P_surv * n'_p * len_i) (SEQ_MEAN)
+ *             for kept rollouts, 0 otherwise; with DENOM_ALL the denominators are the
+ *             present tokens T_present, resp. all P prompts.
+ * key == NULL selects the default key: the high 32 bits of SplitMix64 applied to
+ * seed + (i+1) * 0x9E3779B97F4A7C15, i the global rollout index.
+ *
+ * Inputs   go [P+1] i32, reward [R] f32, cs [R+1] i64, key [R] u32 or NULL,
+ *          keep_in [R] u8 or NULL, alpha_in/beta_in [P] f32 or both NULL.
+ * Outputs  adv [R] f32, w [R] f32, keep [R] u8, gmask [P] u8 (1 iff any rollout
+ *          kept), cat [P] u8, u_tilde/alpha_out/beta_out [P] f32, kept_ids [R] i32
+ *          (first R_kept entries: kept rollout indices, ascending; rest -1),
+ *          kept_tok_off [R+1] i64 (exclusive scan of kept lengths over kept_ids;
+ *          entries past R_kept hold T_kept), counters [8] i64 (AERO_CNT_*),
+ *          metrics [4] f32 or NULL: zero-accuracy ratio x^zero (Sec. 3.2), mean
+ *          |advantage| over kept rollouts, kept rollout fraction, kept token fraction.
+ *          Integer outputs are exact; alpha_out/beta_out may alias alpha_in/beta_in.
+ * workspace: at least aero_group_workspace_bytes(P, R) bytes, 256-byte aligned.
+ * P == 0 or R == 0 is valid (counters are zeroed).
+ */
+size_t aero_group_workspace_bytes(int32_t P, int32_t R);
+
+int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
+                     const int32_t* go, const float* reward, const int64_t* cs,
+                     const uint32_t* key, const uint8_t* keep_in,
+                     const float* alpha_in, const float* beta_in,
+                     float* adv, float* w, uint8_t* keep, uint8_t* gmask, uint8_t* cat,
+                     float* u_tilde, float* alpha_out, float* beta_out,
+                     int32_t* kept_ids, int64_t* kept_tok_off, int64_t* counters,
+                     float* metrics, void* workspace, size_t workspace_bytes);
+
+/* ------------------------------------------------------------------------------
+ * Stage (b), forward (Eq. 2; Appendix C "GRPO Training").
+ *
+ * For every token row t of a kept rollout i (keep[i] != 0):
+ *   z_tv = sum_k H[t,k] W[v,k]  (fp32 accumulation of bf16 products, never stored)
+ *   lse_t = log sum_v exp z_tv,  logp_t = z_{t,y_t} - lse_t
+ *   rho_t = exp(logp_t - old_logp_t)
+ *   s_t   = min(rho_t A_i, clip(rho_t, 1-clip_lo, 1+clip_hi) A_i)
+ *   loss  = - sum_t w_i s_t                       (loss = -J)
+ *   g_t   = dloss/dlogp_t = - w_i A_i rho_t [rho_t A_i <= clip(rho_t) A_i]
+ * (equality counts as unclipped; the two-sided form of Eq. 2 governs, so the
+ * indicator is rho <= 1+clip_hi for A > 0 and rho >= 1-clip_lo for A < 0).
+ * Rows of dropped rollouts get logp = lse = g = 0.
+ *
+ * Inputs   H [T,d], W [V,d] (cfg->dtype), y [T] i32, old_logp [T] f32, cs [R+1] i64,
+ *          adv [R] f32, w [R] f32, keep [R] u8 (outputs of aero_group_stats).
+ * Outputs  logp, lse, g [T] f32; loss [1] f32 (overwritten, or added to when
+ *          accumulate != 0, for callers that split a batch into token ranges);
+ *          metrics [4] f32 or NULL: clipped fraction of kept tokens, mean rho,
+ *          mean (old_logp - logp), number of kept tokens.  The loss is reduced in a
+ *          fixed order: repeated calls give identical bits.
+ * workspace: at least aero_fwd_workspace_bytes(T, d, V, R) bytes, 256-byte aligned.
+ */
+size_t aero_fwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R);
+
+int aero_grpo_loss_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                       const void* H, const void* W, const int32_t* y, const float* old_logp,
+                       const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                       float* logp, float* lse, float* g, float* loss, float* metrics,
+                       int accumulate, void* workspace, size_t workspace_bytes);
+
+/* ------------------------------------------------------------------------------
+ * Stage (b), backward (Eq. 3; Appendix A: grad rho = rho grad log pi, clipped tokens
+ * contribute nothing).
+ *
+ *   dz_tv = grad_scale * g_t * (1[v == y_t] - exp(z_tv - lse_t))     (recomputed)
+ *   dH[t,:] = sum_v dz_tv W[v,:]          dW[v,:] (+)= sum_t dz_tv H[t,:]
+ * dz is rounded to bf16 before the two products (fp32 accumulation).  Token rows
+ * are processed in chunks whose dz block lives in `workspace`; a larger workspace
+ * means fewer passes over dW.  Rows of dropped rollouts get dH = 0.
+ *
+ * Inputs   as the forward, plus lse and g from it.
+ * Outputs  dH [T,d] (cfg->dtype); dW [V,d] f32, overwritten or, when
+ *          accumulate_dW != 0, added to.
+ * workspace: at least aero_bwd_workspace_bytes(T, d, V, R, chunk_tokens); chunk_tokens
+ *          (a multiple of 128, >= 128) is the number of token rows per chunk the
+ *          caller is prepared to pay for; the call uses as many as the given
+ *          workspace_bytes allows.
+ */
+size_t aero_bwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R, int64_t chunk_tokens);
+
+int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                       const void* H, const void* W, const int32_t* y,
+                       const int64_t* cs, const uint8_t* keep,
+                       const float* lse, const float* g, float grad_scale,
+                       void* dH, float* dW, int accumulate_dW,
+                       void* workspace, size_t workspace_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* AERO_H_ */
