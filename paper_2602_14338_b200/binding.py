@@ -1,0 +1,241 @@
+"""ctypes binding of libaero_b200.so: argument marshalling only.
+
+Every function here has the name and argument order of its C counterpart in
+include/aero.h.  Tensors are torch CUDA tensors used purely as device buffers;
+the binding passes their data pointers and checks dtype/shape/contiguity.  There
+is no fallback: if the library is missing or has no CUDA device, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libaero_b200.so")
+
+AERO_UNIFORM_MASK, AERO_UNIFORM_BAYES = 0, 1
+AERO_STATS_KEPT, AERO_STATS_ALL = 0, 1
+AERO_TOKEN_MEAN, AERO_SEQ_MEAN = 0, 1
+AERO_DENOM_SURVIVING, AERO_DENOM_ALL = 0, 1
+AERO_BF16, AERO_FP32 = 0, 1
+AERO_ST_BAD_TARGET, AERO_ST_BAD_OFFSETS, AERO_ST_BAD_REWARD, AERO_ST_EMPTY_ROLLOUT, AERO_ST_TIMEOUT = 1, 2, 4, 8, 16
+
+EXPORTS = [
+    "aero_version", "aero_error_string", "aero_cfg_default", "aero_create", "aero_destroy",
+    "aero_set_stream", "aero_last_status", "aero_group_workspace_bytes", "aero_group_stats",
+    "aero_fwd_workspace_bytes", "aero_grpo_loss_fwd", "aero_bwd_workspace_bytes", "aero_grpo_loss_bwd",
+]
+
+
+class AeroCfg(C.Structure):
+    _fields_ = [
+        ("uniform_policy", C.c_int32), ("rejection", C.c_int32), ("k_ratio", C.c_int32),
+        ("rescue_S", C.c_int32), ("n_explore", C.c_int32), ("n_keep_uniform", C.c_int32),
+        ("stats_over", C.c_int32), ("agg", C.c_int32), ("denom", C.c_int32),
+        ("alpha0", C.c_float), ("beta0", C.c_float), ("eps_std", C.c_float),
+        ("clip_lo", C.c_float), ("clip_hi", C.c_float),
+        ("seed", C.c_uint64), ("dtype", C.c_int32), ("reserved", C.c_int32),
+    ]
+
+
+class AeroError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def load_library():
+    """Load libaero_b200.so and declare the C signatures.  Raises if the file is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise AeroError(f"{LIB_PATH} not found: build it with `python -m paper_2602_14338_b200.build`")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
+    lib.aero_version.restype = C.c_int
+    lib.aero_error_string.restype = C.c_char_p
+    lib.aero_error_string.argtypes = [C.c_int]
+    lib.aero_cfg_default.restype = None
+    lib.aero_cfg_default.argtypes = [C.POINTER(AeroCfg)]
+    lib.aero_create.argtypes = [C.POINTER(vp), C.c_int, vp]
+    lib.aero_destroy.argtypes = [vp]
+    lib.aero_set_stream.argtypes = [vp, vp]
+    lib.aero_last_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+    lib.aero_group_workspace_bytes.restype = sz
+    lib.aero_group_workspace_bytes.argtypes = [i32, i32]
+    lib.aero_group_stats.argtypes = [vp, C.POINTER(AeroCfg), i32, i32] + [vp] * 19 + [vp, sz]
+    lib.aero_fwd_workspace_bytes.restype = sz
+    lib.aero_fwd_workspace_bytes.argtypes = [i64, i32, i32, i32]
+    lib.aero_grpo_loss_fwd.argtypes = [vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 13 + [C.c_int, vp, sz]
+    lib.aero_bwd_workspace_bytes.restype = sz
+    lib.aero_bwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i64]
+    lib.aero_grpo_loss_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 7 + [f32] +
+                                       [vp, vp, C.c_int, vp, sz])
+    _lib = lib
+    return lib
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        msg = load_library().aero_error_string(rc).decode()
+        raise AeroError(f"{what} failed: {msg} ({rc})")
+
+
+def cfg_default(**over) -> AeroCfg:
+    cfg = AeroCfg()
+    load_library().aero_cfg_default(C.byref(cfg))
+    for k, v in over.items():
+        if not hasattr(cfg, k):
+            raise AttributeError(k)
+        setattr(cfg, k, v)
+    return cfg
+
+
+def _ptr(t, dtype=None, numel=None, name="tensor"):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise AeroError(f"{name} must be a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise AeroError(f"{name} must have dtype {dtype}, got {t.dtype}")
+    if numel is not None and t.numel() < numel:
+        raise AeroError(f"{name} has {t.numel()} elements, needs {numel}")
+    return t.data_ptr()
+
+
+def _ptr_key(key, R):
+    if key is None:
+        return None
+    if key.dtype not in (torch.int32, torch.uint32):
+        raise AeroError("key must be a 32-bit integer tensor (its bits are read as unsigned)")
+    return _ptr(key, None, R, "key")
+
+
+class Context:
+    """Owns an aero_ctx bound to a device and (borrowed) to the current torch stream."""
+
+    def __init__(self, device=0, stream=None):
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise AeroError("no CUDA device: this library has no CPU path")
+        self.device = torch.device("cuda", device)
+        if stream is None:
+            stream = torch.cuda.current_stream(self.device)
+        self.stream = stream
+        h = C.c_void_p()
+        _check(self.lib.aero_create(C.byref(h), device, C.c_void_p(stream.cuda_stream)), "aero_create")
+        self.h = h
+        self._ws = None
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.aero_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_stream(self, stream):
+        self.stream = stream
+        _check(self.lib.aero_set_stream(self.h, C.c_void_p(stream.cuda_stream)), "aero_set_stream")
+
+    def last_status(self) -> int:
+        bits = C.c_uint32(0)
+        _check(self.lib.aero_last_status(self.h, C.byref(bits)), "aero_last_status")
+        return bits.value
+
+    def workspace(self, nbytes: int):
+        """A cached uint8 device buffer of at least nbytes (256-byte aligned by the torch allocator)."""
+        if self._ws is None or self._ws.numel() < nbytes:
+            self._ws = None
+            self._ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    # ---- stage (a) ------------------------------------------------------------------
+    def group_workspace_bytes(self, P, R):
+        return self.lib.aero_group_workspace_bytes(P, R)
+
+    def group_stats(self, cfg, go, reward, cs, key=None, keep_in=None, alpha_in=None, beta_in=None, out=None):
+        P, R = go.numel() - 1, reward.numel()
+        dev = self.device
+        o = out or {}
+
+        def buf(name, n, dt):
+            if name not in o:
+                o[name] = torch.empty(max(n, 1), dtype=dt, device=dev)
+            return o[name]
+
+        adv, w = buf("adv", R, torch.float32), buf("w", R, torch.float32)
+        keep, gmask, cat = buf("keep", R, torch.uint8), buf("gmask", P, torch.uint8), buf("cat", P, torch.uint8)
+        u, ao, bo = buf("u_tilde", P, torch.float32), buf("alpha_out", P, torch.float32), buf("beta_out", P, torch.float32)
+        kid, kto = buf("kept_ids", R, torch.int32), buf("kept_tok_off", R + 1, torch.int64)
+        cnt, met = buf("counters", 8, torch.int64), buf("metrics", 4, torch.float32)
+        ws = self.workspace(self.group_workspace_bytes(P, R))
+        rc = self.lib.aero_group_stats(
+            self.h, C.byref(cfg), P, R, _ptr(go, torch.int32, P + 1, "go"), _ptr(reward, torch.float32, R, "reward"),
+            _ptr(cs, torch.int64, R + 1, "cs"), _ptr_key(key, R),
+            _ptr(keep_in, torch.uint8, R, "keep_in"), _ptr(alpha_in, torch.float32, P, "alpha_in"),
+            _ptr(beta_in, torch.float32, P, "beta_in"), _ptr(adv), _ptr(w), _ptr(keep), _ptr(gmask), _ptr(cat),
+            _ptr(u), _ptr(ao), _ptr(bo), _ptr(kid), _ptr(kto), _ptr(cnt), _ptr(met), ws.data_ptr(), ws.numel())
+        _check(rc, "aero_group_stats")
+        return o
+
+    # ---- stage (b) ------------------------------------------------------------------
+    def fwd_workspace_bytes(self, T, d, V, R):
+        return self.lib.aero_fwd_workspace_bytes(T, d, V, R)
+
+    def bwd_workspace_bytes(self, T, d, V, R, chunk_tokens):
+        return self.lib.aero_bwd_workspace_bytes(T, d, V, R, chunk_tokens)
+
+    def grpo_loss_fwd(self, cfg, H, W, y, old_logp, cs, adv, w, keep, out=None, accumulate=False):
+        T, d = H.shape
+        V = W.shape[0]
+        R = cs.numel() - 1
+        dt = torch.bfloat16 if cfg.dtype == AERO_BF16 else torch.float32
+        o = out or {}
+        for name in ("logp", "lse", "g"):
+            if name not in o:
+                o[name] = torch.empty(max(T, 1), dtype=torch.float32, device=self.device)
+        if "loss" not in o:
+            o["loss"] = torch.zeros(1, dtype=torch.float32, device=self.device)
+        if "metrics" not in o:
+            o["metrics"] = torch.zeros(4, dtype=torch.float32, device=self.device)
+        ws = self.workspace(self.fwd_workspace_bytes(T, d, V, R))
+        rc = self.lib.aero_grpo_loss_fwd(
+            self.h, C.byref(cfg), T, d, V, R, _ptr(H, dt, T * d, "H"), _ptr(W, dt, V * d, "W"),
+            _ptr(y, torch.int32, T, "y"), _ptr(old_logp, torch.float32, T, "old_logp"),
+            _ptr(cs, torch.int64, R + 1, "cs"), _ptr(adv, torch.float32, R, "adv"), _ptr(w, torch.float32, R, "w"),
+            _ptr(keep, torch.uint8, R, "keep"), _ptr(o["logp"]), _ptr(o["lse"]), _ptr(o["g"]), _ptr(o["loss"]),
+            _ptr(o["metrics"]), 1 if accumulate else 0, ws.data_ptr(), ws.numel())
+        _check(rc, "aero_grpo_loss_fwd")
+        return o
+
+    def grpo_loss_bwd(self, cfg, H, W, y, cs, keep, lse, g, grad_scale=1.0, dH=None, dW=None,
+                      accumulate_dW=False, chunk_tokens=None, workspace=None):
+        T, d = H.shape
+        V = W.shape[0]
+        R = cs.numel() - 1
+        dt = torch.bfloat16 if cfg.dtype == AERO_BF16 else torch.float32
+        if dH is None:
+            dH = torch.empty((max(T, 1), d), dtype=dt, device=self.device)[:T]
+        if dW is None:
+            dW = torch.empty((V, d), dtype=torch.float32, device=self.device)
+        if workspace is None:
+            if chunk_tokens is None:
+                chunk_tokens = min(max(128, (T + 127) // 128 * 128), 2 * 148 * 128)
+            workspace = self.workspace(self.bwd_workspace_bytes(T, d, V, R, chunk_tokens))
+        rc = self.lib.aero_grpo_loss_bwd(
+            self.h, C.byref(cfg), T, d, V, R, _ptr(H, dt, T * d, "H"), _ptr(W, dt, V * d, "W"),
+            _ptr(y, torch.int32, T, "y"), _ptr(cs, torch.int64, R + 1, "cs"), _ptr(keep, torch.uint8, R, "keep"),
+            _ptr(lse, torch.float32, T, "lse"), _ptr(g, torch.float32, T, "g"), C.c_float(grad_scale),
+            _ptr(dH, dt, T * d, "dH"), _ptr(dW, torch.float32, V * d, "dW"), 1 if accumulate_dW else 0,
+            workspace.data_ptr(), workspace.numel())
+        _check(rc, "aero_grpo_loss_bwd")
+        return dH, dW

@@ -1,0 +1,187 @@
+// C ABI entry points: argument validation, context management and dispatch to the
+// stage launchers.  Nothing here touches array data on the host.
+#include "common.cuh"
+
+#include <new>
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+
+int check_ctx(aero_ctx* ctx) {
+  if (!ctx) return AERO_ERR_INVALID;
+  if (cudaSetDevice(ctx->device) != cudaSuccess) return AERO_ERR_CUDA;
+  return AERO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int aero_version(void) { return 100; }
+
+const char* aero_error_string(int code) {
+  switch (code) {
+    case AERO_OK: return "ok";
+    case AERO_ERR_INVALID: return "invalid argument";
+    case AERO_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case AERO_ERR_WORKSPACE: return "workspace too small";
+    case AERO_ERR_CUDA: return "CUDA call failed";
+    default: return "unknown error";
+  }
+}
+
+void aero_cfg_default(aero_cfg* cfg) {
+  if (!cfg) return;
+  cfg->uniform_policy = AERO_UNIFORM_MASK;
+  cfg->rejection = 0;
+  cfg->k_ratio = 1;
+  cfg->rescue_S = 0;
+  cfg->n_explore = 8;
+  cfg->n_keep_uniform = 4;
+  cfg->stats_over = AERO_STATS_KEPT;
+  cfg->agg = AERO_TOKEN_MEAN;
+  cfg->denom = AERO_DENOM_SURVIVING;
+  cfg->alpha0 = 1.f;
+  cfg->beta0 = 1.f;
+  cfg->eps_std = 1e-6f;
+  cfg->clip_lo = 0.2f;
+  cfg->clip_hi = 0.2f;
+  cfg->seed = 0;
+  cfg->dtype = AERO_BF16;
+  cfg->reserved = 0;
+}
+
+int aero_create(aero_ctx** out, int device, void* cuda_stream) {
+  if (!out) return AERO_ERR_INVALID;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return AERO_ERR_CUDA;
+  AERO_CUDA_TRY(cudaSetDevice(device));
+  aero_ctx* ctx = new (std::nothrow) aero_ctx();
+  if (!ctx) return AERO_ERR_INVALID;
+  ctx->device = device;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  ctx->d_status = nullptr;
+  ctx->tmap_encode = nullptr;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return AERO_ERR_CUDA; }
+  ctx->sm_count = prop.multiProcessorCount;
+  if (cudaMalloc(&ctx->d_status, sizeof(uint32_t)) != cudaSuccess) { delete ctx; return AERO_ERR_CUDA; }
+  if (cudaMemset(ctx->d_status, 0, sizeof(uint32_t)) != cudaSuccess) {
+    cudaFree(ctx->d_status); delete ctx; return AERO_ERR_CUDA;
+  }
+  *out = ctx;
+  return AERO_OK;
+}
+
+int aero_destroy(aero_ctx* ctx) {
+  if (!ctx) return AERO_ERR_INVALID;
+  cudaSetDevice(ctx->device);
+  cudaFree(ctx->d_status);
+  delete ctx;
+  return AERO_OK;
+}
+
+int aero_set_stream(aero_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return AERO_ERR_INVALID;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  return AERO_OK;
+}
+
+int aero_last_status(aero_ctx* ctx, uint32_t* bits) {
+  if (!ctx || !bits) return AERO_ERR_INVALID;
+  int rc = check_ctx(ctx);
+  if (rc) return rc;
+  AERO_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+  AERO_CUDA_TRY(cudaMemcpy(bits, ctx->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost));
+  AERO_CUDA_TRY(cudaMemset(ctx->d_status, 0, sizeof(uint32_t)));
+  return AERO_OK;
+}
+
+size_t aero_group_workspace_bytes(int32_t P, int32_t R) { return aero_group_ws_bytes_impl(P, R); }
+
+int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
+                     const int32_t* go, const float* reward, const int64_t* cs,
+                     const uint32_t* key, const uint8_t* keep_in,
+                     const float* alpha_in, const float* beta_in,
+                     float* adv, float* w, uint8_t* keep, uint8_t* gmask, uint8_t* cat,
+                     float* u_tilde, float* alpha_out, float* beta_out,
+                     int32_t* kept_ids, int64_t* kept_tok_off, int64_t* counters,
+                     float* metrics, void* workspace, size_t workspace_bytes) {
+  int rc = check_ctx(ctx);
+  if (rc) return rc;
+  if (!cfg || P < 0 || R < 0) return AERO_ERR_INVALID;
+  if (!go || !cs || !kept_tok_off || !counters) return AERO_ERR_INVALID;
+  if (R > 0 && (!reward || !adv || !w || !keep || !kept_ids)) return AERO_ERR_INVALID;
+  if (P > 0 && (!gmask || !cat || !u_tilde || !alpha_out || !beta_out)) return AERO_ERR_INVALID;
+  if ((alpha_in == nullptr) != (beta_in == nullptr)) return AERO_ERR_INVALID;
+  if (cfg->k_ratio < 1 || cfg->n_explore < 1 || cfg->rescue_S < 0) return AERO_ERR_INVALID;
+  if (!workspace || !aligned256(workspace)) return AERO_ERR_INVALID;
+  if (workspace_bytes < aero_group_ws_bytes_impl(P, R)) return AERO_ERR_WORKSPACE;
+  return aero_group_stats_launch(ctx, cfg, P, R, go, reward, cs, key, keep_in, alpha_in, beta_in,
+                                 adv, w, keep, gmask, cat, u_tilde, alpha_out, beta_out,
+                                 kept_ids, kept_tok_off, counters, metrics, workspace);
+}
+
+size_t aero_fwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R) {
+  (void)d; (void)V;
+  size_t a = aero_fwd_ws_bytes_fp32(T, R), b = aero_fwd_ws_bytes_tc(T, R);
+  return a > b ? a : b;
+}
+
+int aero_grpo_loss_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                       const void* H, const void* W, const int32_t* y, const float* old_logp,
+                       const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                       float* logp, float* lse, float* g, float* loss, float* metrics,
+                       int accumulate, void* workspace, size_t workspace_bytes) {
+  int rc = check_ctx(ctx);
+  if (rc) return rc;
+  if (!cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
+  if (!W || !cs || !loss) return AERO_ERR_INVALID;
+  if (T > 0 && (!H || !y || !old_logp || !logp || !lse || !g)) return AERO_ERR_INVALID;
+  if (R > 0 && (!adv || !w || !keep)) return AERO_ERR_INVALID;
+  if (!workspace || !aligned256(workspace)) return AERO_ERR_INVALID;
+  if (workspace_bytes < aero_fwd_workspace_bytes(T, d, V, R)) return AERO_ERR_WORKSPACE;
+  if (cfg->dtype == AERO_FP32) {
+    return aero_fwd_fp32(ctx, cfg, T, d, V, R, static_cast<const float*>(H), static_cast<const float*>(W),
+                         y, old_logp, cs, adv, w, keep, logp, lse, g, loss, metrics, accumulate, workspace);
+  }
+  if (cfg->dtype != AERO_BF16) return AERO_ERR_UNSUPPORTED;
+  if (d % 64 != 0) return AERO_ERR_UNSUPPORTED;
+  if (!aligned16(H) || !aligned16(W)) return AERO_ERR_INVALID;
+  return aero_fwd_tc(ctx, cfg, T, d, V, R, H, W, y, old_logp, cs, adv, w, keep, logp, lse, g, loss,
+                     metrics, accumulate, workspace);
+}
+
+size_t aero_bwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R, int64_t chunk_tokens) {
+  return aero_bwd_ws_bytes_tc(T, d, V, R, chunk_tokens);
+}
+
+int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                       const void* H, const void* W, const int32_t* y,
+                       const int64_t* cs, const uint8_t* keep,
+                       const float* lse, const float* g, float grad_scale,
+                       void* dH, float* dW, int accumulate_dW,
+                       void* workspace, size_t workspace_bytes) {
+  int rc = check_ctx(ctx);
+  if (rc) return rc;
+  if (!cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
+  if (!W || !cs || !dW) return AERO_ERR_INVALID;
+  if (T > 0 && (!H || !y || !lse || !g || !dH)) return AERO_ERR_INVALID;
+  if (R > 0 && !keep) return AERO_ERR_INVALID;
+  if (cfg->dtype == AERO_FP32) {
+    return aero_bwd_fp32(ctx, cfg, T, d, V, R, static_cast<const float*>(H), static_cast<const float*>(W),
+                         y, cs, keep, lse, g, grad_scale, static_cast<float*>(dH), dW, accumulate_dW);
+  }
+  if (cfg->dtype != AERO_BF16) return AERO_ERR_UNSUPPORTED;
+  if (d % 64 != 0) return AERO_ERR_UNSUPPORTED;
+  if (!aligned16(H) || !aligned16(W) || !aligned16(dH) || !aligned16(dW)) return AERO_ERR_INVALID;
+  if (!workspace || !aligned256(workspace)) return AERO_ERR_INVALID;
+  if (workspace_bytes < aero_bwd_ws_bytes_tc(T, d, V, R, 128)) return AERO_ERR_WORKSPACE;
+  return aero_bwd_tc(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, grad_scale, dH, dW, accumulate_dW,
+                     workspace, workspace_bytes);
+}
+
+}  // extern "C"

@@ -1,0 +1,80 @@
+// Shared declarations of the library's translation units: context, status word,
+// error handling and the launch entry points each .cu file provides.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/aero.h"
+
+struct aero_ctx {
+  int device;
+  cudaStream_t stream;
+  uint32_t* d_status;     // device status word (OR of AERO_ST_* bits)
+  int sm_count;
+  void* tmap_encode;      // cuTensorMapEncodeTiled, resolved once through the runtime
+};
+
+#define AERO_CUDA_TRY(expr)                          \
+  do {                                               \
+    cudaError_t e__ = (expr);                        \
+    if (e__ != cudaSuccess) return AERO_ERR_CUDA;    \
+  } while (0)
+
+static inline size_t aero_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+__device__ __forceinline__ void aero_raise(uint32_t* status, uint32_t bits) {
+  if (bits) atomicOr(status, bits);
+}
+
+// ---- stage (a) ---------------------------------------------------------------------
+size_t aero_group_ws_bytes_impl(int32_t P, int32_t R);
+int aero_group_stats_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
+                            const int32_t* go, const float* reward, const int64_t* cs,
+                            const uint32_t* key, const uint8_t* keep_in,
+                            const float* alpha_in, const float* beta_in,
+                            float* adv, float* w, uint8_t* keep, uint8_t* gmask, uint8_t* cat,
+                            float* u_tilde, float* alpha_out, float* beta_out,
+                            int32_t* kept_ids, int64_t* kept_tok_off, int64_t* counters,
+                            float* metrics, void* ws);
+
+// ---- stage (b): helpers shared by the fp32 and the tensor-core paths ---------------
+// Row-tile work list over maximal runs of consecutive kept rollouts.
+struct aero_tiles {
+  int32_t* tile_row;      // [max_tiles] first token row of each tile
+  int32_t* tile_valid;    // [max_tiles] leading rows of the tile that belong to its run (1..tile_rows)
+  int32_t* n_tiles;       // [1]
+  int32_t max_tiles;
+};
+aero_tiles aero_carve_tiles(void* ws, int64_t T, int32_t R, int tile_rows);
+size_t aero_tiles_bytes(int64_t T, int32_t R, int tile_rows);
+int aero_build_tiles(aero_ctx* ctx, int64_t T, int32_t R, const int64_t* cs, const uint8_t* keep,
+                     int tile_rows, aero_tiles tiles);
+
+// Per-token surrogate terms and the fixed-order loss reduction.
+int aero_loss_finalize(aero_ctx* ctx, const double* partials, int n_partials, int stride,
+                       float* loss, float* metrics, int accumulate);
+
+// ---- stage (b): plain fp32 path -----------------------------------------------------
+size_t aero_fwd_ws_bytes_fp32(int64_t T, int32_t R);
+int aero_fwd_fp32(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                  const float* H, const float* W, const int32_t* y, const float* old_logp,
+                  const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                  float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws);
+int aero_bwd_fp32(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                  const float* H, const float* W, const int32_t* y, const int64_t* cs, const uint8_t* keep,
+                  const float* lse, const float* g, float grad_scale, float* dH, float* dW, int accumulate_dW);
+
+// ---- stage (b): tcgen05 / TMEM / TMA path (bf16) -------------------------------------
+size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t R);
+int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                const void* H, const void* W, const int32_t* y, const float* old_logp,
+                const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws);
+size_t aero_bwd_ws_bytes_tc(int64_t T, int32_t d, int32_t V, int32_t R, int64_t chunk_tokens);
+int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                const void* H, const void* W, const int32_t* y, const int64_t* cs, const uint8_t* keep,
+                const float* lse, const float* g, float grad_scale, void* dH, float* dW, int accumulate_dW,
+                void* ws, size_t ws_bytes);

@@ -1,0 +1,278 @@
+// Token-stationary lm_head kernel: for each 128-row token tile, walk all vocabulary
+// tiles of 256 columns; logits z = H W^T are accumulated in TMEM by tcgen05.mma from
+// bf16 operands staged by TMA, and consumed straight from TMEM by the epilogue warps.
+// The logits never reach shared or global memory.
+//
+//   MODE_FWD : online log-sum-exp over vocabulary tiles + target pick, then the clipped
+//              surrogate of Eq. 2 per token (logp, lse, g, per-tile loss partials).
+//   MODE_DZ  : dz = coef_t * (1[v == y_t] - exp(z - lse_t)) rounded to bf16 and stored to
+//              the chunk's scratch block (Eq. 3 through the softmax).
+//
+// Warp roles (192 threads, one CTA per SM): warps 0-3 epilogue (warp q reads TMEM lanes
+// 32q..32q+31, one token row per thread), warp 4 TMA producer, warp 5 MMA issuer and TMEM
+// owner.  Two 256-column TMEM accumulators let the MMA of vocabulary tile j+1 overlap
+// the epilogue of tile j.
+#pragma once
+
+#include "loss_common.cuh"
+#include "tc_ptx.cuh"
+
+namespace lmhead {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int THREADS = 192;
+constexpr int MODE_FWD = 0, MODE_DZ = 1;
+constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+
+struct Ctl {
+  uint64_t full[STAGES], empty[STAGES], tfull[2], tempty[2];
+  uint32_t tmem_base;
+  int abort;
+};
+constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + sizeof(Ctl);
+
+struct Params {
+  long long T;
+  int d, V, R;
+  const int32_t* tile_row;
+  const int32_t* tile_valid;
+  const int32_t* n_tiles;
+  int tile_begin, tile_end;     // this launch covers tiles [tile_begin, min(tile_end, *n_tiles))
+  const int32_t* y;
+  uint32_t* status;
+  // MODE_FWD
+  const float* old_logp;
+  const int64_t* cs;
+  const float* adv;
+  const float* w;
+  float clip_lo, clip_hi;
+  float* logp;
+  float* lse_out;
+  float* g_out;
+  double* partials;             // [tile][4 epilogue warps][kPartialStride]
+  // MODE_DZ
+  const float* lse_in;
+  const float* g_in;
+  float grad_scale;
+  __nv_bfloat16* dz;            // [(tile - tile_begin) * 128 + r][ldz]
+  long long ldz;
+};
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(THREADS, 1)
+lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW, const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  Ctl* ctl = reinterpret_cast<Ctl*>(smem + (size_t)STAGES * STAGE_BYTES);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&ctl->full[s], 1); tc::mbar_init(&ctl->empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { tc::mbar_init(&ctl->tfull[b], 1); tc::mbar_init(&ctl->tempty[b], 4); }
+    ctl->abort = 0;
+    tc::fence_barrier_init();
+  }
+  if (warp == 4 && lane == 0) { tc::prefetch_tmap(&tmH); tc::prefetch_tmap(&tmW); }
+  if (warp == 5) { tc::tmem_alloc(&ctl->tmem_base, 512); tc::tmem_relinquish(); }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = ctl->tmem_base;
+  volatile int* abort_flag = &ctl->abort;
+
+  const int n_tiles = min(*p.n_tiles, p.tile_end);
+  const int nkb = p.d / BK;
+  const int nvt = (p.V + BN - 1) / BN;
+
+  if (warp == 4) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = p.tile_begin + blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+        const int row0 = p.tile_row[tile];
+        for (int j = 0; ok && j < nvt; ++j) {
+          for (int kb = 0; kb < nkb; ++kb, ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (it / STAGES) & 1u;
+            if (!tc::mbar_wait(&ctl->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+            uint8_t* a_s = smem + (size_t)s * STAGE_BYTES;
+            tc::mbar_arrive_expect_tx(&ctl->full[s], STAGE_BYTES);
+            tc::tma_load_2d(a_s, &tmH, kb * BK, row0, &ctl->full[s]);
+            tc::tma_load_2d(a_s + A_BYTES, &tmW, kb * BK, j * BN, &ctl->full[s]);
+          }
+        }
+      }
+    }
+  } else if (warp == 5) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = tc::make_idesc_bf16(BM, BN, 0, 0);
+      uint32_t it = 0, at = 0;
+      bool ok = true;
+      for (int tile = p.tile_begin + blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+        for (int j = 0; ok && j < nvt; ++j, ++at) {
+          const uint32_t buf = at & 1u, aph = (at >> 1) & 1u;
+          if (!tc::mbar_wait(&ctl->tempty[buf], aph ^ 1u, abort_flag)) { ok = false; break; }
+          tc::tc_fence_after();
+          const uint32_t tmem_d = tmem_base + buf * BN;
+          for (int kb = 0; kb < nkb; ++kb, ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (it / STAGES) & 1u;
+            if (!tc::mbar_wait(&ctl->full[s], ph, abort_flag)) { ok = false; break; }
+            tc::tc_fence_after();
+            const uint32_t a_addr = tc::smem_u32(smem + (size_t)s * STAGE_BYTES);
+            const uint64_t adesc = tc::make_smem_desc(a_addr, 16, 1024);
+            const uint64_t bdesc = tc::make_smem_desc(a_addr + A_BYTES, 16, 1024);
+#pragma unroll
+            for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+              // advance 32 bytes (16 bf16) inside the 128-byte swizzle row: +2 in 16-byte units
+              tc::umma_bf16(tmem_d, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+            }
+            tc::umma_commit(&ctl->empty[s]);     // frees the stage when these MMAs retire
+          }
+          if (ok) tc::umma_commit(&ctl->tfull[buf]);
+        }
+      }
+    }
+  } else {
+    // ---------------- epilogue warps 0..3 ----------------
+    uint32_t at = 0;
+    bool ok = true;
+    const int r_in_tile = warp * 32 + lane;
+    for (int tile = p.tile_begin + blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+      const long long row = (long long)p.tile_row[tile] + r_in_tile;
+      const bool valid_row = r_in_tile < p.tile_valid[tile] && row < p.T;
+      int yt = -1;
+      if (valid_row) yt = p.y[row];
+      const bool bad_y = valid_row && (yt < 0 || yt >= p.V);
+      if (bad_y) { aero_raise(p.status, AERO_ST_BAD_TARGET); yt = -1; }
+      const bool live = valid_row && !bad_y;
+
+      float m2 = -INFINITY, l = 0.f, zy = 0.f;         // MODE_FWD running state (log2 domain)
+      float lse2 = 0.f, coef = 0.f;                    // MODE_DZ per-row constants
+      __nv_bfloat16* dz_row = nullptr;
+      if (MODE == MODE_DZ) {
+        if (live) { lse2 = p.lse_in[row] * kLog2e; coef = p.g_in[row] * p.grad_scale; }
+        dz_row = p.dz + ((long long)(tile - p.tile_begin) * BM + r_in_tile) * p.ldz;
+      }
+
+      for (int j = 0; ok && j < nvt; ++j, ++at) {
+        const uint32_t buf = at & 1u, aph = (at >> 1) & 1u;
+        // the TMEM loads below are warp-collective: take the decision for the whole warp
+        if (!__all_sync(0xffffffffu, tc::mbar_wait(&ctl->tfull[buf], aph, abort_flag))) { ok = false; break; }
+        tc::tc_fence_after();
+        const int col_base = j * BN;
+        const int ncol = min(BN, (MODE == MODE_DZ ? (int)p.ldz : p.V) - col_base);
+        const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + buf * BN;
+        for (int c = 0; c * 32 < ncol; ++c) {
+          uint32_t r[32];
+          __syncwarp();                     // the TMEM load is warp-collective
+          tc::tmem_ld_32x32(taddr + c * 32, r);
+          tc::tmem_ld_wait();
+          const int col0 = col_base + c * 32;
+          if (MODE == MODE_FWD) {
+            float z[32];
+#pragma unroll
+            for (int q = 0; q < 32; ++q) z[q] = __uint_as_float(r[q]);
+            if (col0 + 32 > p.V) {
+#pragma unroll
+              for (int q = 0; q < 32; ++q) if (col0 + q >= p.V) z[q] = -INFINITY;
+            }
+            float cmax = z[0];
+#pragma unroll
+            for (int q = 1; q < 32; ++q) cmax = fmaxf(cmax, z[q]);
+            const float m2n = fmaxf(m2, cmax * kLog2e);
+            float acc = 0.f;
+#pragma unroll
+            for (int q = 0; q < 32; ++q) acc += ex2(fmaf(z[q], kLog2e, -m2n));
+            l = fmaf(l, ex2(m2 - m2n), acc);
+            m2 = m2n;
+            if ((unsigned)(yt - col0) < 32u) {
+              const int sel = yt - col0;
+#pragma unroll
+              for (int q = 0; q < 32; ++q) if (q == sel) zy = z[q];
+            }
+          } else {
+            uint32_t pk[16];
+#pragma unroll
+            for (int q = 0; q < 32; q += 2) {
+              float v0 = -coef * ex2(fmaf(__uint_as_float(r[q]), kLog2e, -lse2));
+              float v1 = -coef * ex2(fmaf(__uint_as_float(r[q + 1]), kLog2e, -lse2));
+              if (col0 + q == yt) v0 += coef;
+              if (col0 + q + 1 == yt) v1 += coef;
+              if (!live || col0 + q >= p.V) v0 = 0.f;
+              if (!live || col0 + q + 1 >= p.V) v1 = 0.f;
+              pk[q >> 1] = pack_bf16(v0, v1);
+            }
+            uint4* dst = reinterpret_cast<uint4*>(dz_row + col0);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) dst[q] = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+          }
+        }
+        tc::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&ctl->tempty[buf]);
+      }
+
+      if (MODE == MODE_FWD && ok) {
+        double part[kPartialStride] = {0.0, 0.0, 0.0, 0.0, 0.0};
+        if (live) {
+          const float ls = (m2 + __log2f(l)) * kLn2;
+          const float lp = zy - ls;
+          const int i = aero_owner(p.cs, p.R, row);
+          const float old = p.old_logp[row];
+          const float wi = p.w[i];
+          const SurrogateOut so = aero_surrogate(lp, old, p.adv[i], wi, p.clip_lo, p.clip_hi);
+          p.logp[row] = lp;
+          p.lse_out[row] = ls;
+          p.g_out[row] = so.g;
+          part[0] = (double)wi * (double)so.s;
+          part[1] = so.clipped;
+          part[2] = so.rho;
+          part[3] = (double)old - (double)lp;
+          part[4] = 1.0;
+        }
+        // fixed-shape reduction: a shuffle tree per warp; the four warps' records are
+        // added later by the finalising kernel in a fixed order
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+          for (int k = 0; k < kPartialStride; ++k) part[k] += __shfl_xor_sync(0xffffffffu, part[k], o);
+        if (lane == 0)
+          for (int k = 0; k < kPartialStride; ++k)
+            p.partials[((size_t)tile * 4 + warp) * kPartialStride + k] = part[k];
+      }
+    }
+  }
+
+  // ---------------- teardown ----------------
+  __syncwarp();
+  if (*abort_flag) {
+    // a wait gave up: let copies and MMAs already in flight land before shared memory and
+    // TMEM are released
+    const unsigned long long t0 = tc::globaltimer_ns();
+    while (tc::globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) aero_raise(p.status, AERO_ST_TIMEOUT);
+  if (warp == 5) {
+    tc::tc_fence_after();
+    tc::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace lmhead

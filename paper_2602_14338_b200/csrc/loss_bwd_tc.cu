@@ -1,0 +1,107 @@
+// Stage (b) backward on the tensor-core path.  Token tiles are processed in chunks:
+// for each chunk the lm_head kernel recomputes the logits and writes the bf16 dz block,
+// then two GEMM launches produce the chunk's rows of dH and add the chunk's share of dW.
+#include "gemm_bwd_kernel.cuh"
+#include "lmhead_kernel.cuh"
+#include "tmap.cuh"
+
+namespace {
+
+inline long long ldz_of(int32_t V) { return ((long long)V + 63) / 64 * 64; }
+
+// dH rows of dropped rollouts are defined to be zero; one warp per row.
+__global__ void __launch_bounds__(256) zero_dropped_rows_kernel(long long T, int d, int R,
+                                                                const int64_t* __restrict__ cs,
+                                                                const uint8_t* __restrict__ keep,
+                                                                __nv_bfloat16* __restrict__ dH) {
+  const int lane = threadIdx.x & 31;
+  const long long warp0 = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const long long nwarps = (long long)gridDim.x * 8;
+  for (long long t = warp0; t < T; t += nwarps) {
+    const int i = aero_owner(cs, R, t);
+    if (keep[i]) continue;
+    uint4* row = reinterpret_cast<uint4*>(dH + t * d);
+    for (int k = lane; k < d / 8; k += 32) row[k] = make_uint4(0, 0, 0, 0);
+  }
+}
+
+}  // namespace
+
+size_t aero_bwd_ws_bytes_tc(int64_t T, int32_t d, int32_t V, int32_t R, int64_t chunk_tokens) {
+  (void)d;
+  if (chunk_tokens < 128) chunk_tokens = 128;
+  const size_t rows = (size_t)((chunk_tokens + 127) / 128 * 128);
+  return aero_tiles_bytes(T, R, lmhead::BM) + aero_align_up(rows * (size_t)ldz_of(V) * 2, 256);
+}
+
+int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                const void* H, const void* W, const int32_t* y, const int64_t* cs, const uint8_t* keep,
+                const float* lse, const float* g, float grad_scale, void* dH, float* dW, int accumulate_dW,
+                void* ws, size_t ws_bytes) {
+  (void)cfg;
+  if (!accumulate_dW) AERO_CUDA_TRY(cudaMemsetAsync(dW, 0, (size_t)V * d * sizeof(float), ctx->stream));
+  if (T == 0 || R == 0) return AERO_OK;
+
+  const long long ldz = ldz_of(V);
+  aero_tiles tiles = aero_carve_tiles(ws, T, R, lmhead::BM);
+  const size_t tiles_bytes = aero_tiles_bytes(T, R, lmhead::BM);
+  __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + tiles_bytes);
+  long long tpc = (long long)((ws_bytes - tiles_bytes) / ((size_t)lmhead::BM * (size_t)ldz * 2));
+  if (tpc < 1) return AERO_ERR_WORKSPACE;
+  if (tpc > tiles.max_tiles) tpc = tiles.max_tiles;
+  if (tpc > ctx->sm_count) tpc = tpc / ctx->sm_count * ctx->sm_count;   // whole waves of token tiles
+
+  int rc = aero_build_tiles(ctx, T, R, cs, keep, lmhead::BM, tiles);
+  if (rc) return rc;
+  {
+    const long long blocks = (T + 7) / 8;
+    zero_dropped_rows_kernel<<<(int)(blocks < 4096 ? blocks : 4096), 256, 0, ctx->stream>>>(
+        T, d, R, cs, keep, static_cast<__nv_bfloat16*>(dH));
+    AERO_CUDA_TRY(cudaGetLastError());
+  }
+
+  const CUtensorMapDataType BF = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+  CUtensorMap tmH_k, tmW_k, tmDZ_k, tmW_mn, tmDZ_mn, tmH_mn;
+  const uint64_t dz_rows = (uint64_t)tpc * lmhead::BM;
+  // K-major views (inner extent 64 = one 128-byte swizzle row) for the recompute and for dz as A of dH
+  if ((rc = aero_make_tmap_2d(ctx, &tmH_k, BF, 2, H, T, d, d, lmhead::BM, 64))) return rc;
+  if ((rc = aero_make_tmap_2d(ctx, &tmW_k, BF, 2, W, V, d, d, lmhead::BN, 64))) return rc;
+  if ((rc = aero_make_tmap_2d(ctx, &tmDZ_k, BF, 2, dz, dz_rows, ldz, ldz, gemmbwd::BM, 64))) return rc;
+  // MN-major views: 64 x 64 boxes
+  if ((rc = aero_make_tmap_2d(ctx, &tmW_mn, BF, 2, W, V, d, d, 64, 64))) return rc;
+  if ((rc = aero_make_tmap_2d(ctx, &tmDZ_mn, BF, 2, dz, dz_rows, ldz, ldz, 64, 64))) return rc;
+  if ((rc = aero_make_tmap_2d(ctx, &tmH_mn, BF, 2, H, T, d, d, 64, 64))) return rc;
+
+  auto k_dz = lmhead::lmhead_kernel<lmhead::MODE_DZ>;
+  auto k_dh = gemmbwd::gemm_kernel<gemmbwd::KIND_DH>;
+  auto k_dw = gemmbwd::gemm_kernel<gemmbwd::KIND_DW>;
+  AERO_CUDA_TRY(cudaFuncSetAttribute(k_dz, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lmhead::SMEM_BYTES));
+  AERO_CUDA_TRY(cudaFuncSetAttribute(k_dh, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::SMEM_BYTES));
+  AERO_CUDA_TRY(cudaFuncSetAttribute(k_dw, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::SMEM_BYTES));
+
+  const int n_nt = (d + gemmbwd::BN - 1) / gemmbwd::BN;
+  const long long dw_units = (long long)((V + gemmbwd::BM - 1) / gemmbwd::BM) * n_nt;
+  for (long long begin = 0; begin < tiles.max_tiles; begin += tpc) {
+    lmhead::Params lp = {};
+    lp.T = T; lp.d = d; lp.V = V; lp.R = R;
+    lp.tile_row = tiles.tile_row; lp.tile_valid = tiles.tile_valid; lp.n_tiles = tiles.n_tiles;
+    lp.tile_begin = (int)begin; lp.tile_end = (int)(begin + tpc);
+    lp.y = y; lp.status = ctx->d_status;
+    lp.lse_in = lse; lp.g_in = g; lp.grad_scale = grad_scale; lp.dz = dz; lp.ldz = ldz;
+    const int grid_dz = (int)(tpc < ctx->sm_count ? tpc : ctx->sm_count);
+    k_dz<<<grid_dz, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH_k, tmW_k, lp);
+
+    gemmbwd::Params gp = {};
+    gp.T = T; gp.d = d; gp.V = V; gp.ldz = ldz;
+    gp.tile_row = tiles.tile_row; gp.tile_valid = tiles.tile_valid; gp.n_tiles = tiles.n_tiles;
+    gp.tile_begin = (int)begin; gp.tpc = (int)tpc;
+    gp.dH = static_cast<__nv_bfloat16*>(dH); gp.dW = dW; gp.status = ctx->d_status;
+    const long long dh_units = tpc * n_nt;
+    k_dh<<<(int)(dh_units < ctx->sm_count ? dh_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
+           ctx->stream>>>(tmDZ_k, tmW_mn, gp);
+    k_dw<<<(int)(dw_units < ctx->sm_count ? dw_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
+           ctx->stream>>>(tmDZ_mn, tmH_mn, gp);
+    AERO_CUDA_TRY(cudaGetLastError());
+  }
+  return AERO_OK;
+}

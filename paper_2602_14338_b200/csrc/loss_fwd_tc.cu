@@ -1,0 +1,67 @@
+// Stage (b) forward on the tensor-core path: tile list, fused lm_head kernel in
+// forward mode, fixed-order reduction of the loss partials.
+#include "lmhead_kernel.cuh"
+#include "tmap.cuh"
+
+namespace {
+
+struct FwdWs {
+  aero_tiles tiles;
+  double* partials;
+  size_t n_partials;
+};
+
+FwdWs carve_fwd(void* ws, int64_t T, int32_t R) {
+  FwdWs f;
+  f.tiles = aero_carve_tiles(ws, T, R, lmhead::BM);
+  char* p = static_cast<char*>(ws) + aero_tiles_bytes(T, R, lmhead::BM);
+  f.partials = reinterpret_cast<double*>(p);
+  f.n_partials = (size_t)f.tiles.max_tiles * 4;
+  return f;
+}
+
+}  // namespace
+
+size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t R) {
+  const size_t mt = (size_t)(T / lmhead::BM) + (size_t)R + 2;
+  return aero_tiles_bytes(T, R, lmhead::BM) + aero_align_up(mt * 4 * kPartialStride * sizeof(double), 256);
+}
+
+int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                const void* H, const void* W, const int32_t* y, const float* old_logp,
+                const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws) {
+  FwdWs f = carve_fwd(ws, T, R);
+  AERO_CUDA_TRY(cudaMemsetAsync(f.partials, 0, f.n_partials * kPartialStride * sizeof(double), ctx->stream));
+  if (T > 0) {
+    AERO_CUDA_TRY(cudaMemsetAsync(logp, 0, (size_t)T * sizeof(float), ctx->stream));
+    AERO_CUDA_TRY(cudaMemsetAsync(lse, 0, (size_t)T * sizeof(float), ctx->stream));
+    AERO_CUDA_TRY(cudaMemsetAsync(g, 0, (size_t)T * sizeof(float), ctx->stream));
+  }
+  int rc = aero_build_tiles(ctx, T, R, cs, keep, lmhead::BM, f.tiles);
+  if (rc) return rc;
+  if (T > 0 && R > 0) {
+    CUtensorMap tmH, tmW;
+    rc = aero_make_tmap_2d(ctx, &tmH, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, H, (uint64_t)T, (uint64_t)d, (uint64_t)d,
+                           lmhead::BM, lmhead::BK);
+    if (rc) return rc;
+    rc = aero_make_tmap_2d(ctx, &tmW, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)V, (uint64_t)d, (uint64_t)d,
+                           lmhead::BN, lmhead::BK);
+    if (rc) return rc;
+    lmhead::Params p = {};
+    p.T = T; p.d = d; p.V = V; p.R = R;
+    p.tile_row = f.tiles.tile_row; p.tile_valid = f.tiles.tile_valid; p.n_tiles = f.tiles.n_tiles;
+    p.tile_begin = 0; p.tile_end = f.tiles.max_tiles;
+    p.y = y; p.status = ctx->d_status;
+    p.old_logp = old_logp; p.cs = cs; p.adv = adv; p.w = w;
+    p.clip_lo = cfg->clip_lo; p.clip_hi = cfg->clip_hi;
+    p.logp = logp; p.lse_out = lse; p.g_out = g; p.partials = f.partials;
+    auto kern = lmhead::lmhead_kernel<lmhead::MODE_FWD>;
+    AERO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lmhead::SMEM_BYTES));
+    const int64_t upper = T / lmhead::BM + R + 1;
+    const int grid = (int)(upper < ctx->sm_count ? upper : ctx->sm_count);
+    kern<<<grid, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH, tmW, p);
+    AERO_CUDA_TRY(cudaGetLastError());
+  }
+  return aero_loss_finalize(ctx, f.partials, (int)f.n_partials, kPartialStride, loss, metrics, accumulate);
+}

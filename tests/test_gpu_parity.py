@@ -1,0 +1,278 @@
+"""GPU parity tests: the CUDA library, called through its C ABI, against the fp64 oracle
+on the same seeded inputs.  Tolerances are the ones the path is specified with:
+integer outputs bit-exact; per-token log-probs abs <= 1e-2; loss rel <= 1e-3; dH and dW
+relative L2 <= 1e-2 (bf16 path).  The fp32 path is held to 1e-4."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import aero_oracle as O
+from paper_2602_14338_b200 import binding as B
+from paper_2602_14338_b200 import synth
+from tests import aero_testlib as TL
+
+pytestmark = pytest.mark.gpu
+
+LOGP_ABS, LOSS_REL, GRAD_L2 = 1e-2, 1e-3, 1e-2
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = B.Context(0)
+    yield c
+    assert c.last_status() == 0
+    c.close()
+
+
+# ------------------------------------------------------------------ stage (a)
+GROUP_MODES = [
+    dict(),
+    dict(uniform_policy=O.UNIFORM_BAYES),
+    dict(uniform_policy=O.UNIFORM_BAYES, rejection=1),
+    dict(uniform_policy=O.UNIFORM_BAYES, rejection=1, k_ratio=2, agg=O.AGG_SEQ_MEAN),
+    dict(rejection=1, stats_over=O.STATS_ALL, denom=O.DENOM_ALL),
+    dict(uniform_policy=O.UNIFORM_BAYES, rejection=1, rescue_S=4, n_keep_uniform=0, agg=O.AGG_SEQ_MEAN, denom=O.DENOM_ALL),
+]
+
+
+@pytest.mark.parametrize("config", [0, 1, 2, 3, 4])
+@pytest.mark.parametrize("mode", range(len(GROUP_MODES)))
+def test_group_stats_matches_oracle(ctx, config, mode):
+    wl = synth.WORKLOADS[config]
+    st = synth.make_structure(wl)
+    ocfg = O.Cfg(seed=wl.seed, **GROUP_MODES[mode])
+    ref = O.group_stats(ocfg, st.go, st.reward, st.cs, key=st.key, alpha_in=st.alpha, beta_in=st.beta)
+    _, out = TL.run_group_gpu(ctx, TL.lib_cfg(ocfg, "bf16"), st)
+    TL.check_group(out, ref, len(st.reward), len(st.go) - 1)
+    assert ctx.last_status() == 0
+
+
+def test_group_stats_default_key_and_keep_in(ctx):
+    wl = synth.scaled(synth.WORKLOADS[3], P=300, n_lo=1, n_hi=40, seed=77)   # groups longer than a team
+    st = synth.make_structure(wl)
+    rng = np.random.default_rng(5)
+    keep_in = (rng.random(len(st.reward)) < 0.8).astype(np.uint8)
+    ocfg = O.Cfg(seed=991, uniform_policy=O.UNIFORM_BAYES, rejection=1)
+    ref = O.group_stats(ocfg, st.go, st.reward, st.cs, keep_in=keep_in, alpha_in=st.alpha, beta_in=st.beta)
+    _, out = TL.run_group_gpu(ctx, TL.lib_cfg(ocfg, "bf16"), st, use_key=False, keep_in=TL.dev(keep_in))
+    TL.check_group(out, ref, len(st.reward), len(st.go) - 1)
+
+
+def test_group_stats_ties_and_small_groups(ctx):
+    wl = synth.scaled(synth.WORKLOADS[3], P=500, n_lo=1, n_hi=6, seed=78)
+    st = synth.make_structure(wl)
+    st.key[:] = st.key % 3            # heavy ties: the index must break them
+    ocfg = O.Cfg(uniform_policy=O.UNIFORM_BAYES, rejection=1, n_keep_uniform=2)
+    ref = O.group_stats(ocfg, st.go, st.reward, st.cs, key=st.key, alpha_in=st.alpha, beta_in=st.beta)
+    _, out = TL.run_group_gpu(ctx, TL.lib_cfg(ocfg, "bf16"), st)
+    TL.check_group(out, ref, len(st.reward), len(st.go) - 1)
+
+
+def test_group_stats_empty_inputs_and_status_bits(ctx):
+    cfg = B.cfg_default()
+    go = torch.zeros(1, dtype=torch.int32, device="cuda")
+    cs = torch.zeros(1, dtype=torch.int64, device="cuda")
+    rw = torch.zeros(0, dtype=torch.float32, device="cuda")
+    out = ctx.group_stats(cfg, go, rw, cs)
+    assert out["counters"].cpu().tolist() == [0] * 8 and int(out["kept_tok_off"][0]) == 0
+    # empty groups among real ones
+    go = torch.tensor([0, 0, 3, 3], dtype=torch.int32, device="cuda")
+    rw = torch.tensor([1, 0, 0], dtype=torch.float32, device="cuda")
+    cs = torch.tensor([0, 2, 4, 6], dtype=torch.int64, device="cuda")
+    out = ctx.group_stats(cfg, go, rw, cs)
+    ref = O.group_stats(O.Cfg(), go.cpu().numpy(), rw.cpu().numpy(), cs.cpu().numpy())
+    TL.check_group(out, ref, 3, 3)
+    assert ctx.last_status() == 0
+    # a non-binary reward and an empty rollout raise status bits and nothing traps
+    rw2 = torch.tensor([1, 0.25, 0], dtype=torch.float32, device="cuda")
+    cs2 = torch.tensor([0, 2, 2, 6], dtype=torch.int64, device="cuda")
+    ctx.group_stats(cfg, go, rw2, cs2)
+    bits = ctx.last_status()
+    assert bits & B.AERO_ST_BAD_REWARD and bits & B.AERO_ST_EMPTY_ROLLOUT
+    assert ctx.last_status() == 0
+
+
+def test_group_stats_large_properties(ctx):
+    """2^20 prompts (too many for the oracle's loops): exact invariants plus sampled prompts."""
+    wl = synth.scaled(synth.WORKLOADS[3], P=1 << 20, seed=4242, len_median=64.0, len_cap=256)
+    st = synth.make_structure(wl)
+    ocfg = O.Cfg(uniform_policy=O.UNIFORM_BAYES, rejection=1)
+    _, out = TL.run_group_gpu(ctx, TL.lib_cfg(ocfg, "bf16"), st)
+    g = {k: v.cpu().numpy() for k, v in out.items()}
+    R, P = len(st.reward), wl.P
+    lens = st.cs[1:] - st.cs[:-1]
+    keep = g["keep"][:R].astype(bool)
+    assert g["counters"][0] == keep.sum() and g["counters"][1] == lens[keep].sum()
+    assert np.array_equal(g["kept_ids"][:keep.sum()], np.nonzero(keep)[0])
+    assert np.array_equal(g["kept_tok_off"][1:keep.sum() + 1], np.cumsum(lens[keep]))
+    assert abs(float((g["w"][:R].astype(np.float64) * lens).sum()) - 1.0) < 1e-4
+    rng = np.random.default_rng(0)
+    for p in rng.integers(0, P, 200):
+        a, b = st.go[p], st.go[p + 1]
+        sub_go = np.array([0, b - a], np.int32)
+        sub_cs = (st.cs[a:b + 1] - st.cs[a]).astype(np.int64)
+        ref = O.group_stats(ocfg, sub_go, st.reward[a:b], sub_cs, key=st.key[a:b],
+                            alpha_in=st.alpha[p:p + 1], beta_in=st.beta[p:p + 1])
+        assert np.array_equal(g["keep"][a:b], ref["keep"])
+        np.testing.assert_allclose(g["adv"][a:b], ref["adv"], rtol=2e-5, atol=1e-6)
+        assert g["cat"][p] == ref["cat"][0]
+
+
+# ------------------------------------------------------------------ stage (b)
+def run_fwd_bwd(ctx, batch, dtype, grad_scale=1.0, chunk_tokens=None):
+    cfg = TL.lib_cfg(batch.ocfg, dtype)
+    dv = batch.to_device()
+    f = ctx.grpo_loss_fwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"], dv["keep"])
+    dH, dW = ctx.grpo_loss_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], dv["keep"], f["lse"], f["g"],
+                               grad_scale=grad_scale, chunk_tokens=chunk_tokens)
+    torch.cuda.synchronize()
+    return cfg, dv, f, dH, dW
+
+
+def check_fwd(batch, f, ref, logp_abs, loss_rel, g_rtol):
+    T = batch.T
+    owner = O.token_rollout(batch.st.cs, T)
+    kept = batch.ref_g["keep"][owner] != 0
+    logp = f["logp"][:T].cpu().numpy()
+    lse = f["lse"][:T].cpu().numpy()
+    g = f["g"][:T].cpu().numpy()
+    assert np.abs(logp - ref["logp"]).max() <= logp_abs
+    assert np.abs(lse - ref["lse"]).max() <= logp_abs
+    assert not logp[~kept].any() and not g[~kept].any() and not lse[~kept].any()
+    assert (logp[kept] <= 1e-6).all()
+    loss = float(f["loss"].item())
+    assert abs(loss - ref["loss"]) <= loss_rel * abs(ref["loss"]) + 1e-7
+    # clip indicators may legitimately flip when rho sits within rounding of a clip edge
+    rho = ref["rho"]
+    edge = (np.abs(rho - (1 + batch.ocfg.clip_hi)) < 1e-3) | (np.abs(rho - (1 - batch.ocfg.clip_lo)) < 1e-3)
+    ok = ~edge
+    np.testing.assert_allclose(g[ok], ref["g"][ok], rtol=g_rtol, atol=1e-12)
+    met = f["metrics"].cpu().numpy()
+    assert met[3] == kept.sum()
+    assert abs(met[0] - ref["metrics"][0]) <= (edge.sum() + 0.5) / max(kept.sum(), 1)
+    assert abs(met[1] - ref["metrics"][1]) < 1e-3
+
+
+def test_tiny_workload_fp32(ctx):
+    wl = synth.WORKLOADS[0]
+    batch = TL.Batch(wl, TL.cfg_for(wl))
+    assert batch.ref_g["gmask"][0] == 0 and batch.ref_g["gmask"][1] == 0      # forced uniform groups
+    ref = batch.oracle_fwd()
+    cfg, dv, f, dH, dW = run_fwd_bwd(ctx, batch, "fp32", grad_scale=1.5)
+    check_fwd(batch, f, ref, 1e-4, 1e-4, 1e-3)
+    rdH, rdW = batch.oracle_bwd(ref, 1.5)
+    assert TL.rel_l2(dH.cpu().numpy(), rdH) < 1e-4
+    assert TL.rel_l2(dW.cpu().numpy(), rdW) < 1e-4
+    assert ctx.last_status() == 0
+
+
+BF16_CASES = {
+    # name: (workload overrides, cfg overrides, peak strength)
+    "tiny_bf16": (dict(dtype="bf16"), dict(), 0.0),
+    "ragged_tail": (dict(P=6, n_lo=3, n_hi=9, d=128, V=1000, len_median=70.0, len_cap=300, dtype="bf16", seed=11),
+                    dict(), 0.0),
+    "aero_dropped": (dict(P=24, n_lo=2, n_hi=12, d=192, V=3001, len_median=40.0, len_cap=160, dtype="bf16",
+                          aero=True, old_noise=0.15, seed=12), dict(uniform_policy=O.UNIFORM_BAYES, rejection=1), 0.0),
+    "seq_mean_clipped": (dict(P=8, n_lo=4, n_hi=4, d=256, V=2048, len_median=50.0, len_cap=100, dtype="bf16",
+                              old_noise=0.25, seed=13), dict(agg=O.AGG_SEQ_MEAN), 0.0),
+    "peaked": (dict(P=6, n_lo=4, n_hi=8, d=128, V=4096, len_median=60.0, len_cap=200, dtype="bf16", seed=14),
+               dict(), 45.0),
+}
+
+
+@pytest.mark.parametrize("name", list(BF16_CASES))
+def test_bf16_tensor_core_path(ctx, name):
+    over, cover, peak = BF16_CASES[name]
+    base = synth.WORKLOADS[0] if name == "tiny_bf16" else synth.WORKLOADS[1]
+    wl = synth.scaled(base, **over)
+    batch = TL.Batch(wl, O.Cfg(seed=wl.seed, **cover), peak=peak)
+    ref = batch.oracle_fwd()
+    cfg, dv, f, dH, dW = run_fwd_bwd(ctx, batch, "bf16")
+    assert ctx.last_status() == 0
+    check_fwd(batch, f, ref, LOGP_ABS, LOSS_REL, 2e-2)
+    # backward from the oracle's own lse and g, so that only the backward is under test ...
+    rdH, rdW = batch.oracle_bwd(ref)
+    dH2, dW2 = ctx.grpo_loss_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], dv["keep"],
+                                 TL.dev(ref["lse"], torch.float32), TL.dev(ref["g"], torch.float32))
+    assert TL.rel_l2(dH2.float().cpu().numpy(), rdH) < GRAD_L2
+    assert TL.rel_l2(dW2.cpu().numpy(), rdW) < GRAD_L2
+    # ... and end to end from the library's forward outputs
+    assert TL.rel_l2(dH.float().cpu().numpy(), rdH) < GRAD_L2
+    assert TL.rel_l2(dW.cpu().numpy(), rdW) < GRAD_L2
+    # invariants: columns of dW sum to zero; dropped rows of dH are zero
+    owner = O.token_rollout(batch.st.cs, batch.T)
+    dropped = batch.ref_g["keep"][owner] == 0
+    assert not dH.float().cpu().numpy()[dropped].any()
+    col = np.abs(dW.double().cpu().numpy().sum(axis=0)).max()
+    assert col <= 2e-2 * np.abs(rdW).sum(axis=0).max() + 1e-9
+    if peak > 0:
+        # the softmax part alone (one-hot part removed) must also agree: it is what a kernel
+        # that dropped the softmax term would get wrong
+        Wm, y, g = batch.W, batch.st.y, ref["g"]
+        soft_ref = rdH - g[:, None] * Wm[y]
+        soft_gpu = dH2.float().cpu().numpy() - g[:, None] * Wm[y]
+        live = g != 0
+        assert np.linalg.norm(soft_ref[live]) > 0.05 * np.linalg.norm(rdH[live])
+        assert TL.rel_l2(soft_gpu[live], soft_ref[live]) < 3e-2
+        never_hit = np.setdiff1d(np.arange(wl.V), y)
+        assert TL.rel_l2(dW2.cpu().numpy()[never_hit], rdW[never_hit]) < GRAD_L2
+
+
+def test_bwd_chunking_and_accumulation(ctx):
+    over, cover, _ = BF16_CASES["aero_dropped"]
+    wl = synth.scaled(synth.WORKLOADS[1], **over)
+    batch = TL.Batch(wl, O.Cfg(seed=wl.seed, **cover))
+    cfg, dv, f, dH, dW = run_fwd_bwd(ctx, batch, "bf16")
+    # one 128-row tile per chunk: many chunks, dW accumulated across them
+    dH1, dW1 = ctx.grpo_loss_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], dv["keep"], f["lse"], f["g"],
+                                 chunk_tokens=128, workspace=torch.empty(
+                                     ctx.bwd_workspace_bytes(batch.T, wl.d, wl.V, batch.R, 128), dtype=torch.uint8, device="cuda"))
+    assert torch.equal(dH1, dH)
+    assert TL.rel_l2(dW1.cpu().numpy(), dW.cpu().numpy()) < 1e-5
+    # accumulate_dW adds to what is there
+    dW2 = dW.clone()
+    ctx.grpo_loss_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], dv["keep"], f["lse"], f["g"], dW=dW2, accumulate_dW=True)
+    assert TL.rel_l2(dW2.cpu().numpy(), 2 * dW.cpu().numpy()) < 1e-5
+    # the loss reduction is order-fixed: identical bits on a second run; accumulate adds
+    f2 = ctx.grpo_loss_fwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"], dv["keep"])
+    assert torch.equal(f2["loss"], f["loss"]) and torch.equal(f2["logp"], f["logp"])
+    ctx.grpo_loss_fwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"], dv["keep"],
+                      out=f2, accumulate=True)
+    assert abs(f2["loss"].item() - 2 * f["loss"].item()) <= 1e-6 * abs(f["loss"].item()) + 1e-9
+    assert ctx.last_status() == 0
+
+
+def test_all_dropped_and_bad_target(ctx):
+    wl = synth.scaled(synth.WORKLOADS[1], P=3, n_lo=4, n_hi=4, d=64, V=300, len_median=30.0, len_cap=64, seed=21)
+    batch = TL.Batch(wl, O.Cfg())
+    cfg = TL.lib_cfg(batch.ocfg, "bf16")
+    dv = batch.to_device()
+    zero_keep = torch.zeros_like(dv["keep"])
+    f = ctx.grpo_loss_fwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"], zero_keep)
+    dH, dW = ctx.grpo_loss_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], zero_keep, f["lse"], f["g"])
+    assert f["loss"].item() == 0.0 and not dH.float().abs().sum().item() and not dW.abs().sum().item()
+    assert ctx.last_status() == 0
+    # an out-of-range target is reported and its row skipped
+    keep = torch.ones_like(dv["keep"])
+    y = dv["y"].clone()
+    y[5] = wl.V + 7
+    f = ctx.grpo_loss_fwd(cfg, dv["H"], dv["W"], y, dv["old"], dv["cs"], dv["adv"], dv["w"], keep)
+    assert ctx.last_status() & B.AERO_ST_BAD_TARGET
+    assert f["g"][5].item() == 0.0 and f["logp"][5].item() == 0.0
+
+
+def test_full_width_qwen_1p5b_shape(ctx):
+    """Full d = 1536 and V = 151936 of the Qwen2.5-Math-1.5B workload on a batch the oracle can
+    finish: 8 rollouts of ~80 tokens (several row tiles, 594 vocabulary tiles with the ragged
+    last one).  Every output against the oracle; dW on the target rows plus 1024 random rows."""
+    wl = synth.scaled(synth.WORKLOADS[1], P=2, n_lo=4, n_hi=4, len_median=80.0, len_cap=200, seed=31)
+    batch = TL.Batch(wl, TL.cfg_for(wl, uniform_policy=O.UNIFORM_BAYES))
+    assert batch.T >= 384
+    ref = batch.oracle_fwd()
+    cfg, dv, f, dH, dW = run_fwd_bwd(ctx, batch, "bf16")
+    assert ctx.last_status() == 0
+    check_fwd(batch, f, ref, LOGP_ABS, LOSS_REL, 2e-2)
+    rows = np.unique(np.concatenate([batch.st.y[:64], np.random.default_rng(1).integers(0, wl.V, 1024)]))
+    rdH, rdW = batch.oracle_bwd(ref, dw_rows=rows)
+    assert TL.rel_l2(dH.float().cpu().numpy(), rdH) < GRAD_L2
+    assert TL.rel_l2(dW.cpu().numpy()[rows], rdW) < GRAD_L2
