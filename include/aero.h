@@ -236,6 +236,38 @@ int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d,
                        void* dH, float* dW, int accumulate_dW,
                        void* workspace, size_t workspace_bytes);
 
+/* ------------------------------------------------------------------------------
+ * One whole step of the path from HOST buffers: stage (a), forward and backward
+ * (the same operations and citations as the three calls above), for callers whose
+ * rollout batch lives in host memory.  The call copies the batch to the device,
+ * runs aero_group_stats, aero_grpo_loss_fwd and aero_grpo_loss_bwd on the context's
+ * stream, copies the scalars back and synchronises the stream before returning.
+ *
+ * HOST inputs (pinned memory makes the copies asynchronous): go_h [P+1] i32,
+ *   reward_h [R] f32, cs_h [R+1] i64, key_h [R] u32 or NULL, alpha_h/beta_h [P] f32 or
+ *   both NULL, H_h [T,d] (cfg->dtype), y_h [T] i32, old_logp_h [T] f32.
+ * DEVICE arrays: W [V,d] (the resident weight), dH [T,d] and dW [V,d] f32 (outputs, as in
+ *   aero_grpo_loss_bwd), workspace of at least aero_step_workspace_bytes(...) bytes,
+ *   256-byte aligned; it holds the staged inputs and every intermediate array.
+ * HOST outputs: loss_h [1] f32, counters_h [8] i64 (AERO_CNT_*), metrics_h [8] f32 (the
+ *   four group metrics followed by the four token metrics); any may be NULL.
+ * Errors as above; the status word is read with aero_last_status.
+ */
+size_t aero_step_workspace_bytes(int32_t P, int32_t R, int64_t T, int32_t d, int32_t V, int64_t chunk_tokens,
+                                 int32_t dtype);
+
+int aero_grpo_step_host(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R, int64_t T, int32_t d, int32_t V,
+                        const int32_t* go_h, const float* reward_h, const int64_t* cs_h, const uint32_t* key_h,
+                        const float* alpha_h, const float* beta_h,
+                        const void* H_h, const int32_t* y_h, const float* old_logp_h,
+                        const void* W, void* dH, float* dW, int accumulate_dW,
+                        float* loss_h, int64_t* counters_h, float* metrics_h,
+                        void* workspace, size_t workspace_bytes);
+
+/* Number of kernels the library has launched through this context since it was created
+ * (copies and memsets are not counted).  Host-side counter, no synchronisation. */
+int64_t aero_launch_count(aero_ctx* ctx);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,6 +26,7 @@ EXPORTS = [
     "aero_version", "aero_error_string", "aero_cfg_default", "aero_create", "aero_destroy",
     "aero_set_stream", "aero_last_status", "aero_group_workspace_bytes", "aero_group_stats",
     "aero_fwd_workspace_bytes", "aero_grpo_loss_fwd", "aero_bwd_workspace_bytes", "aero_grpo_loss_bwd",
+    "aero_step_workspace_bytes", "aero_grpo_step_host", "aero_launch_count",
 ]
 
 
@@ -75,6 +76,12 @@ def load_library():
     lib.aero_bwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i64]
     lib.aero_grpo_loss_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 7 + [f32] +
                                        [vp, vp, C.c_int, vp, sz])
+    lib.aero_step_workspace_bytes.restype = sz
+    lib.aero_step_workspace_bytes.argtypes = [i32, i32, i64, i32, i32, i64, i32]
+    lib.aero_grpo_step_host.argtypes = ([vp, C.POINTER(AeroCfg), i32, i32, i64, i32, i32] + [vp] * 12 + [C.c_int] +
+                                        [vp, vp, vp, vp, sz])
+    lib.aero_launch_count.restype = C.c_int64
+    lib.aero_launch_count.argtypes = [vp]
     _lib = lib
     return lib
 
@@ -239,3 +246,34 @@ class Context:
             workspace.data_ptr(), workspace.numel())
         _check(rc, "aero_grpo_loss_bwd")
         return dH, dW
+
+    # ---- whole step from host buffers ---------------------------------------------------
+    def launch_count(self) -> int:
+        return int(self.lib.aero_launch_count(self.h))
+
+    def step_workspace_bytes(self, P, R, T, d, V, chunk_tokens, dtype=AERO_BF16):
+        return self.lib.aero_step_workspace_bytes(P, R, T, d, V, chunk_tokens, dtype)
+
+    def grpo_step_host(self, cfg, go_h, reward_h, cs_h, key_h, alpha_h, beta_h, H_h, y_h, old_h, W, dH, dW,
+                       workspace, accumulate_dW=False):
+        """Host tensors (ideally pinned) in, device W/dH/dW, returns (loss, counters, metrics) host tensors."""
+        P, R = go_h.numel() - 1, reward_h.numel()
+        T, d = H_h.shape
+        V = W.shape[0]
+
+        def hp(t):
+            if t is None:
+                return None
+            if t.is_cuda or not t.is_contiguous():
+                raise AeroError("host inputs must be contiguous CPU tensors")
+            return t.data_ptr()
+
+        loss = torch.zeros(1, dtype=torch.float32)
+        counters = torch.zeros(8, dtype=torch.int64)
+        metrics = torch.zeros(8, dtype=torch.float32)
+        rc = self.lib.aero_grpo_step_host(
+            self.h, C.byref(cfg), P, R, T, d, V, hp(go_h), hp(reward_h), hp(cs_h), hp(key_h), hp(alpha_h), hp(beta_h),
+            hp(H_h), hp(y_h), hp(old_h), _ptr(W), _ptr(dH), _ptr(dW, torch.float32), 1 if accumulate_dW else 0,
+            loss.data_ptr(), counters.data_ptr(), metrics.data_ptr(), workspace.data_ptr(), workspace.numel())
+        _check(rc, "aero_grpo_step_host")
+        return loss, counters, metrics

@@ -65,6 +65,7 @@ int aero_create(aero_ctx** out, int device, void* cuda_stream) {
   ctx->stream = static_cast<cudaStream_t>(cuda_stream);
   ctx->d_status = nullptr;
   ctx->tmap_encode = nullptr;
+  ctx->launches = 0;
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return AERO_ERR_CUDA; }
   ctx->sm_count = prop.multiProcessorCount;

@@ -15,6 +15,7 @@ struct aero_ctx {
   uint32_t* d_status;     // device status word (OR of AERO_ST_* bits)
   int sm_count;
   void* tmap_encode;      // cuTensorMapEncodeTiled, resolved once through the runtime
+  long long launches;     // kernels launched so far (host-side count)
 };
 
 #define AERO_CUDA_TRY(expr)                          \

@@ -439,6 +439,7 @@ int launch_all(aero_ctx* ctx, const Args& a, void* wsp) {
   group_kernel<L><<<nb, kThreads, 0, ctx->stream>>>(a, ws);
   scan_kernel<<<1, 1024, 0, ctx->stream>>>(a, ws, nb);
   compact_kernel<L><<<nb, kThreads, 0, ctx->stream>>>(a, ws);
+  ctx->launches += 3;
   AERO_CUDA_TRY(cudaGetLastError());
   return AERO_OK;
 }

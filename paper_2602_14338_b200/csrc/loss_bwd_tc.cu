@@ -57,6 +57,7 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     const long long blocks = (T + 7) / 8;
     zero_dropped_rows_kernel<<<(int)(blocks < 4096 ? blocks : 4096), 256, 0, ctx->stream>>>(
         T, d, R, cs, keep, static_cast<__nv_bfloat16*>(dH));
+    ctx->launches += 1;
     AERO_CUDA_TRY(cudaGetLastError());
   }
 
@@ -101,6 +102,7 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
            ctx->stream>>>(tmDZ_k, tmW_mn, gp);
     k_dw<<<(int)(dw_units < ctx->sm_count ? dw_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
            ctx->stream>>>(tmDZ_mn, tmH_mn, gp);
+    ctx->launches += 3;
     AERO_CUDA_TRY(cudaGetLastError());
   }
   return AERO_OK;

@@ -158,6 +158,7 @@ int aero_build_tiles(aero_ctx* ctx, int64_t T, int32_t R, const int64_t* cs, con
   }
   build_tiles_kernel<<<1, 1024, 0, ctx->stream>>>(T, R, cs, keep, tile_rows, tiles.tile_row,
                                                   tiles.tile_valid, tiles.n_tiles, tiles.max_tiles);
+  ctx->launches += 1;
   AERO_CUDA_TRY(cudaGetLastError());
   return AERO_OK;
 }
@@ -165,6 +166,7 @@ int aero_build_tiles(aero_ctx* ctx, int64_t T, int32_t R, const int64_t* cs, con
 int aero_loss_finalize(aero_ctx* ctx, const double* partials, int n_partials, int stride,
                        float* loss, float* metrics, int accumulate) {
   finalize_kernel<<<1, 1024, 0, ctx->stream>>>(partials, n_partials, stride, loss, metrics, accumulate);
+  ctx->launches += 1;
   AERO_CUDA_TRY(cudaGetLastError());
   return AERO_OK;
 }

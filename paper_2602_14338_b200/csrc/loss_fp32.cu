@@ -172,6 +172,7 @@ int aero_fwd_fp32(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int3
     const int grid = (int)(blocks < 65535 ? blocks : 65535);
     fwd_fp32_kernel<<<grid, kWarpsPerBlock * 32, 0, ctx->stream>>>(*cfg, T, d, V, R, H, W, y, old_logp, cs, adv, w,
                                                                    keep, logp, lse, g, partials, ctx->d_status);
+    ctx->launches += 1;
     AERO_CUDA_TRY(cudaGetLastError());
   }
   return aero_loss_finalize(ctx, partials, (T > 0 && R > 0) ? (int)T : 0, kPartialStride, loss, metrics, accumulate);
@@ -185,11 +186,13 @@ int aero_bwd_fp32(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int3
     const long long blocks = (T + kWarpsPerBlock - 1) / kWarpsPerBlock;
     const int grid = (int)(blocks < 65535 ? blocks : 65535);
     bwd_dh_fp32_kernel<<<grid, kWarpsPerBlock * 32, 0, ctx->stream>>>(T, d, V, H, W, y, lse, g, grad_scale, dH);
+    ctx->launches += 1;
     AERO_CUDA_TRY(cudaGetLastError());
   }
   const int vblocks = (V + kWarpsPerBlock - 1) / kWarpsPerBlock;
   bwd_dw_fp32_kernel<<<vblocks < 65535 ? vblocks : 65535, kWarpsPerBlock * 32, 0, ctx->stream>>>(
       T, d, V, H, W, y, lse, g, grad_scale, dW, accumulate_dW);
+  ctx->launches += 1;
   AERO_CUDA_TRY(cudaGetLastError());
   return AERO_OK;
 }

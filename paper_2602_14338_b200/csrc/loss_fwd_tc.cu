@@ -61,6 +61,7 @@ int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     const int64_t upper = T / lmhead::BM + R + 1;
     const int grid = (int)(upper < ctx->sm_count ? upper : ctx->sm_count);
     kern<<<grid, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH, tmW, p);
+    ctx->launches += 1;
     AERO_CUDA_TRY(cudaGetLastError());
   }
   return aero_loss_finalize(ctx, f.partials, (int)f.n_partials, kPartialStride, loss, metrics, accumulate);

@@ -276,3 +276,30 @@ def test_full_width_qwen_1p5b_shape(ctx):
     rdH, rdW = batch.oracle_bwd(ref, dw_rows=rows)
     assert TL.rel_l2(dH.float().cpu().numpy(), rdH) < GRAD_L2
     assert TL.rel_l2(dW.cpu().numpy()[rows], rdW) < GRAD_L2
+
+
+def test_step_from_host_buffers_matches_device_calls(ctx):
+    over, cover, _ = BF16_CASES["aero_dropped"]
+    wl = synth.scaled(synth.WORKLOADS[1], **over)
+    batch = TL.Batch(wl, O.Cfg(seed=wl.seed, **cover))
+    st = batch.st
+    cfg = TL.lib_cfg(batch.ocfg, "bf16")
+    dv = batch.to_device()
+    gi, g = TL.run_group_gpu(ctx, cfg, st)
+    f = ctx.grpo_loss_fwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], g["adv"], g["w"], g["keep"])
+    dH, dW = ctx.grpo_loss_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], g["keep"], f["lse"], f["g"])
+    l0 = ctx.launch_count()
+    dH2, dW2 = torch.empty_like(dH), torch.empty_like(dW)
+    ws = torch.empty(ctx.step_workspace_bytes(batch.P, batch.R, batch.T, wl.d, wl.V, 1024, cfg.dtype),
+                     dtype=torch.uint8, device="cuda")
+    h = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    loss, counters, metrics = ctx.grpo_step_host(
+        cfg, h(st.go), h(st.reward), h(st.cs), h(st.key.view(np.int32)), h(st.alpha), h(st.beta),
+        batch.H_t.pin_memory(), h(st.y), h(batch.old), dv["W"], dH2, dW2, ws)
+    assert ctx.launch_count() > l0
+    assert loss.item() == f["loss"].item()
+    assert counters.tolist() == g["counters"].cpu().tolist()
+    assert torch.equal(dH2, dH)
+    assert TL.rel_l2(dW2.cpu().numpy(), dW.cpu().numpy()) < 1e-5
+    assert metrics[7].item() == f["metrics"][3].item()
+    assert ctx.last_status() == 0
