@@ -172,7 +172,7 @@ class Context:
     def group_stats(self, cfg, go, reward, cs, key=None, keep_in=None, alpha_in=None, beta_in=None, out=None):
         P, R = go.numel() - 1, reward.numel()
         dev = self.device
-        o = out or {}
+        o = out if out is not None else {}
 
         def buf(name, n, dt):
             if name not in o:
@@ -206,7 +206,7 @@ class Context:
         V = W.shape[0]
         R = cs.numel() - 1
         dt = torch.bfloat16 if cfg.dtype == AERO_BF16 else torch.float32
-        o = out or {}
+        o = out if out is not None else {}
         for name in ("logp", "lse", "g"):
             if name not in o:
                 o[name] = torch.empty(max(T, 1), dtype=torch.float32, device=self.device)
