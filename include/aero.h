@@ -53,6 +53,7 @@ extern "C" {
 #define AERO_ERR_UNSUPPORTED -2   /* shape the kernels do not cover (e.g. d % 64 != 0) */
 #define AERO_ERR_WORKSPACE   -3   /* workspace smaller than aero_*_workspace_bytes     */
 #define AERO_ERR_CUDA        -4   /* a CUDA runtime/driver call failed                 */
+#define AERO_ERR_TOO_LARGE   -5   /* problem exceeds the library-owned scratch array   */
 
 /* ---- device status bits (aero_last_status) ------------------------------------ */
 #define AERO_ST_BAD_TARGET     1u   /* y[t] outside [0,V): row treated as dropped      */
@@ -177,6 +178,39 @@ int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
                      float* u_tilde, float* alpha_out, float* beta_out,
                      int32_t* kept_ids, int64_t* kept_tok_off, int64_t* counters,
                      float* metrics, void* workspace, size_t workspace_bytes);
+
+/* aero_group_stats for callers that cannot allocate device memory.  (The paper has no
+ * counterpart to this call: it computes exactly what aero_group_stats computes; only the
+ * origin of the scratch memory differs.)
+ *
+ * Who needs it: code that is handed its input and output buffers but has no way to get a
+ * workspace at the point of the call -- a plug-in inside a host program that owns all
+ * device memory, or a latency-bound loop that must not call the allocator because an
+ * allocation can synchronise the whole device.  Instead of a caller workspace, the scratch
+ * is a fixed array in device memory that belongs to the loaded library itself: about
+ * 1.4 MB per GPU that loads the library, held until the process exits, sized for at most
+ * AERO_STATIC_MAX_PROMPTS prompts (R is not limited).  A larger P returns
+ * AERO_ERR_TOO_LARGE and launches nothing.  The call, and everything it calls, performs
+ * no cudaMalloc/cudaFree and uses no allocating library routine.
+ *
+ * The first call on each device looks up the array's device address (once per device,
+ * with that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array: two calls whose kernels may overlap on the
+ * GPU (different streams, or different contexts of this library on one device) race on
+ * it -- order them on one stream or with events.  The array keeps the previous call's
+ * contents; nothing in it needs clearing, because each call writes every word it later
+ * reads.  Arguments, outputs and status bits are those of aero_group_stats.
+ */
+#define AERO_STATIC_MAX_PROMPTS 65536
+
+int aero_group_stats_static(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
+                            const int32_t* go, const float* reward, const int64_t* cs,
+                            const uint32_t* key, const uint8_t* keep_in,
+                            const float* alpha_in, const float* beta_in,
+                            float* adv, float* w, uint8_t* keep, uint8_t* gmask, uint8_t* cat,
+                            float* u_tilde, float* alpha_out, float* beta_out,
+                            int32_t* kept_ids, int64_t* kept_tok_off, int64_t* counters,
+                            float* metrics);
 
 /* ------------------------------------------------------------------------------
  * Stage (b), forward (Eq. 2; Appendix C "GRPO Training").

@@ -26,7 +26,7 @@ EXPORTS = [
     "aero_version", "aero_error_string", "aero_cfg_default", "aero_create", "aero_destroy",
     "aero_set_stream", "aero_last_status", "aero_group_workspace_bytes", "aero_group_stats",
     "aero_fwd_workspace_bytes", "aero_grpo_loss_fwd", "aero_bwd_workspace_bytes", "aero_grpo_loss_bwd",
-    "aero_step_workspace_bytes", "aero_grpo_step_host", "aero_launch_count",
+    "aero_step_workspace_bytes", "aero_grpo_step_host", "aero_launch_count", "aero_group_stats_static",
 ]
 
 
@@ -69,6 +69,7 @@ def load_library():
     lib.aero_group_workspace_bytes.restype = sz
     lib.aero_group_workspace_bytes.argtypes = [i32, i32]
     lib.aero_group_stats.argtypes = [vp, C.POINTER(AeroCfg), i32, i32] + [vp] * 19 + [vp, sz]
+    lib.aero_group_stats_static.argtypes = [vp, C.POINTER(AeroCfg), i32, i32] + [vp] * 19
     lib.aero_fwd_workspace_bytes.restype = sz
     lib.aero_fwd_workspace_bytes.argtypes = [i64, i32, i32, i32]
     lib.aero_grpo_loss_fwd.argtypes = [vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 13 + [C.c_int, vp, sz]
@@ -193,6 +194,32 @@ class Context:
             _ptr(u), _ptr(ao), _ptr(bo), _ptr(kid), _ptr(kto), _ptr(cnt), _ptr(met), ws.data_ptr(), ws.numel())
         _check(rc, "aero_group_stats")
         return o
+
+    GROUP_OUTPUTS = (("adv", "R", torch.float32), ("w", "R", torch.float32), ("keep", "R", torch.uint8),
+                     ("gmask", "P", torch.uint8), ("cat", "P", torch.uint8), ("u_tilde", "P", torch.float32),
+                     ("alpha_out", "P", torch.float32), ("beta_out", "P", torch.float32),
+                     ("kept_ids", "R", torch.int32), ("kept_tok_off", "R1", torch.int64),
+                     ("counters", "8", torch.int64), ("metrics", "4", torch.float32))
+
+    def group_stats_static(self, cfg, go, reward, cs, out, key=None, keep_in=None, alpha_in=None, beta_in=None):
+        """aero_group_stats_static: the results of group_stats with the scratch taken from the array
+        that is part of the loaded library.  Nothing is allocated here either: `out` must already
+        hold every output tensor (names and sizes as group_stats returns them), so a caller that
+        cannot allocate at this point can still make the call."""
+        P, R = go.numel() - 1, reward.numel()
+        size = {"R": R, "P": P, "R1": R + 1, "8": 8, "4": 4}
+        ptrs = []
+        for name, n, dt in self.GROUP_OUTPUTS:
+            if name not in out:
+                raise AeroError(f"group_stats_static needs a preallocated '{name}' tensor")
+            ptrs.append(_ptr(out[name], dt, size[n], name))
+        rc = self.lib.aero_group_stats_static(
+            self.h, C.byref(cfg), P, R, _ptr(go, torch.int32, P + 1, "go"), _ptr(reward, torch.float32, R, "reward"),
+            _ptr(cs, torch.int64, R + 1, "cs"), _ptr_key(key, R),
+            _ptr(keep_in, torch.uint8, R, "keep_in"), _ptr(alpha_in, torch.float32, P, "alpha_in"),
+            _ptr(beta_in, torch.float32, P, "beta_in"), *ptrs)
+        _check(rc, "aero_group_stats_static")
+        return out
 
     # ---- stage (b) ------------------------------------------------------------------
     def fwd_workspace_bytes(self, T, d, V, R):

@@ -28,6 +28,7 @@ const char* aero_error_string(int code) {
     case AERO_ERR_UNSUPPORTED: return "unsupported shape or dtype";
     case AERO_ERR_WORKSPACE: return "workspace too small";
     case AERO_ERR_CUDA: return "CUDA call failed";
+    case AERO_ERR_TOO_LARGE: return "problem exceeds the library-owned scratch array";
     default: return "unknown error";
   }
 }

@@ -8,6 +8,8 @@
 // its loads and stores touch one contiguous range of the rollout arrays.
 #include "common.cuh"
 
+#include <mutex>
+
 namespace {
 
 constexpr int kThreads = 256;
@@ -480,4 +482,67 @@ int aero_group_stats_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32
     case 16: return launch_all<16>(ctx, a, ws);
     default: return launch_all<32>(ctx, a, ws);
   }
+}
+
+// ---- variant with library-owned scratch ------------------------------------------------
+// The three kernels above need a few bytes of scratch per prompt.  This entry point takes
+// them from a fixed array in device memory that is part of the loaded library image, so the
+// caller passes inputs and outputs only and nothing is allocated, by this call or before it.
+namespace {
+
+constexpr int32_t kStaticMaxP = AERO_STATIC_MAX_PROMPTS;
+constexpr size_t cup256(size_t x) { return (x + 255) / 256 * 256; }
+constexpr size_t kStaticNb = (size_t)(kStaticMaxP + 7) / 8 + 1;
+constexpr size_t kStaticBytes = cup256(sizeof(int) * (size_t)kStaticMaxP) + cup256(sizeof(long long) * (size_t)kStaticMaxP) +
+                                cup256(sizeof(BlockPartial) * kStaticNb) + cup256(sizeof(BlockOffset) * kStaticNb) +
+                                cup256(sizeof(Globals));
+
+static __device__ __align__(256) unsigned char g_group_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mu;
+void* g_scratch_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on `device`, looked up once per device.  In host code
+// the array's name is only a handle for this lookup, never a pointer a kernel could use.
+int static_scratch(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return AERO_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_scratch_mu);
+  if (!g_scratch_ptr[device]) {
+    void* p = nullptr;
+    if (cudaSetDevice(device) != cudaSuccess) return AERO_ERR_CUDA;
+    if (cudaGetSymbolAddress(&p, g_group_scratch) != cudaSuccess || !p) return AERO_ERR_CUDA;
+    g_scratch_ptr[device] = p;
+  }
+  *out = g_scratch_ptr[device];
+  return AERO_OK;
+}
+
+}  // namespace
+
+extern "C" int aero_group_stats_static(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
+                                       const int32_t* go, const float* reward, const int64_t* cs,
+                                       const uint32_t* key, const uint8_t* keep_in,
+                                       const float* alpha_in, const float* beta_in,
+                                       float* adv, float* w, uint8_t* keep, uint8_t* gmask, uint8_t* cat,
+                                       float* u_tilde, float* alpha_out, float* beta_out,
+                                       int32_t* kept_ids, int64_t* kept_tok_off, int64_t* counters,
+                                       float* metrics) {
+  if (!ctx || !cfg || P < 0 || R < 0) return AERO_ERR_INVALID;
+  if (P > kStaticMaxP) return AERO_ERR_TOO_LARGE;
+  if (aero_group_ws_bytes_impl(P, R) > kStaticBytes) return AERO_ERR_TOO_LARGE;
+  if (!go || !cs || !kept_tok_off || !counters) return AERO_ERR_INVALID;
+  if (R > 0 && (!reward || !adv || !w || !keep || !kept_ids)) return AERO_ERR_INVALID;
+  if (P > 0 && (!gmask || !cat || !u_tilde || !alpha_out || !beta_out)) return AERO_ERR_INVALID;
+  if ((alpha_in == nullptr) != (beta_in == nullptr)) return AERO_ERR_INVALID;
+  if (cfg->k_ratio < 1 || cfg->n_explore < 1 || cfg->rescue_S < 0) return AERO_ERR_INVALID;
+  if (cudaSetDevice(ctx->device) != cudaSuccess) return AERO_ERR_CUDA;
+  void* scratch = nullptr;
+  const int rc = static_scratch(ctx->device, &scratch);
+  if (rc) return rc;
+  // every scratch word the kernels read is written earlier in the same call, so nothing
+  // has to be cleared between calls
+  return aero_group_stats_launch(ctx, cfg, P, R, go, reward, cs, key, keep_in, alpha_in, beta_in,
+                                 adv, w, keep, gmask, cat, u_tilde, alpha_out, beta_out,
+                                 kept_ids, kept_tok_off, counters, metrics, scratch);
 }
