@@ -38,6 +38,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1, help="workload index 0..4")
     ap.add_argument("--chunk-tokens", type=int, default=2 * 148 * 128)
+    ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (reduced runs for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -196,6 +197,8 @@ def run_ours(args):
 
     base = synth.WORKLOADS[args.config]
     wl = synth.scaled(base, seed=base.seed + 100 * rank)      # an independent batch per replica
+    if args.prompts > 0:
+        wl = synth.scaled(wl, P=args.prompts)
     st = synth.make_structure(wl)
     P, R, T = len(st.go) - 1, len(st.reward), int(st.cs[-1])
     H, W = synth.make_tensors(wl, T, device=dev)
@@ -230,7 +233,7 @@ def run_ours(args):
         ctx.grpo_loss_bwd(cfg, H, W, y, cs, g["keep"], f["lse"], f["g"], dH=dH, dW=dW, workspace=ws_b)
         return g, f
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(args.warmup, 1)):
         g, f = step()
     torch.cuda.synchronize()
     T_kept = int(g["counters"][1].item())
@@ -274,7 +277,7 @@ def run_ours(args):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": max(args.warmup, 1), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
         "config": {"workload": wl.name, "P": P, "R": R, "T_input": T, "T_kept": T_kept, "d": wl.d, "V": wl.V,
                    "parallelism": f"replicas x{world}", "chunk_tokens": int(chunk),
