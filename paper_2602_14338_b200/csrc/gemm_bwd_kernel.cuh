@@ -82,6 +82,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
+      int row_cur = 0, row_next = 0;
       for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
         const int mt = u / n_nt, nt = u % n_nt;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
@@ -92,22 +93,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           uint8_t* b_s = a_s + A_BYTES;
           tc::mbar_arrive_expect_tx(&ctl->full[s], STAGE_BYTES);
           if (KIND == KIND_DH) {
-            // A: dz rows of the tile (K-major, K = vocabulary); B: W rows kb*64.. (MN-major)
+            // A: dz rows of the tile (K-major, K = vocabulary); B: W rows kb*64.. as four
+            // 64-column blocks (MN-major, blocked view)
             tc::tma_load_2d(a_s, &tmA, kb * BK, mt * BM, &ctl->full[s]);
-#pragma unroll
-            for (int q = 0; q < BN / 64; ++q)
-              tc::tma_load_2d(b_s + q * BOX_BYTES, &tmB, nt * BN + q * 64, kb * BK, &ctl->full[s]);
+            tc::tma_load_3d(b_s, &tmB, 0, kb * BK, nt * (BN / 64), &ctl->full[s]);
           } else {
-            // A: dz columns of the vocabulary tile over 64 chunk rows (MN-major);
-            // B: the 64 rows of H those chunk rows stand for (MN-major)
-            const int tile = p.tile_begin + kb / (BM / BK);
-            const int hrow = p.tile_row[tile] + (kb % (BM / BK)) * BK;
-#pragma unroll
-            for (int q = 0; q < BM / 64; ++q)
-              tc::tma_load_2d(a_s + q * BOX_BYTES, &tmA, mt * BM + q * 64, kb * BK, &ctl->full[s]);
-#pragma unroll
-            for (int q = 0; q < BN / 64; ++q)
-              tc::tma_load_2d(b_s + q * BOX_BYTES, &tmB, nt * BN + q * 64, hrow, &ctl->full[s]);
+            // A: two 64-column blocks of dz over 64 chunk rows (MN-major);
+            // B: the 64 rows of H those chunk rows stand for, four 64-column blocks (MN-major)
+            if ((kb % (BM / BK)) == 0) {
+              // the row of the tile after this one is fetched now and used two slabs later
+              row_cur = kb == 0 ? __ldg(p.tile_row + p.tile_begin) : row_next;
+              const int nxt = kb / (BM / BK) + 1;
+              row_next = nxt < chunk_tiles ? __ldg(p.tile_row + p.tile_begin + nxt) : 0;
+            }
+            const int hrow = row_cur + (kb % (BM / BK)) * BK;
+            tc::tma_load_3d(a_s, &tmA, 0, kb * BK, mt * (BM / 64), &ctl->full[s]);
+            tc::tma_load_3d(b_s, &tmB, 0, hrow, nt * (BN / 64), &ctl->full[s]);
           }
         }
       }

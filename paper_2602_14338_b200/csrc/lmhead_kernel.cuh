@@ -30,7 +30,9 @@ struct Ctl {
   uint32_t tmem_base;
   int abort;
 };
-constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + sizeof(Ctl);
+// dz staging for the TMA stores of MODE_DZ: per epilogue warp two buffers of 32 rows x 64 bf16
+constexpr uint32_t STG_BUF_BYTES = 32 * 64 * 2, STG_BYTES = 4 * 2 * STG_BUF_BYTES;
+constexpr size_t SMEM_BYTES = 1024 + (size_t)STAGES * STAGE_BYTES + STG_BYTES + sizeof(Ctl);
 
 struct Params {
   long long T;
@@ -72,10 +74,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 template <int MODE>
 __global__ void __launch_bounds__(THREADS, 1)
-lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW, const Params p) {
+lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW,
+              const __grid_constant__ CUtensorMap tmDZ, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  Ctl* ctl = reinterpret_cast<Ctl*>(smem + (size_t)STAGES * STAGE_BYTES);
+  uint8_t* stg_all = smem + (size_t)STAGES * STAGE_BYTES;
+  Ctl* ctl = reinterpret_cast<Ctl*>(stg_all + STG_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
@@ -149,9 +153,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
     }
   } else {
     // ---------------- epilogue warps 0..3 ----------------
-    uint32_t at = 0;
+    uint32_t at = 0, nstore = 0;
     bool ok = true;
     const int r_in_tile = warp * 32 + lane;
+    uint8_t* stg_warp = stg_all + warp * 2 * STG_BUF_BYTES;
     for (int tile = p.tile_begin + blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
       const long long row = (long long)p.tile_row[tile] + r_in_tile;
       const bool valid_row = r_in_tile < p.tile_valid[tile] && row < p.T;
@@ -163,11 +168,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
 
       float m2 = -INFINITY, l = 0.f, zy = 0.f;         // MODE_FWD running state (log2 domain)
       float lse2 = 0.f, coef = 0.f;                    // MODE_DZ per-row constants
-      __nv_bfloat16* dz_row = nullptr;
       if (MODE == MODE_DZ) {
         if (live) { lse2 = p.lse_in[row] * kLog2e; coef = p.g_in[row] * p.grad_scale; }
-        dz_row = p.dz + ((long long)(tile - p.tile_begin) * BM + r_in_tile) * p.ldz;
       }
+      const int dz_row0 = (tile - p.tile_begin) * BM + warp * 32;   // first dz row of this warp
 
       for (int j = 0; ok && j < nvt; ++j, ++at) {
         const uint32_t buf = at & 1u, aph = (at >> 1) & 1u;
@@ -177,11 +181,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
         const int col_base = j * BN;
         const int ncol = min(BN, (MODE == MODE_DZ ? (int)p.ldz : p.V) - col_base);
         const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + buf * BN;
-        for (int c = 0; c * 32 < ncol; ++c) {
-          uint32_t r[32];
-          __syncwarp();                     // the TMEM load is warp-collective
-          tc::tmem_ld_32x32(taddr + c * 32, r);
-          tc::tmem_ld_wait();
+        // One 32-column chunk of this thread's row, already in registers.
+        auto process = [&](const uint32_t (&r)[32], int c) {
           const int col0 = col_base + c * 32;
           if (MODE == MODE_FWD) {
             float z[32];
@@ -206,20 +207,70 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
               for (int q = 0; q < 32; ++q) if (q == sel) zy = z[q];
             }
           } else {
+            // 32 columns -> 16 packed words -> half of this row's 128-byte line in the staging
+            // buffer (16-byte chunks XOR-swizzled with the row, matching the store's tensor map)
             uint32_t pk[16];
+            if (live && col0 + 32 <= p.V) {
+              float v[32];
 #pragma unroll
-            for (int q = 0; q < 32; q += 2) {
-              float v0 = -coef * ex2(fmaf(__uint_as_float(r[q]), kLog2e, -lse2));
-              float v1 = -coef * ex2(fmaf(__uint_as_float(r[q + 1]), kLog2e, -lse2));
-              if (col0 + q == yt) v0 += coef;
-              if (col0 + q + 1 == yt) v1 += coef;
-              if (!live || col0 + q >= p.V) v0 = 0.f;
-              if (!live || col0 + q + 1 >= p.V) v1 = 0.f;
-              pk[q >> 1] = pack_bf16(v0, v1);
+              for (int q = 0; q < 32; ++q) v[q] = -coef * ex2(fmaf(__uint_as_float(r[q]), kLog2e, -lse2));
+              if ((unsigned)(yt - col0) < 32u) {
+                const int sel = yt - col0;
+#pragma unroll
+                for (int q = 0; q < 32; ++q) if (q == sel) v[q] += coef;
+              }
+#pragma unroll
+              for (int q = 0; q < 32; q += 2) pk[q >> 1] = pack_bf16(v[q], v[q + 1]);
+            } else {
+#pragma unroll
+              for (int q = 0; q < 32; q += 2) {
+                float v0 = -coef * ex2(fmaf(__uint_as_float(r[q]), kLog2e, -lse2));
+                float v1 = -coef * ex2(fmaf(__uint_as_float(r[q + 1]), kLog2e, -lse2));
+                if (col0 + q == yt) v0 += coef;
+                if (col0 + q + 1 == yt) v1 += coef;
+                if (!live || col0 + q >= p.V) v0 = 0.f;
+                if (!live || col0 + q + 1 >= p.V) v1 = 0.f;
+                pk[q >> 1] = pack_bf16(v0, v1);
+              }
             }
-            uint4* dst = reinterpret_cast<uint4*>(dz_row + col0);
+            const int half = c & 1;
+            if (half == 0) {
+              // the buffer is free once the store issued two blocks ago has read it
+              if (lane == 0) tc::tma_store_wait_read<1>();
+              __syncwarp();
+            }
+            uint8_t* stg = stg_warp + (nstore & 1u) * STG_BUF_BYTES;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) dst[q] = make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+            for (int q = 0; q < 4; ++q) {
+              const int chunk = (half * 4 + q) ^ (lane & 7);
+              *reinterpret_cast<uint4*>(stg + lane * 128 + chunk * 16) =
+                  make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+            }
+            if (half == 1) {
+              tc::fence_proxy_async();
+              __syncwarp();
+              if (lane == 0) {
+                tc::tma_store_2d(&tmDZ, stg, col0 - 32, dz_row0);
+                tc::tma_store_commit();
+              }
+              ++nstore;
+            }
+          }
+        };
+        // TMEM loads are software-pipelined: the load of chunk c+1 is in flight while chunk c
+        // is processed (every load is warp-collective, hence the __syncwarp before each)
+        const int nch = (ncol + 31) / 32;
+        uint32_t ra[32], rb[32];
+        __syncwarp();
+        tc::tmem_ld_32x32(taddr, ra);
+        for (int c = 0; c < nch; c += 2) {
+          tc::tmem_ld_wait();
+          if (c + 1 < nch) { __syncwarp(); tc::tmem_ld_32x32(taddr + (c + 1) * 32, rb); }
+          process(ra, c);
+          if (c + 1 < nch) {
+            tc::tmem_ld_wait();
+            if (c + 2 < nch) { __syncwarp(); tc::tmem_ld_32x32(taddr + (c + 2) * 32, ra); }
+            process(rb, c + 1);
           }
         }
         tc::tc_fence_before();
@@ -259,6 +310,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
   }
 
   // ---------------- teardown ----------------
+  if (MODE == MODE_DZ && warp < 4 && lane == 0) tc::tma_store_wait_all<0>();   // own stores have landed
   __syncwarp();
   if (*abort_flag) {
     // a wait gave up: let copies and MMAs already in flight land before shared memory and

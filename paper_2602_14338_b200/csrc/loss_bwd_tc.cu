@@ -68,10 +68,13 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
   if ((rc = aero_make_tmap_2d(ctx, &tmH_k, BF, 2, H, T, d, d, lmhead::BM, 64))) return rc;
   if ((rc = aero_make_tmap_2d(ctx, &tmW_k, BF, 2, W, V, d, d, lmhead::BN, 64))) return rc;
   if ((rc = aero_make_tmap_2d(ctx, &tmDZ_k, BF, 2, dz, dz_rows, ldz, ldz, gemmbwd::BM, 64))) return rc;
-  // MN-major views: 64 x 64 boxes
-  if ((rc = aero_make_tmap_2d(ctx, &tmW_mn, BF, 2, W, V, d, d, 64, 64))) return rc;
-  if ((rc = aero_make_tmap_2d(ctx, &tmDZ_mn, BF, 2, dz, dz_rows, ldz, ldz, 64, 64))) return rc;
-  if ((rc = aero_make_tmap_2d(ctx, &tmH_mn, BF, 2, H, T, d, d, 64, 64))) return rc;
+  // MN-major operands: blocked views, one box = 64 rows x (4 or 2) column blocks of 64
+  if ((rc = aero_make_tmap_blocked(ctx, &tmW_mn, W, V, d, d, 64, gemmbwd::BN / 64))) return rc;
+  if ((rc = aero_make_tmap_blocked(ctx, &tmDZ_mn, dz, dz_rows, ldz, ldz, 64, gemmbwd::BM / 64))) return rc;
+  if ((rc = aero_make_tmap_blocked(ctx, &tmH_mn, H, T, d, d, 64, gemmbwd::BN / 64))) return rc;
+  // store view of the dz block for the lm_head kernel's epilogue: 32 rows x 64 columns per copy
+  CUtensorMap tmDZ_st;
+  if ((rc = aero_make_tmap_2d(ctx, &tmDZ_st, BF, 2, dz, dz_rows, ldz, ldz, 32, 64))) return rc;
 
   auto k_dz = lmhead::lmhead_kernel<lmhead::MODE_DZ>;
   auto k_dh = gemmbwd::gemm_kernel<gemmbwd::KIND_DH>;
@@ -90,7 +93,7 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     lp.y = y; lp.status = ctx->d_status;
     lp.lse_in = lse; lp.g_in = g; lp.grad_scale = grad_scale; lp.dz = dz; lp.ldz = ldz;
     const int grid_dz = (int)(tpc < ctx->sm_count ? tpc : ctx->sm_count);
-    k_dz<<<grid_dz, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH_k, tmW_k, lp);
+    k_dz<<<grid_dz, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH_k, tmW_k, tmDZ_st, lp);
 
     gemmbwd::Params gp = {};
     gp.T = T; gp.d = d; gp.V = V; gp.ldz = ldz;

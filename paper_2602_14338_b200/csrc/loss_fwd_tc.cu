@@ -60,7 +60,7 @@ int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     AERO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lmhead::SMEM_BYTES));
     const int64_t upper = T / lmhead::BM + R + 1;
     const int grid = (int)(upper < ctx->sm_count ? upper : ctx->sm_count);
-    kern<<<grid, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH, tmW, p);
+    kern<<<grid, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH, tmW, tmH, p);   // third map unused in forward mode
     ctx->launches += 1;
     AERO_CUDA_TRY(cudaGetLastError());
   }

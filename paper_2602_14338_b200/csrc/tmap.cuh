@@ -32,3 +32,29 @@ inline int aero_make_tmap_2d(aero_ctx* ctx, CUtensorMap* out, CUtensorMapDataTyp
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? AERO_OK : AERO_ERR_CUDA;
 }
+
+// Blocked 3-D view of a row-major bf16 matrix whose column count is a multiple of 64:
+// dimension 0 = the 64 elements of a column block (128 bytes), dimension 1 = rows,
+// dimension 2 = column blocks.  A box of (64, box_rows, n_blocks) lands in shared memory as
+// n_blocks consecutive [box_rows][64] sub-tiles, which is the MN-major operand layout of
+// tcgen05.mma with 128-byte swizzle -- one copy instead of one per 64-column block.
+inline int aero_make_tmap_blocked(aero_ctx* ctx, CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols,
+                                  uint64_t ld_elems, uint32_t box_rows, uint32_t n_blocks) {
+  if (!ctx->tmap_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess || !fn)
+      return AERO_ERR_CUDA;
+    ctx->tmap_encode = fn;
+  }
+  auto encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ctx->tmap_encode);
+  cuuint64_t gdim[3] = {64, rows, cols / 64};
+  cuuint64_t gstride[2] = {ld_elems * 2, 128};
+  cuuint32_t box[3] = {64, box_rows, n_blocks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstride, box, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? AERO_OK : AERO_ERR_CUDA;
+}
