@@ -13,7 +13,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libaero_b200.so")
+LIB_PATH = os.environ.get("AERO_B200_LIB") or os.path.join(_HERE, "libaero_b200.so")
 
 AERO_UNIFORM_MASK, AERO_UNIFORM_BAYES = 0, 1
 AERO_STATS_KEPT, AERO_STATS_ALL = 0, 1

@@ -17,7 +17,10 @@
 
 namespace gemmbwd {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+#ifndef AERO_TC_STAGES
+#define AERO_TC_STAGES 4          // depth of the TMA -> MMA shared-memory ring
+#endif
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = AERO_TC_STAGES, UMMA_K = 16;
 constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr uint32_t BOX_BYTES = 64 * 64 * 2;     // one 64 x 64 bf16 box of an MN-major operand
 constexpr int THREADS = 192;

@@ -303,3 +303,95 @@ def test_step_from_host_buffers_matches_device_calls(ctx):
     assert TL.rel_l2(dW2.cpu().numpy(), dW.cpu().numpy()) < 1e-5
     assert metrics[7].item() == f["metrics"][3].item()
     assert ctx.last_status() == 0
+
+
+def test_full_size_qwen_1p5b_in_bench_configuration(ctx):
+    """The whole Qwen2.5-Math-1.5B shaped workload (~283k tokens) in the launch configuration
+    bench.py times.  The oracle cannot produce all of it, so: the group stage is compared in
+    full; 96 sampled token rows are compared one by one (log-prob, lse, g, dH row); the loss and
+    sampled rows of dW are checked through identities that hold at any size."""
+    wl = synth.WORKLOADS[1]
+    st = synth.make_structure(wl)
+    P, R, T = len(st.go) - 1, len(st.reward), int(st.cs[-1])
+    ocfg = TL.cfg_for(wl)
+    cfg = TL.lib_cfg(ocfg, "bf16")
+    H, W = synth.make_tensors(wl, T, device="cuda")
+    ref_g = O.group_stats(ocfg, st.go, st.reward, st.cs, key=st.key)
+    gi, g = TL.run_group_gpu(ctx, cfg, st)
+    TL.check_group(g, ref_g, R, P)
+
+    owner = O.token_rollout(st.cs, T)
+    kept_rows = np.nonzero(ref_g["keep"][owner] != 0)[0]
+    rng = np.random.default_rng(7)
+    sample = np.unique(np.concatenate([kept_rows[:2], kept_rows[-2:], rng.choice(kept_rows, 92, replace=False)]))
+    W64 = W.double().cpu().numpy()
+    Hs = H[torch.from_numpy(sample).cuda()].double().cpu().numpy()
+    zs = O.logits(Hs, W64)
+    lp_s, lse_s = O.log_softmax_pick(zs, st.y[sample])
+    # old log-probs: model-independent constant for the bulk, oracle log-prob + noise on the sample,
+    # with a few large perturbations so that both clip edges are exercised
+    old = np.full(T, -12.2, np.float32) + st.noise
+    pert = st.noise[sample].astype(np.float64)
+    pert[::7] *= 8.0
+    old[sample] = (lp_s + pert).astype(np.float32)
+
+    y, cs, oldd = TL.dev(st.y), TL.dev(st.cs), TL.dev(old)
+    f = ctx.grpo_loss_fwd(cfg, H, W, y, oldd, cs, g["adv"], g["w"], g["keep"])
+    chunk = 2 * 148 * 128
+    ws = torch.empty(ctx.bwd_workspace_bytes(T, wl.d, wl.V, R, chunk), dtype=torch.uint8, device="cuda")
+    dH, dW = ctx.grpo_loss_bwd(cfg, H, W, y, cs, g["keep"], f["lse"], f["g"], workspace=ws)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+
+    # --- sampled rows against the oracle
+    adv32 = g["adv"][:R].cpu().numpy().astype(np.float64)
+    w32 = g["w"][:R].cpu().numpy().astype(np.float64)
+    s_ref, g_ref, rho_ref, ind_ref = O.surrogate(ocfg, lp_s, old[sample].astype(np.float64),
+                                                 adv32[owner[sample]], w32[owner[sample]])
+    logp = f["logp"][:T].cpu().numpy()
+    lse = f["lse"][:T].cpu().numpy()
+    gg = f["g"][:T].cpu().numpy()
+    assert np.abs(logp[sample] - lp_s).max() <= LOGP_ABS
+    assert np.abs(lse[sample] - lse_s).max() <= LOGP_ABS
+    edge = (np.abs(rho_ref - 1.2) < 1e-3) | (np.abs(rho_ref - 0.8) < 1e-3)
+    np.testing.assert_allclose(gg[sample][~edge], g_ref[~edge], rtol=2e-2, atol=1e-14)
+    assert (ind_ref == 0).any() and (ind_ref == 1).any()
+    mini_cs = np.arange(len(sample) + 1, dtype=np.int64)
+    rdH, _ = O.grpo_loss_bwd(Hs, W64, st.y[sample], mini_cs, np.ones(len(sample), np.uint8), lse_s, g_ref,
+                             dw_rows=[0])
+    dHs = dH[torch.from_numpy(sample).cuda()].float().cpu().numpy()
+    live = (g_ref != 0) & ~edge
+    assert TL.rel_l2(dHs[live], rdH[live]) < GRAD_L2
+    assert not dHs[(g_ref == 0) & ~edge].any()
+    # dropped rows: zero outputs
+    dropped = torch.from_numpy(np.nonzero(ref_g["keep"][owner] == 0)[0][::97].copy()).cuda()
+    assert not dH[dropped].float().abs().sum().item() and not f["g"][dropped].abs().sum().item()
+
+    # --- identities at full size (test-side arithmetic on the library's outputs)
+    kept = ref_g["keep"][owner] != 0
+    A_t, w_t = adv32[owner], w32[owner]
+    rho = np.exp(logp.astype(np.float64) - old.astype(np.float64))
+    surr = np.minimum(rho * A_t, np.clip(rho, 0.8, 1.2) * A_t)
+    loss_re = -float(np.sum((w_t * surr)[kept]))
+    assert abs(f["loss"].item() - loss_re) <= 1e-4 * abs(loss_re) + 1e-8
+    assert (logp[kept] <= 1e-6).all() and not logp[~kept].any()
+    # columns of dW sum to zero because each row of dz does
+    colsum = dW.double().sum(dim=0).abs().max().item()
+    assert colsum <= 1e-2 * dW.double().abs().sum(dim=0).max().item()
+    # rows of dW from the definition, with the library's own lse and g (fp64 on the device)
+    vrows = np.unique(np.concatenate([st.y[kept_rows[:8]], rng.integers(0, wl.V, 24)]))
+    vr = torch.from_numpy(vrows).cuda()
+    H64 = H.double()
+    z = H64 @ W[vr].double().T
+    dz = -torch.exp(z - f["lse"][:T].double()[:, None])
+    dz += (y[:, None] == vr[None, :].to(y.dtype)).double()
+    dz *= f["g"][:T].double()[:, None]
+    ref_rows = (dz.T @ H64).cpu().numpy()
+    assert TL.rel_l2(dW[vr].cpu().numpy(), ref_rows) < GRAD_L2
+    del H64, z, dz
+    # a different chunking gives the same dH bits and the same dW up to fp32 summation order
+    ws2 = torch.empty(ctx.bwd_workspace_bytes(T, wl.d, wl.V, R, 148 * 128), dtype=torch.uint8, device="cuda")
+    dH2, dW2 = ctx.grpo_loss_bwd(cfg, H, W, y, cs, g["keep"], f["lse"], f["g"], workspace=ws2)
+    assert torch.equal(dH2, dH)
+    assert ((dW2 - dW).double().norm() / dW.double().norm()).item() < 1e-5
+    assert ctx.last_status() == 0
