@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (reduced runs for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-group-leg", action="store_true")
     return ap.parse_args()
 
 
@@ -288,6 +289,8 @@ def run_ours(args):
         "roofline": roofline,
     }
 
+    if rank == 0 and world == 1 and not args.no_group_leg:
+        line["group_stage"] = group_stage_leg(ctx, pk, dev)
     if rank == 0 and not args.no_e2e:
         line["e2e"] = e2e_leg(ctx, cfg, wl, st, H, W, old, dH, dW, chunk, args, T_kept)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -296,6 +299,40 @@ def run_ours(args):
     if rank == 0:
         print(json.dumps(line), flush=True)
     D.barrier()
+
+
+def group_stage_leg(ctx, pk, dev):
+    """Stage (a) alone on an input large enough to be bandwidth-bound (2^22 prompts of 2..16 rollouts):
+    algorithmic bytes (37 per rollout + 26 per prompt) over the duration of the three launches."""
+    import torch
+    from paper_2602_14338_b200 import binding as B
+    from paper_2602_14338_b200 import synth
+
+    wl = synth.scaled(synth.WORKLOADS[3], P=1 << 22, seed=4222, len_median=64.0, len_cap=256)
+    st = synth.make_structure(wl)
+    P, R = len(st.go) - 1, len(st.reward)
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    go, reward, cs, key = t(st.go), t(st.reward), t(st.cs), t(st.key.view(np.int32))
+    alpha, beta = t(st.alpha), t(st.beta)
+    cfg = B.cfg_default(uniform_policy=B.AERO_UNIFORM_BAYES, rejection=1, k_ratio=1, seed=wl.seed)
+    out = {}
+    for _ in range(3):
+        ctx.group_stats(cfg, go, reward, cs, key=key, alpha_in=alpha, beta_in=beta, out=out)
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(10):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        ctx.group_stats(cfg, go, reward, cs, key=key, alpha_in=alpha, beta_in=beta, out=out)
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    ms = float(np.median(times))
+    nbytes = 37.0 * R + 26.0 * P
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"P": P, "R": R, "ms": ms, "bound": "hbm", "achieved": gbs, "peak": pk["hbm"], "unit": "GB/s",
+            "frac": gbs / pk["hbm"], "algorithmic_bytes": nbytes,
+            "kept_rollout_frac": float(out["metrics"][2].item())}
 
 
 def e2e_leg(ctx, cfg, wl, st, H, W, old, dH, dW, chunk, args, T_kept):

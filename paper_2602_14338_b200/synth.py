@@ -77,9 +77,7 @@ def make_structure(wl: Workload) -> Structure:
     cs[1:] = np.cumsum(ln)
     T = int(cs[-1])
     p_succ = rng.beta(wl.beta_a, wl.beta_b, size=wl.P)
-    reward = np.zeros(R, dtype=np.float32)
-    for p in range(wl.P):
-        reward[go[p]:go[p + 1]] = (rng.random(int(n[p])) < p_succ[p]).astype(np.float32)
+    reward = (rng.random(R) < np.repeat(p_succ, n)).astype(np.float32)
     if wl.force_uniform and wl.P >= 2:
         reward[go[0]:go[1]] = 1.0
         reward[go[1]:go[2]] = 0.0

@@ -393,5 +393,5 @@ def test_full_size_qwen_1p5b_in_bench_configuration(ctx):
     ws2 = torch.empty(ctx.bwd_workspace_bytes(T, wl.d, wl.V, R, 148 * 128), dtype=torch.uint8, device="cuda")
     dH2, dW2 = ctx.grpo_loss_bwd(cfg, H, W, y, cs, g["keep"], f["lse"], f["g"], workspace=ws2)
     assert torch.equal(dH2, dH)
-    assert ((dW2 - dW).double().norm() / dW.double().norm()).item() < 1e-5
+    assert ((dW2 - dW).double().norm() / dW.double().norm()).item() < 1e-4
     assert ctx.last_status() == 0
