@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-group-leg", action="store_true")
+    ap.add_argument("--only-group-leg", action="store_true",
+                    help="run only the large-input group-stage measurement (for profiling that stage alone)")
     return ap.parse_args()
 
 
@@ -195,6 +197,10 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     pk = peaks()
+    if args.only_group_leg:
+        ctx = B.Context(local)
+        print(json.dumps({"group_stage": group_stage_leg(ctx, pk, dev)}), flush=True)
+        return
 
     base = synth.WORKLOADS[args.config]
     wl = synth.scaled(base, seed=base.seed + 100 * rank)      # an independent batch per replica
