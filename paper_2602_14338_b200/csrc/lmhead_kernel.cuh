@@ -8,10 +8,20 @@
 //   MODE_DZ  : dz = coef_t * (1[v == y_t] - exp(z - lse_t)) rounded to bf16 and stored to
 //              the chunk's scratch block (Eq. 3 through the softmax).
 //
+// CTAs work in pairs (a cluster of two, tcgen05 cta_group::2): the pair takes two token tiles,
+// one per CTA, and one MMA covers both (M = 256).  Each CTA stages its own 128 rows of H and
+// only half of the 256 W rows of the vocabulary tile; the tensor cores of the pair share the
+// two halves, so a CTA moves 32 KB per 64-deep slab instead of 48 KB.  Each CTA's TMEM holds
+// the 128 x 256 logits of its own token tile.
+//
 // Warp roles (192 threads, one CTA per SM): warps 0-3 epilogue (warp q reads TMEM lanes
-// 32q..32q+31, one token row per thread), warp 4 TMA producer, warp 5 MMA issuer and TMEM
-// owner.  Two 256-column TMEM accumulators let the MMA of vocabulary tile j+1 overlap
-// the epilogue of tile j.
+// 32q..32q+31, one token row per thread), warp 4 TMA producer, warp 5 TMEM owner and, in the
+// CTA of cluster rank 0, MMA issuer for the pair.  Two 256-column TMEM accumulators let the
+// MMA of vocabulary tile j+1 overlap the epilogue of tile j.
+//
+// Barriers: full[s] lives in the rank-0 CTA and collects the bytes of both CTAs' loads;
+// empty[s] and tfull[b] exist in both CTAs and are signalled for both by the issuer's commits;
+// tempty[b] lives in the rank-0 CTA and counts the eight epilogue warps of the pair.
 #pragma once
 
 #include "loss_common.cuh"
@@ -20,10 +30,11 @@
 namespace lmhead {
 
 #ifndef AERO_TC_STAGES
-#define AERO_TC_STAGES 4          // depth of the TMA -> MMA shared-memory ring
+#define AERO_TC_STAGES 6          // depth of the TMA -> MMA shared-memory ring
 #endif
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = AERO_TC_STAGES, UMMA_K = 16;
-constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+// BM rows of H per CTA, BN vocabulary columns per accumulator, BNH of them staged by each CTA
+constexpr int BM = 128, BN = 256, BNH = BN / 2, BK = 64, STAGES = AERO_TC_STAGES, UMMA_K = 16;
+constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BNH * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
 constexpr int MODE_FWD = 0, MODE_DZ = 1;
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
@@ -76,7 +87,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW,
               const __grid_constant__ CUtensorMap tmDZ, const Params p) {
   extern __shared__ uint8_t smem_raw[];
@@ -85,16 +96,20 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
   Ctl* ctl = reinterpret_cast<Ctl*>(stg_all + STG_BYTES);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+  const uint32_t rank = tc::cluster_ctarank();        // 0 issues the MMAs of the pair
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&ctl->full[s], 1); tc::mbar_init(&ctl->empty[s], 1); }
-    for (int b = 0; b < 2; ++b) { tc::mbar_init(&ctl->tfull[b], 1); tc::mbar_init(&ctl->tempty[b], 4); }
+    for (int b = 0; b < 2; ++b) { tc::mbar_init(&ctl->tfull[b], 1); tc::mbar_init(&ctl->tempty[b], 8); }
     ctl->abort = 0;
     tc::fence_barrier_init();
   }
   if (warp == 4 && lane == 0) { tc::prefetch_tmap(&tmH); tc::prefetch_tmap(&tmW); }
-  if (warp == 5) { tc::tmem_alloc(&ctl->tmem_base, 512); tc::tmem_relinquish(); }
+  if (warp == 5) { tc::tmem_alloc_pair(&ctl->tmem_base, 512); tc::tmem_relinquish_pair(); }
   tc::tc_fence_before();
   __syncthreads();
+  tc::cluster_sync_all();        // the peer's barriers exist before anything signals them
   tc::tc_fence_after();
   const uint32_t tmem_base = ctl->tmem_base;
   volatile int* abort_flag = &ctl->abort;
@@ -102,34 +117,39 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
   const int n_tiles = min(*p.n_tiles, p.tile_end);
   const int nkb = p.d / BK;
   const int nvt = (p.V + BN - 1) / BN;
+  // The pair's k-th unit is token tiles first, first + 1 (the second may not exist: its CTA
+  // then stages the first tile's rows again and discards the result).
+  auto unit_first = [&](int k) { return p.tile_begin + 2 * (pair + k * npairs); };
 
   if (warp == 4) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = p.tile_begin + blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
-        const int row0 = p.tile_row[tile];
+      for (int k = 0; ok && unit_first(k) < n_tiles; ++k) {
+        const int mine = unit_first(k) + (int)rank;
+        const int row0 = p.tile_row[mine < n_tiles ? mine : unit_first(k)];
         for (int j = 0; ok && j < nvt; ++j) {
           for (int kb = 0; kb < nkb; ++kb, ++it) {
             const int s = it % STAGES;
             const uint32_t ph = (it / STAGES) & 1u;
             if (!tc::mbar_wait(&ctl->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
             uint8_t* a_s = smem + (size_t)s * STAGE_BYTES;
-            tc::mbar_arrive_expect_tx(&ctl->full[s], STAGE_BYTES);
-            tc::tma_load_2d(a_s, &tmH, kb * BK, row0, &ctl->full[s]);
-            tc::tma_load_2d(a_s + A_BYTES, &tmW, kb * BK, j * BN, &ctl->full[s]);
+            const uint32_t full0 = tc::mapa_shared(tc::smem_u32(&ctl->full[s]), 0);
+            if (rank == 0) tc::mbar_arrive_expect_tx(&ctl->full[s], 2 * STAGE_BYTES);
+            tc::tma_load_2d_pair(a_s, &tmH, kb * BK, row0, full0);
+            tc::tma_load_2d_pair(a_s + A_BYTES, &tmW, kb * BK, j * BN + (int)rank * BNH, full0);
           }
         }
       }
     }
   } else if (warp == 5) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = tc::make_idesc_bf16(BM, BN, 0, 0);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = tc::make_idesc_bf16(2 * BM, BN, 0, 0);
       uint32_t it = 0, at = 0;
       bool ok = true;
-      for (int tile = p.tile_begin + blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+      for (int k = 0; ok && unit_first(k) < n_tiles; ++k) {
         for (int j = 0; ok && j < nvt; ++j, ++at) {
           const uint32_t buf = at & 1u, aph = (at >> 1) & 1u;
           if (!tc::mbar_wait(&ctl->tempty[buf], aph ^ 1u, abort_flag)) { ok = false; break; }
@@ -146,11 +166,11 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
 #pragma unroll
             for (int kk = 0; kk < BK / UMMA_K; ++kk) {
               // advance 32 bytes (16 bf16) inside the 128-byte swizzle row: +2 in 16-byte units
-              tc::umma_bf16(tmem_d, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
+              tc::umma_bf16_pair(tmem_d, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb | kk) != 0 ? 1u : 0u);
             }
-            tc::umma_commit(&ctl->empty[s]);     // frees the stage when these MMAs retire
+            tc::umma_commit_pair(&ctl->empty[s], 3);     // frees the stage in both CTAs when these MMAs retire
           }
-          if (ok) tc::umma_commit(&ctl->tfull[buf]);
+          if (ok) tc::umma_commit_pair(&ctl->tfull[buf], 3);
         }
       }
     }
@@ -160,9 +180,11 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
     bool ok = true;
     const int r_in_tile = warp * 32 + lane;
     uint8_t* stg_warp = stg_all + warp * 2 * STG_BUF_BYTES;
-    for (int tile = p.tile_begin + blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
-      const long long row = (long long)p.tile_row[tile] + r_in_tile;
-      const bool valid_row = r_in_tile < p.tile_valid[tile] && row < p.T;
+    for (int k = 0; ok && unit_first(k) < n_tiles; ++k) {
+      const int tile = unit_first(k) + (int)rank;
+      const bool have_tile = tile < n_tiles;
+      const long long row = have_tile ? (long long)p.tile_row[tile] + r_in_tile : 0;
+      const bool valid_row = have_tile && r_in_tile < p.tile_valid[tile] && row < p.T;
       int yt = -1;
       if (valid_row) yt = p.y[row];
       const bool bad_y = valid_row && (yt < 0 || yt >= p.V);
@@ -181,6 +203,13 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
         // the TMEM loads below are warp-collective: take the decision for the whole warp
         if (!__all_sync(0xffffffffu, tc::mbar_wait(&ctl->tfull[buf], aph, abort_flag))) { ok = false; break; }
         tc::tc_fence_after();
+        if (!have_tile) {
+          // nothing to read: hand the accumulator straight back
+          tc::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive_cluster(tc::mapa_shared(tc::smem_u32(&ctl->tempty[buf]), 0));
+          continue;
+        }
         const int col_base = j * BN;
         const int ncol = min(BN, (MODE == MODE_DZ ? (int)p.ldz : p.V) - col_base);
         const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + buf * BN;
@@ -278,10 +307,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
         }
         tc::tc_fence_before();
         __syncwarp();
-        if (lane == 0) tc::mbar_arrive(&ctl->tempty[buf]);
+        if (lane == 0) tc::mbar_arrive_cluster(tc::mapa_shared(tc::smem_u32(&ctl->tempty[buf]), 0));
       }
 
-      if (MODE == MODE_FWD && ok) {
+      if (MODE == MODE_FWD && ok && have_tile) {
         double part[kPartialStride] = {0.0, 0.0, 0.0, 0.0, 0.0};
         if (live) {
           const float ls = (m2 + __log2f(l)) * kLn2;
@@ -323,10 +352,13 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
   }
   tc::tc_fence_before();
   __syncthreads();
+  // neither CTA may leave, or free its TMEM, while the other can still signal its barriers,
+  // read its shared memory or write its accumulators
+  tc::cluster_sync_all();
   if (threadIdx.x == 0 && *abort_flag) aero_raise(p.status, AERO_ST_TIMEOUT);
   if (warp == 5) {
     tc::tc_fence_after();
-    tc::tmem_dealloc(tmem_base, 512);
+    tc::tmem_dealloc_pair(tmem_base, 512);
   }
 }
 

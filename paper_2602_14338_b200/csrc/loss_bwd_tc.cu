@@ -66,7 +66,7 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
   const uint64_t dz_rows = (uint64_t)tpc * lmhead::BM;
   // K-major views (inner extent 64 = one 128-byte swizzle row) for the recompute and for dz as A of dH
   if ((rc = aero_make_tmap_2d(ctx, &tmH_k, BF, 2, H, T, d, d, lmhead::BM, 64))) return rc;
-  if ((rc = aero_make_tmap_2d(ctx, &tmW_k, BF, 2, W, V, d, d, lmhead::BN, 64))) return rc;
+  if ((rc = aero_make_tmap_2d(ctx, &tmW_k, BF, 2, W, V, d, d, lmhead::BNH, 64))) return rc;
   if ((rc = aero_make_tmap_2d(ctx, &tmDZ_k, BF, 2, dz, dz_rows, ldz, ldz, gemmbwd::BM, 64))) return rc;
   // MN-major operands: blocked views, one box = 64 rows x (4 or 2) column blocks of 64
   if ((rc = aero_make_tmap_blocked(ctx, &tmW_mn, W, V, d, d, 64, gemmbwd::BN / 64))) return rc;
@@ -92,7 +92,9 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     lp.tile_begin = (int)begin; lp.tile_end = (int)(begin + tpc);
     lp.y = y; lp.status = ctx->d_status;
     lp.lse_in = lse; lp.g_in = g; lp.grad_scale = grad_scale; lp.dz = dz; lp.ldz = ldz;
-    const int grid_dz = (int)(tpc < ctx->sm_count ? tpc : ctx->sm_count);
+    const long long max_pairs = ctx->sm_count / 2 > 0 ? ctx->sm_count / 2 : 1;
+    const long long dz_pairs = (tpc + 1) / 2;
+    const int grid_dz = 2 * (int)(dz_pairs < max_pairs ? dz_pairs : max_pairs);
     k_dz<<<grid_dz, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH_k, tmW_k, tmDZ_st, lp);
 
     gemmbwd::Params gp = {};

@@ -46,7 +46,7 @@ int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
                            lmhead::BM, lmhead::BK);
     if (rc) return rc;
     rc = aero_make_tmap_2d(ctx, &tmW, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, W, (uint64_t)V, (uint64_t)d, (uint64_t)d,
-                           lmhead::BN, lmhead::BK);
+                           lmhead::BNH, lmhead::BK);
     if (rc) return rc;
     lmhead::Params p = {};
     p.T = T; p.d = d; p.V = V; p.R = R;
@@ -58,8 +58,10 @@ int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     p.logp = logp; p.lse_out = lse; p.g_out = g; p.partials = f.partials;
     auto kern = lmhead::lmhead_kernel<lmhead::MODE_FWD>;
     AERO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lmhead::SMEM_BYTES));
-    const int64_t upper = T / lmhead::BM + R + 1;
-    const int grid = (int)(upper < ctx->sm_count ? upper : ctx->sm_count);
+    // one CTA pair per two token tiles, at most one pair per two SMs
+    const int64_t upper_pairs = (T / lmhead::BM + R + 2) / 2;
+    const int64_t max_pairs = ctx->sm_count / 2 > 0 ? ctx->sm_count / 2 : 1;
+    const int grid = 2 * (int)(upper_pairs < max_pairs ? upper_pairs : max_pairs);
     kern<<<grid, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH, tmW, tmH, p);   // third map unused in forward mode
     ctx->launches += 1;
     AERO_CUDA_TRY(cudaGetLastError());
