@@ -145,7 +145,9 @@ int aero_last_status(aero_ctx* ctx, uint32_t* bits);
  *             all correct + the min(k*c, n-c) incorrect of smallest (key, index),
  *             where low-success means Partial, or c*n_explore <= rescue_S*n when
  *             rescue_S > 0;  any other group: all present rollouts;
- *   advantage mixed group: (r - mean)/(std + eps_std) with the population std over
+ *   advantage (r enters as the bit r > 0.5; a reward other than 0 or 1 raises
+ *             AERO_ST_BAD_REWARD)
+ *             mixed group: (r - mean)/(std + eps_std) with the population std over
  *             the kept subset (STATS_KEPT) or the present group (STATS_ALL);
  *             uniform group under BAYES: (r - u~)/(sqrt(u~(1-u~)) + eps_std);
  *             0 for every rollout that is not kept;
@@ -188,18 +190,23 @@ int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
  * device memory, or a latency-bound loop that must not call the allocator because an
  * allocation can synchronise the whole device.  Instead of a caller workspace, the scratch
  * is a fixed array in device memory that belongs to the loaded library itself: about
- * 1.4 MB per GPU that loads the library, held until the process exits, sized for at most
- * AERO_STATIC_MAX_PROMPTS prompts (R is not limited).  A larger P returns
- * AERO_ERR_TOO_LARGE and launches nothing.  The call, and everything it calls, performs
- * no cudaMalloc/cudaFree and uses no allocating library routine.
+ * 1.2 MB per GPU that loads the library, held until the process exits, sized for at most
+ * AERO_STATIC_MAX_PROMPTS prompts in at most 16384 tiles (the stage works on tiles of up to
+ * 256 consecutive prompts holding about 1800 rollouts, so the tile limit only binds when
+ * P > 16384 and the mean group has more than about 450 rollouts; R itself is not limited).
+ * A batch beyond either limit returns AERO_ERR_TOO_LARGE and launches nothing.  The call,
+ * and everything it calls, performs no cudaMalloc/cudaFree and uses no allocating library
+ * routine.
  *
  * The first call on each device looks up the array's device address (once per device,
  * with that device current); make that first call outside any stream capture.
  * All calls on a device share the one array: two calls whose kernels may overlap on the
  * GPU (different streams, or different contexts of this library on one device) race on
  * it -- order them on one stream or with events.  The array keeps the previous call's
- * contents; nothing in it needs clearing, because each call writes every word it later
- * reads.  Arguments, outputs and status bits are those of aero_group_stats.
+ * contents; each call clears the words that must start at zero (the scan records and the
+ * tile counters at its head, with one asynchronous memset on the context's stream) and
+ * writes every other word before reading it.  Arguments, outputs and status bits are
+ * those of aero_group_stats.
  */
 #define AERO_STATIC_MAX_PROMPTS 65536
 

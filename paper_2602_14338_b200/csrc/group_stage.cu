@@ -131,6 +131,8 @@ struct Args {
 // Per-prompt state of a tile (shared memory, one entry per prompt of the tile).
 struct PromptState {
   int lo[kMaxPT + 1];        // rollout range of each prompt, relative to the tile's first rollout
+  unsigned nc[kMaxPT];       // present rollouts | correct ones << 16   (staged path)
+  unsigned kb[kMaxPT];       // kept rollouts | kept correct ones << 16 (staged path)
   int quota[kMaxPT];
   uint8_t mode[kMaxPT];      // 0 keep all present, 1 keep none, 2 select by rank
   uint8_t reject[kMaxPT];    // select among the incorrect only, keep every correct one
@@ -138,75 +140,35 @@ struct PromptState {
   float ut[kMaxPT];
   float mu[kMaxPT];
   float inv[kMaxPT];
-  int nk[kMaxPT];            // kept rollouts, then their exclusive prefix inside the tile
-  long long ktok[kMaxPT];    // kept tokens, then their exclusive prefix inside the tile
+  int nk[kMaxPT];            // global path: kept rollouts, then their exclusive prefix inside the tile
+  long long ktok[kMaxPT];    // global path: kept tokens, then their exclusive prefix inside the tile
 };
 
-// Per-rollout staging of a tile.  `ck` is the selection key (key << 32 | local index) of a
-// candidate and kNone otherwise; after selection the same words hold the token offset of a
-// kept rollout inside the tile, and `len` its position among the tile's kept rollouts.
+// Per-rollout staging of a tile.  `ck` orders the candidates of a selection:
+// correct << 63 | key << 16 | local index for a present rollout, all ones for an absent one, so
+// that in a group that selects among its incorrect rollouts no correct one ever compares
+// smaller.  After the selection the same words hold a kept rollout's token offset inside its
+// 32-rollout chunk, and `len` its position among the chunk's kept rollouts.
+constexpr int kChunks = kCap / 32;
 struct RolloutStage {
   unsigned long long ck[kCap];
   int len[kCap];
-  float r[kCap];
   uint16_t pid[kCap];
-  uint8_t flag[kCap];        // bit 0 present, bit 1 kept
+  uint8_t flag[kCap];        // bit 0 present, bit 1 correct, bit 2 kept
+  long long chunk_tok[kChunks];   // kept tokens per chunk, then their exclusive prefix inside the tile
+  int chunk_cnt[kChunks];
 };
 
 struct TileShared {
   PromptState ps;
   RolloutStage rs;
+  TilePartial red[kThreads / 32];
   long long warp_tok[kThreads / 32];
   int warp_cnt[kThreads / 32];
   long long base_tok;
   int base_roll;
   int tile;
   int failed;
-  TilePartial part;
-};
-
-// Rollout accessors: from the staging area when the tile fits (STAGED), else from the
-// caller's arrays.
-template <bool STAGED>
-struct Acc {
-  const Args& a;
-  TileShared& sh;
-  int r0;          // first rollout of the tile
-  __device__ __forceinline__ bool present(int j) const {
-    if (STAGED) return sh.rs.flag[j] & 1;
-    return a.keep_in ? a.keep_in[r0 + j] != 0 : true;
-  }
-  __device__ __forceinline__ float r(int j) const { return STAGED ? sh.rs.r[j] : a.reward[r0 + j]; }
-  __device__ __forceinline__ long long len(int j) const {
-    if (STAGED) return sh.rs.len[j];
-    const long long l = a.cs[r0 + j + 1] - a.cs[r0 + j];
-    return l > 0 ? l : 0;
-  }
-  __device__ __forceinline__ uint32_t key(int j) const {
-    return a.key ? a.key[r0 + j] : default_key(a.cfg.seed, (uint32_t)(r0 + j));
-  }
-  __device__ __forceinline__ bool kept(int j) const {
-    return STAGED ? (sh.rs.flag[j] & 2) != 0 : a.keep[r0 + j] != 0;
-  }
-  __device__ __forceinline__ void set_kept(int j, bool k) const {
-    if (STAGED) sh.rs.flag[j] = (uint8_t)((sh.rs.flag[j] & 1) | (k ? 2 : 0));
-    else a.keep[r0 + j] = k ? 1 : 0;
-  }
-  // selection key of rollout j in a group that selects (kNone: not a candidate)
-  __device__ __forceinline__ unsigned long long ck(int j, bool reject) const {
-    if (STAGED) return sh.rs.ck[j];
-    if (!present(j) || (reject && r(j) > 0.5f)) return kNone;
-    return ((unsigned long long)key(j) << 32) | (unsigned)j;
-  }
-  __device__ __forceinline__ int pid(int j, int npt) const {
-    if (STAGED) return sh.rs.pid[j];
-    int lo = 0, hi = npt;                 // last prompt whose range starts at or before j
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (sh.ps.lo[mid] <= j) lo = mid; else hi = mid;
-    }
-    return lo;
-  }
 };
 
 __device__ __forceinline__ bool aborted(const Workspace& ws) {
@@ -229,7 +191,7 @@ __device__ bool scan_predecessors(const Workspace& ws, int tile, int lane, int* 
         const bool give_up = aborted(ws) || timer_ns() - t0 > kSpinLimitNs;
         if (__any_sync(0xffffffffu, give_up)) return false;
       }
-      __nanosleep(64);
+      __nanosleep(200);
     }
     if (!done_r) {
       const unsigned m = __ballot_sync(0xffffffffu, (vr >> 62) == 2);
@@ -255,264 +217,371 @@ __device__ bool scan_predecessors(const Workspace& ws, int tile, int lane, int* 
   return true;
 }
 
-template <bool STAGED>
-__device__ void run_tile(const Args& a, const Workspace& ws, TileShared& sh, int tile, int p0, int npt, int r0, int nroll,
-                         uint32_t& st) {
-  const Acc<STAGED> acc{a, sh, r0};
-  const int tid = threadIdx.x;
-  PromptState& ps = sh.ps;
+// Publish the tile's totals, sum the predecessors', publish the running totals (warp 0).
+// Leaves the totals of all earlier tiles in sh.base_roll / sh.base_tok.
+__device__ void chain_tile(const Workspace& ws, TileShared& sh, int tile, int tile_cnt, long long tile_tok, uint32_t& st) {
+  const int lane = threadIdx.x;
+  if (lane == 0 && tile > 0) {
+    st_release(ws.desc_roll + tile, kFlagAgg | (unsigned long long)tile_cnt);
+    st_release(ws.desc_tok + tile, kFlagAgg | (unsigned long long)tile_tok);
+  }
+  int excl_roll = 0;
+  long long excl_tok = 0;
+  const bool ok = scan_predecessors(ws, tile, lane, &excl_roll, &excl_tok);
+  if (lane == 0) {
+    if (ok) {
+      st_release(ws.desc_roll + tile, kFlagPrefix | (unsigned long long)(excl_roll + tile_cnt));
+      st_release(ws.desc_tok + tile, kFlagPrefix | (unsigned long long)(excl_tok + tile_tok));
+    } else {
+      atomicExch(ws.ctrl + 2, 1u);
+      st |= AERO_ST_TIMEOUT;
+    }
+    sh.failed = ok ? 0 : 1;
+    sh.base_roll = excl_roll;
+    sh.base_tok = excl_tok;
+  }
+}
 
-  // ---- stage the rollouts (one thread per rollout, coalesced) ----
+// Category, posterior and curation rule of one prompt from its counts (Appendix C; Sec. 4.2).
+struct Rule {
+  int category, mode;
+  long long quota;
+  bool reject, uniform;
+  float al, be, ut;
+};
+__device__ __forceinline__ Rule decide(const Args& a, int p, int n, int c) {
+  Rule r;
+  if (n == 0) r.category = AERO_CAT_EMPTY;
+  else if (c == 0) r.category = AERO_CAT_ZERO;
+  else if (c == n) r.category = AERO_CAT_PERFECT;
+  else if (2 * c < n) r.category = AERO_CAT_PARTIAL;
+  else r.category = AERO_CAT_GOOD;
+  r.al = (a.alpha_in ? a.alpha_in[p] : a.cfg.alpha0) + (float)c;
+  r.be = (a.beta_in ? a.beta_in[p] : a.cfg.beta0) + (float)(n - c);
+  r.ut = r.al / (r.al + r.be);
+  r.uniform = (c == 0 || c == n);
+  r.mode = 0;
+  r.quota = 0;
+  r.reject = false;
+  if (n == 0) {
+    r.mode = 1;
+  } else if (r.uniform) {
+    if (a.cfg.uniform_policy == AERO_UNIFORM_MASK) r.mode = 1;
+    else if (a.cfg.n_keep_uniform > 0 && a.cfg.n_keep_uniform < n) { r.mode = 2; r.quota = a.cfg.n_keep_uniform; }
+  } else {
+    const bool low = r.category == AERO_CAT_PARTIAL ||
+                     (a.cfg.rescue_S > 0 && (long long)c * a.cfg.n_explore <= (long long)a.cfg.rescue_S * n);
+    if (a.cfg.rejection && low) {
+      const long long m = min((long long)a.cfg.k_ratio * c, (long long)(n - c));
+      if (m < n - c) { r.mode = 2; r.quota = m; r.reject = true; }
+    }
+  }
+  return r;
+}
+
+// Metrics record of the tile: shuffle tree per warp, warps added in order by thread 0.
+__device__ __forceinline__ void reduce_partial(TileShared& sh, TilePartial mine) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mine.present_tok += __shfl_xor_sync(0xffffffffu, mine.present_tok, o);
+    mine.present_roll += __shfl_xor_sync(0xffffffffu, mine.present_roll, o);
+    mine.surv += __shfl_xor_sync(0xffffffffu, mine.surv, o);
+#pragma unroll
+    for (int k = 0; k < 5; ++k) mine.cat[k] += __shfl_xor_sync(0xffffffffu, mine.cat[k], o);
+    mine.abs_adv += __shfl_xor_sync(0xffffffffu, mine.abs_adv, o);
+  }
+  if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = mine;
+}
+__device__ __forceinline__ TilePartial sum_partials(const TileShared& sh) {
+  TilePartial tot = {};
+  for (int k = 0; k < kThreads / 32; ++k) {
+    tot.present_tok += sh.red[k].present_tok; tot.present_roll += sh.red[k].present_roll; tot.surv += sh.red[k].surv;
+    for (int c = 0; c < 5; ++c) tot.cat[c] += sh.red[k].cat[c];
+    tot.abs_adv += sh.red[k].abs_adv;
+  }
+  return tot;
+}
+
+// A tile whose rollouts fit the staging area.  Rewards enter as the bit r > 0.5 (they must be
+// exactly 0 or 1; anything else raises AERO_ST_BAD_REWARD), so per-prompt sums are counts,
+// gathered with shared-memory atomics, and mean and deviation are closed forms of the counts.
+__device__ void run_tile_staged(const Args& a, const Workspace& ws, TileShared& sh, int tile, int p0, int npt, int r0,
+                                int nroll, uint32_t& st) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  PromptState& ps = sh.ps;
+  RolloutStage& rs = sh.rs;
+
+  // ---- which prompt owns which rollout ----
+  if (tid < npt) {
+    for (int j = ps.lo[tid]; j < ps.lo[tid + 1]; ++j) rs.pid[j] = (uint16_t)tid;
+    ps.nc[tid] = 0;
+    ps.kb[tid] = 0;
+  }
+  __syncthreads();
+
+  // ---- stage the rollouts (coalesced) and count per prompt ----
+  TilePartial mine = {};
   for (int j = tid; j < nroll; j += kThreads) {
     const int i = r0 + j;
     const bool pres = a.keep_in ? a.keep_in[i] != 0 : true;
     const float r = a.reward[i];
     const long long len = a.cs[i + 1] - a.cs[i];
+    const bool corr = r > 0.5f;
+    unsigned long long ck = kNone;
     if (pres) {
       if (r != 0.f && r != 1.f) st |= AERO_ST_BAD_REWARD;
       if (len < 0) st |= AERO_ST_BAD_OFFSETS;
       if (len == 0) st |= AERO_ST_EMPTY_ROLLOUT;
+      const uint32_t key = a.key ? a.key[i] : default_key(a.cfg.seed, (uint32_t)i);
+      ck = (corr ? 1ull << 63 : 0ull) | ((unsigned long long)key << 16) | (unsigned)j;
+      atomicAdd(&ps.nc[rs.pid[j]], corr ? 0x10001u : 1u);
+      mine.present_tok += len > 0 ? len : 0;
+      mine.present_roll += 1;
     }
-    if (STAGED) {
-      sh.rs.flag[j] = pres ? 1 : 0;
-      sh.rs.r[j] = r;
-      sh.rs.len[j] = len > 0 ? (int)(len < 0x7fffffffLL ? len : 0x7fffffffLL) : 0;
-      sh.rs.ck[j] = kNone;
-    }
+    rs.ck[j] = ck;
+    rs.len[j] = len > 0 ? (int)(len < 0x7fffffffLL ? len : 0x7fffffffLL) : 0;
+    rs.flag[j] = (uint8_t)((pres ? 1 : 0) | (corr ? 2 : 0));
   }
   __syncthreads();
 
-  // ---- per prompt: counts, category, posterior, curation rule ----
-  TilePartial mine = {};
+  // ---- per prompt: category, posterior, curation rule ----
   if (tid < npt) {
-    const int q = tid, p = p0 + q;
-    const int lo = ps.lo[q], hi = ps.lo[q + 1];
-    int n = 0, c = 0;
-    long long ptok = 0;
-    for (int j = lo; j < hi; ++j) {
-      if (STAGED) sh.rs.pid[j] = (uint16_t)q;
-      if (acc.present(j)) { n += 1; c += acc.r(j) > 0.5f ? 1 : 0; ptok += acc.len(j); }
-    }
-    int category;
-    if (n == 0) category = AERO_CAT_EMPTY;
-    else if (c == 0) category = AERO_CAT_ZERO;
-    else if (c == n) category = AERO_CAT_PERFECT;
-    else if (2 * c < n) category = AERO_CAT_PARTIAL;
-    else category = AERO_CAT_GOOD;
-
-    const float al = (a.alpha_in ? a.alpha_in[p] : a.cfg.alpha0) + (float)c;
-    const float be = (a.beta_in ? a.beta_in[p] : a.cfg.beta0) + (float)(n - c);
-    const float ut = al / (al + be);
-    a.cat[p] = (uint8_t)category;
-    a.u_tilde[p] = ut;
-    a.alpha_out[p] = al;
-    a.beta_out[p] = be;
-
-    const bool uniform = (c == 0 || c == n);
-    int mode = 0;
-    long long quota = 0;
-    bool reject = false;
-    if (n == 0) {
-      mode = 1;
-    } else if (uniform) {
-      if (a.cfg.uniform_policy == AERO_UNIFORM_MASK) mode = 1;
-      else if (a.cfg.n_keep_uniform > 0 && a.cfg.n_keep_uniform < n) { mode = 2; quota = a.cfg.n_keep_uniform; }
-    } else {
-      const bool low = category == AERO_CAT_PARTIAL ||
-                       (a.cfg.rescue_S > 0 && (long long)c * a.cfg.n_explore <= (long long)a.cfg.rescue_S * n);
-      if (a.cfg.rejection && low) {
-        const long long m = min((long long)a.cfg.k_ratio * c, (long long)(n - c));
-        if (m < n - c) { mode = 2; quota = m; reject = true; }
-      }
-    }
-    ps.mode[q] = (uint8_t)mode;
-    ps.reject[q] = reject ? 1 : 0;
-    ps.quota[q] = (int)quota;
-    ps.uniform[q] = uniform ? 1 : 0;
-    ps.ut[q] = ut;
-    if (STAGED && mode == 2) {
-      for (int j = lo; j < hi; ++j)
-        if (acc.present(j) && !(reject && acc.r(j) > 0.5f))
-          sh.rs.ck[j] = ((unsigned long long)acc.key(j) << 32) | (unsigned)j;
-    }
-    mine.present_tok = ptok;
-    mine.present_roll = n;
-    mine.cat[category] = 1;
+    const int p = p0 + tid;
+    const int n = (int)(ps.nc[tid] & 0xffffu), c = (int)(ps.nc[tid] >> 16);
+    const Rule ru = decide(a, p, n, c);
+    a.cat[p] = (uint8_t)ru.category;
+    a.u_tilde[p] = ru.ut;
+    a.alpha_out[p] = ru.al;
+    a.beta_out[p] = ru.be;
+    ps.mode[tid] = (uint8_t)ru.mode;
+    ps.reject[tid] = ru.reject ? 1 : 0;
+    ps.quota[tid] = (int)ru.quota;
+    ps.uniform[tid] = ru.uniform ? 1 : 0;
+    ps.ut[tid] = ru.ut;
+    mine.cat[ru.category] = 1;
   }
   __syncthreads();
 
   // ---- per rollout: keep decision (rank among the group's candidates) ----
   for (int j = tid; j < nroll; j += kThreads) {
-    const int q = acc.pid(j, npt);
+    const int q = rs.pid[j];
     const int mode = ps.mode[q];
-    bool kp = acc.present(j) && mode != 1;
-    if (kp && mode == 2) {
-      const bool reject = ps.reject[q] != 0;
-      const unsigned long long mykey = acc.ck(j, reject);
-      if (mykey != kNone) {
-        const int lo = ps.lo[q], hi = ps.lo[q + 1];
-        int rank = 0;
-        for (int k = lo; k < hi; ++k) rank += acc.ck(k, reject) < mykey ? 1 : 0;
-        kp = rank < ps.quota[q];
-      }
+    const uint8_t f = rs.flag[j];
+    bool kp = (f & 1) && mode != 1;
+    if (kp && mode == 2 && !(ps.reject[q] && (f & 2))) {
+      const unsigned long long mykey = rs.ck[j];
+      const int lo = ps.lo[q], hi = ps.lo[q + 1];
+      int rank = 0;
+      for (int k = lo; k < hi; ++k) rank += rs.ck[k] < mykey ? 1 : 0;
+      kp = rank < ps.quota[q];
     }
-    acc.set_kept(j, kp);
+    if (kp) {
+      rs.flag[j] = f | 4;
+      atomicAdd(&ps.kb[q], (f & 2) ? 0x10001u : 1u);
+    }
   }
   __syncthreads();
 
-  // ---- per prompt: statistics over the base set, kept totals ----
+  // ---- per prompt: mean and deviation of the base set; per chunk of 32 rollouts: kept counts and tokens ----
   if (tid < npt) {
-    const int q = tid, p = p0 + q;
-    const int lo = ps.lo[q], hi = ps.lo[q + 1];
-    int nk = 0, nbase = 0;
-    long long ktok = 0;
-    float sum_r = 0.f;
-    for (int j = lo; j < hi; ++j) {
-      const bool kp = acc.kept(j);
-      if (kp) { nk += 1; ktok += acc.len(j); }
-      const bool in_base = a.cfg.stats_over == AERO_STATS_KEPT ? kp : acc.present(j);
-      if (in_base) { nbase += 1; sum_r += acc.r(j); }
-    }
+    const int p = p0 + tid;
+    const int nk = (int)(ps.kb[tid] & 0xffffu), ck = (int)(ps.kb[tid] >> 16);
+    const bool over_kept = a.cfg.stats_over == AERO_STATS_KEPT;
+    const int nb = over_kept ? nk : (int)(ps.nc[tid] & 0xffffu);
+    const int cb = over_kept ? ck : (int)(ps.nc[tid] >> 16);
     float mu = 0.f, sd = 0.f;
-    if (ps.uniform[q]) {
-      mu = ps.ut[q];
+    if (ps.uniform[tid]) {
+      mu = ps.ut[tid];
       sd = sqrtf(mu * (1.f - mu));
-    } else if (nbase > 0) {
-      mu = sum_r / (float)nbase;
-      float ss = 0.f;
-      for (int j = lo; j < hi; ++j) {
-        const bool in_base = a.cfg.stats_over == AERO_STATS_KEPT ? acc.kept(j) : acc.present(j);
-        if (in_base) { const float dlt = acc.r(j) - mu; ss += dlt * dlt; }
-      }
-      sd = sqrtf(ss / (float)nbase);
+    } else if (nb > 0) {
+      mu = (float)cb / (float)nb;
+      const float d1 = 1.f - mu;
+      sd = sqrtf(((float)cb * d1 * d1 + (float)(nb - cb) * mu * mu) / (float)nb);
     }
     const float inv = 1.f / (sd + a.cfg.eps_std);
-    float abs_adv = 0.f;
-    for (int j = lo; j < hi; ++j)
-      if (acc.kept(j)) abs_adv += fabsf((acc.r(j) - mu) * inv);
-    ps.mu[q] = mu;
-    ps.inv[q] = inv;
-    ps.nk[q] = nk;
-    ps.ktok[q] = ktok;
+    ps.mu[tid] = mu;
+    ps.inv[tid] = inv;
     a.gmask[p] = nk > 0 ? 1 : 0;
     if (a.cfg.agg != AERO_TOKEN_MEAN) ws.nkept[p] = nk;
     mine.surv = nk > 0 ? 1 : 0;
-    mine.abs_adv = abs_adv;
+    mine.abs_adv = ((float)ck * fabsf(1.f - mu) + (float)(nk - ck) * fabsf(mu)) * inv;
   }
-
-  // ---- tile totals and exclusive prefixes over the tile's prompts (block scan, fixed order) ----
-  {
-    const int lane = tid & 31, warp = tid >> 5;
-    int cnt = tid < npt ? ps.nk[tid] : 0;
-    long long tok = tid < npt ? ps.ktok[tid] : 0;
-    const int my_cnt = cnt;
-    const long long my_tok = tok;
+  for (int j0 = warp * 32; j0 < nroll; j0 += kThreads) {     // whole warps: the scan is warp-wide
+    const int j = j0 + lane;
+    const bool kp = j < nroll && (rs.flag[j] & 4);
+    const unsigned kept_mask = __ballot_sync(0xffffffffu, kp);
+    long long tok = kp ? rs.len[j] : 0;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const int c2 = __shfl_up_sync(0xffffffffu, cnt, o);
       const long long t2 = __shfl_up_sync(0xffffffffu, tok, o);
-      if (lane >= o) { cnt += c2; tok += t2; }
+      if (lane >= o) tok += t2;
     }
-    if (lane == 31) { sh.warp_cnt[warp] = cnt; sh.warp_tok[warp] = tok; }
-    // metrics record of the tile: shuffle tree per warp, warps added in order by thread 0
-    TilePartial red = mine;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      red.present_tok += __shfl_xor_sync(0xffffffffu, red.present_tok, o);
-      red.present_roll += __shfl_xor_sync(0xffffffffu, red.present_roll, o);
-      red.surv += __shfl_xor_sync(0xffffffffu, red.surv, o);
-#pragma unroll
-      for (int k = 0; k < 5; ++k) red.cat[k] += __shfl_xor_sync(0xffffffffu, red.cat[k], o);
-      red.abs_adv += __shfl_xor_sync(0xffffffffu, red.abs_adv, o);
+    if (kp) {
+      rs.ck[j] = (unsigned long long)(tok - rs.len[j]);
+      rs.len[j] = __popc(kept_mask & ((1u << lane) - 1u));
     }
-    __shared__ TilePartial s_red[kThreads / 32];
-    if (lane == 0) s_red[warp] = red;
-    __syncthreads();
-    int wbase_cnt = 0;
-    long long wbase_tok = 0;
-    for (int k = 0; k < warp; ++k) { wbase_cnt += sh.warp_cnt[k]; wbase_tok += sh.warp_tok[k]; }
-    if (tid < npt) { ps.nk[tid] = wbase_cnt + cnt - my_cnt; ps.ktok[tid] = wbase_tok + tok - my_tok; }
-    if (tid == 0) {
-      TilePartial tot = {};
-      int tile_cnt = 0;
-      long long tile_tok = 0;
-      for (int k = 0; k < kThreads / 32; ++k) {
-        tile_cnt += sh.warp_cnt[k]; tile_tok += sh.warp_tok[k];
-        tot.present_tok += s_red[k].present_tok; tot.present_roll += s_red[k].present_roll; tot.surv += s_red[k].surv;
-        for (int c = 0; c < 5; ++c) tot.cat[c] += s_red[k].cat[c];
-        tot.abs_adv += s_red[k].abs_adv;
-      }
-      ws.part[tile] = tot;
-      sh.base_roll = tile_cnt;      // tile totals, replaced by the running totals below
-      sh.base_tok = tile_tok;
-    }
-    __syncthreads();
+    if (lane == 31) { rs.chunk_cnt[j0 >> 5] = __popc(kept_mask); rs.chunk_tok[j0 >> 5] = tok; }
   }
+  reduce_partial(sh, mine);
+  __syncthreads();
 
-  // ---- chained scan across tiles (warp 0) ----
+  // ---- warp 0: exclusive prefixes over the chunks, then the chained scan across tiles ----
   if (tid < 32) {
-    const int tile_cnt = sh.base_roll;
-    const long long tile_tok = sh.base_tok;
-    if (tid == 0 && tile > 0) {
-      st_release(ws.desc_roll + tile, kFlagAgg | (unsigned long long)tile_cnt);
-      st_release(ws.desc_tok + tile, kFlagAgg | (unsigned long long)tile_tok);
-    }
-    int excl_roll = 0;
-    long long excl_tok = 0;
-    const bool ok = scan_predecessors(ws, tile, tid, &excl_roll, &excl_tok);
-    if (tid == 0) {
-      if (ok) {
-        st_release(ws.desc_roll + tile, kFlagPrefix | (unsigned long long)(excl_roll + tile_cnt));
-        st_release(ws.desc_tok + tile, kFlagPrefix | (unsigned long long)(excl_tok + tile_tok));
-      } else {
-        atomicExch(ws.ctrl + 2, 1u);
-        st |= AERO_ST_TIMEOUT;
+    const int nchunks = (nroll + 31) >> 5;
+    int run_cnt = 0;
+    long long run_tok = 0;
+    for (int c0 = 0; c0 < nchunks; c0 += 32) {
+      const int c = c0 + lane;
+      int cnt = c < nchunks ? rs.chunk_cnt[c] : 0;
+      long long tok = c < nchunks ? rs.chunk_tok[c] : 0;
+      const int my_cnt = cnt;
+      const long long my_tok = tok;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int c2 = __shfl_up_sync(0xffffffffu, cnt, o);
+        const long long t2 = __shfl_up_sync(0xffffffffu, tok, o);
+        if (lane >= o) { cnt += c2; tok += t2; }
       }
-      sh.failed = ok ? 0 : 1;
-      sh.base_roll = excl_roll;
-      sh.base_tok = excl_tok;
+      if (c < nchunks) { rs.chunk_cnt[c] = run_cnt + cnt - my_cnt; rs.chunk_tok[c] = run_tok + tok - my_tok; }
+      run_cnt += __shfl_sync(0xffffffffu, cnt, 31);
+      run_tok += __shfl_sync(0xffffffffu, tok, 31);
     }
+    if (tid == 0) ws.part[tile] = sum_partials(sh);
+    chain_tile(ws, sh, tile, run_cnt, run_tok, st);
   }
   __syncthreads();
   const bool failed = sh.failed != 0;
   const int base_roll = sh.base_roll;
   const long long base_tok = sh.base_tok;
 
-  // ---- per prompt: positions of the kept rollouts inside the compacted outputs ----
-  if (tid < npt && !failed) {
-    const int q = tid;
-    const int lo = ps.lo[q], hi = ps.lo[q + 1];
-    int pos = ps.nk[q];
-    long long toff = ps.ktok[q];
-    for (int j = lo; j < hi; ++j) {
-      if (!acc.kept(j)) continue;
-      const long long len = acc.len(j);
-      if (STAGED) {
-        sh.rs.len[j] = pos;
-        sh.rs.ck[j] = (unsigned long long)toff;
-      } else {
-        a.kept_ids[base_roll + pos] = r0 + j;
-        a.kept_tok_off[base_roll + pos] = base_tok + toff;
-      }
-      pos += 1;
-      toff += len;
-    }
-  }
-  __syncthreads();
-
   // ---- per rollout: advantage, keep flag, compacted id and token offset ----
   for (int j = tid; j < nroll; j += kThreads) {
     const int i = r0 + j;
-    const int q = acc.pid(j, npt);
-    const bool kp = acc.kept(j);
-    a.adv[i] = kp ? (acc.r(j) - ps.mu[q]) * ps.inv[q] : 0.f;
-    if (STAGED) {
-      a.keep[i] = kp ? 1 : 0;
-      if (kp && !failed) {
-        const int pos = base_roll + sh.rs.len[j];
-        a.kept_ids[pos] = i;
-        a.kept_tok_off[pos] = base_tok + (long long)sh.rs.ck[j];
+    const int q = rs.pid[j];
+    const uint8_t f = rs.flag[j];
+    const bool kp = (f & 4) != 0;
+    a.adv[i] = kp ? (((f & 2) ? 1.f : 0.f) - ps.mu[q]) * ps.inv[q] : 0.f;
+    a.keep[i] = kp ? 1 : 0;
+    if (kp && !failed) {
+      const int pos = base_roll + rs.chunk_cnt[j >> 5] + rs.len[j];
+      a.kept_ids[pos] = i;
+      a.kept_tok_off[pos] = base_tok + rs.chunk_tok[j >> 5] + (long long)rs.ck[j];
+    }
+  }
+}
+
+// A tile whose rollouts exceed the staging area (a very large group): the same steps with
+// one thread per prompt walking the caller's arrays.
+__device__ void run_tile_global(const Args& a, const Workspace& ws, TileShared& sh, int tile, int p0, int npt, int r0,
+                                uint32_t& st) {
+  const int tid = threadIdx.x;
+  PromptState& ps = sh.ps;
+  auto present = [&](int j) { return a.keep_in ? a.keep_in[r0 + j] != 0 : true; };
+  auto length = [&](int j) { const long long l = a.cs[r0 + j + 1] - a.cs[r0 + j]; return l > 0 ? l : 0; };
+  auto order_key = [&](int j) {
+    if (!present(j)) return kNone;
+    const uint32_t key = a.key ? a.key[r0 + j] : default_key(a.cfg.seed, (uint32_t)(r0 + j));
+    return ((unsigned long long)key << 32) | (unsigned)j;
+  };
+  TilePartial mine = {};
+  if (tid < npt) {
+    const int p = p0 + tid;
+    const int lo = ps.lo[tid], hi = ps.lo[tid + 1];
+    int n = 0, c = 0;
+    for (int j = lo; j < hi; ++j) {
+      if (!present(j)) continue;
+      const float r = a.reward[r0 + j];
+      const long long len = a.cs[r0 + j + 1] - a.cs[r0 + j];
+      if (r != 0.f && r != 1.f) st |= AERO_ST_BAD_REWARD;
+      if (len < 0) st |= AERO_ST_BAD_OFFSETS;
+      if (len == 0) st |= AERO_ST_EMPTY_ROLLOUT;
+      n += 1; c += r > 0.5f ? 1 : 0;
+      mine.present_tok += len > 0 ? len : 0;
+    }
+    mine.present_roll = n;
+    const Rule ru = decide(a, p, n, c);
+    a.cat[p] = (uint8_t)ru.category;
+    a.u_tilde[p] = ru.ut;
+    a.alpha_out[p] = ru.al;
+    a.beta_out[p] = ru.be;
+    mine.cat[ru.category] = 1;
+
+    int nk = 0, ck = 0;
+    long long ktok = 0;
+    for (int j = lo; j < hi; ++j) {
+      const bool corr = a.reward[r0 + j] > 0.5f;
+      bool kp = present(j) && ru.mode != 1;
+      if (kp && ru.mode == 2 && !(ru.reject && corr)) {
+        const unsigned long long mykey = order_key(j);
+        long long rank = 0;
+        for (int k = lo; k < hi; ++k) {
+          if (ru.reject && a.reward[r0 + k] > 0.5f) continue;
+          rank += order_key(k) < mykey ? 1 : 0;
+        }
+        kp = rank < ru.quota;
       }
+      a.keep[r0 + j] = kp ? 1 : 0;
+      if (kp) { nk += 1; ck += corr ? 1 : 0; ktok += length(j); }
+    }
+    const bool over_kept = a.cfg.stats_over == AERO_STATS_KEPT;
+    const int nb = over_kept ? nk : n, cb = over_kept ? ck : c;
+    float mu = 0.f, sd = 0.f;
+    if (ru.uniform) {
+      mu = ru.ut;
+      sd = sqrtf(mu * (1.f - mu));
+    } else if (nb > 0) {
+      mu = (float)cb / (float)nb;
+      const float d1 = 1.f - mu;
+      sd = sqrtf(((float)cb * d1 * d1 + (float)(nb - cb) * mu * mu) / (float)nb);
+    }
+    const float inv = 1.f / (sd + a.cfg.eps_std);
+    for (int j = lo; j < hi; ++j)
+      a.adv[r0 + j] = a.keep[r0 + j] ? ((a.reward[r0 + j] > 0.5f ? 1.f : 0.f) - mu) * inv : 0.f;
+    ps.nk[tid] = nk;
+    ps.ktok[tid] = ktok;
+    a.gmask[p] = nk > 0 ? 1 : 0;
+    if (a.cfg.agg != AERO_TOKEN_MEAN) ws.nkept[p] = nk;
+    mine.surv = nk > 0 ? 1 : 0;
+    mine.abs_adv = ((float)ck * fabsf(1.f - mu) + (float)(nk - ck) * fabsf(mu)) * inv;
+  }
+
+  // tile totals and exclusive prefixes over the tile's prompts (block scan, fixed order)
+  const int lane = tid & 31, warp = tid >> 5;
+  int cnt = tid < npt ? ps.nk[tid] : 0;
+  long long tok = tid < npt ? ps.ktok[tid] : 0;
+  const int my_cnt = cnt;
+  const long long my_tok = tok;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int c2 = __shfl_up_sync(0xffffffffu, cnt, o);
+    const long long t2 = __shfl_up_sync(0xffffffffu, tok, o);
+    if (lane >= o) { cnt += c2; tok += t2; }
+  }
+  if (lane == 31) { sh.warp_cnt[warp] = cnt; sh.warp_tok[warp] = tok; }
+  reduce_partial(sh, mine);
+  __syncthreads();
+  int wbase_cnt = 0;
+  long long wbase_tok = 0;
+  for (int k = 0; k < warp; ++k) { wbase_cnt += sh.warp_cnt[k]; wbase_tok += sh.warp_tok[k]; }
+  const int excl_cnt = wbase_cnt + cnt - my_cnt;
+  const long long excl_tok = wbase_tok + tok - my_tok;
+  if (tid < 32) {
+    int tile_cnt = 0;
+    long long tile_tok = 0;
+    for (int k = 0; k < kThreads / 32; ++k) { tile_cnt += sh.warp_cnt[k]; tile_tok += sh.warp_tok[k]; }
+    if (tid == 0) ws.part[tile] = sum_partials(sh);
+    chain_tile(ws, sh, tile, tile_cnt, tile_tok, st);
+  }
+  __syncthreads();
+  if (tid < npt && !sh.failed) {
+    int pos = sh.base_roll + excl_cnt;
+    long long toff = sh.base_tok + excl_tok;
+    for (int j = ps.lo[tid]; j < ps.lo[tid + 1]; ++j) {
+      if (!a.keep[r0 + j]) continue;
+      a.kept_ids[pos] = r0 + j;
+      a.kept_tok_off[pos] = toff;
+      pos += 1;
+      toff += length(j);
     }
   }
 }
@@ -577,7 +646,7 @@ __device__ void finish_batch(const Args& a, const Workspace& ws, int ntiles) {
   }
 }
 
-__global__ void __launch_bounds__(kThreads) curate_kernel(Args a, Workspace ws, int pt, int ntiles) {
+__global__ void __launch_bounds__(kThreads, 4) curate_kernel(Args a, Workspace ws, int pt, int ntiles) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   TileShared& sh = *reinterpret_cast<TileShared*>(smem_raw);
   const int tid = threadIdx.x;
@@ -607,8 +676,8 @@ __global__ void __launch_bounds__(kThreads) curate_kernel(Args a, Workspace ws, 
     __syncthreads();
     for (int q = tid; q <= npt; q += kThreads) sh.ps.lo[q] -= r0;
     __syncthreads();
-    if (nroll <= kCap) run_tile<true>(a, ws, sh, tile, p0, npt, r0, nroll, st);
-    else run_tile<false>(a, ws, sh, tile, p0, npt, r0, nroll, st);
+    if (nroll <= kCap) run_tile_staged(a, ws, sh, tile, p0, npt, r0, nroll, st);
+    else run_tile_global(a, ws, sh, tile, p0, npt, r0, st);
   }
   st = __reduce_or_sync(0xffffffffu, st);
   if ((tid & 31) == 0) aero_raise(a.status, st);
