@@ -11,6 +11,9 @@ taken is stated in the docstring.
 
 Parity unpinned (no passage of the paper fixes the value; pinned only by
 brute force inside the tests):
+  * the per-token estimator of Eq. 2's KL term (the paper prints D_KL[pi || pi_ref]
+    and nothing more; here the non-negative estimator exp(q) - q - 1 with
+    q = ref_logp - logp, the one GRPO uses);
   * which individual incorrect rollouts the rejection step keeps (the paper
     says "top-m most informative" without defining it; here: smallest key);
   * the denominator of the Bayesian advantage for uniform groups (the paper
@@ -62,6 +65,8 @@ class Cfg:
     clip_lo: float = 0.2        # Table 9: clip ratio 0.2
     clip_hi: float = 0.2
     seed: int = 0
+    kl_beta: float = 0.0        # Eq. 2's beta (the paper never gives a value; Theorem 4.1 sets 0)
+    ent_coef: float = 0.0       # Table 9: entropy coefficient 1e-3
 
 
 # ----------------------------------------------------------------------------
@@ -323,6 +328,83 @@ def grpo_loss_bwd(H, W, y, cs, keep, lse, g, grad_scale=1.0, dw_rows=None):
         dz = -np.exp(z - np.asarray(lse, np.float64)[idx][:, None])
         dz[np.arange(len(idx)), np.asarray(y, np.int64)[idx]] += 1.0
         dz *= (grad_scale * np.asarray(g, np.float64)[idx])[:, None]
+        dH[idx] = dz @ W
+        dW = dz[:, rows].T @ H[idx]
+    return dH, dW
+
+
+# ----------------------------------------------------------------------------
+# stage (b) with the regularisers of Eq. 2 and Table 9: KL to a reference policy
+# and an entropy bonus
+# ----------------------------------------------------------------------------
+def entropy_rows(z):
+    """Entropy of softmax(z_t) per row, H_t = -sum_v p_tv log p_tv, from the definition."""
+    m = z.max(axis=1, keepdims=True)
+    e = np.exp(z - m)
+    p = e / e.sum(axis=1, keepdims=True)
+    logp = (z - m) - np.log(e.sum(axis=1, keepdims=True))
+    return -(p * logp).sum(axis=1)
+
+
+def kl_to_reference(logp, ref_logp):
+    """Per-token estimate of Eq. 2's D_KL[pi_theta || pi_ref] on the sampled token:
+    D = exp(q) - q - 1 with q = ref_logp - logp (non-negative, zero iff q = 0), and its
+    derivative dD/dlogp = 1 - exp(q).  The paper does not print the estimator: this is a
+    reading (parity unpinned)."""
+    q = np.asarray(ref_logp, np.float64) - np.asarray(logp, np.float64)
+    return np.exp(q) - q - 1.0, 1.0 - np.exp(q)
+
+
+def grpo_loss_reg_fwd(cfg: Cfg, H, W, y, old_logp, ref_logp, cs, adv, w, keep):
+    """Forward with the regularisers.  Per kept token of rollout i:
+        loss_t = w_i * ( -s_t + kl_beta * D_t - ent_coef * H_t )        (loss = -J, Eq. 2)
+        g_t    = dloss/dlogp_t = -w_i A_i rho_t I_t + kl_beta w_i (1 - exp(ref_t - logp_t))
+    The entropy acts on every logit, not only through logp_t, so it is returned per row
+    (`entropy`) for the backward.  ref_logp may be None when kl_beta == 0."""
+    base = grpo_loss_fwd(cfg, H, W, y, old_logp, cs, adv, w, keep)
+    H = np.asarray(H, np.float64)
+    T = H.shape[0]
+    owner = token_rollout(cs, T)
+    kept_t = np.asarray(keep)[owner] != 0
+    idx = np.nonzero(kept_t)[0]
+    w_t = np.asarray(w, np.float64)[owner]
+    ent = np.zeros(T)
+    kl = np.zeros(T)
+    g = base["g"].copy()
+    if len(idx):
+        ent[idx] = entropy_rows(logits(H[idx], W))
+        if cfg.kl_beta != 0.0:
+            D, dD = kl_to_reference(base["logp"][idx], np.asarray(ref_logp, np.float64)[idx])
+            kl[idx] = D
+            g[idx] += cfg.kl_beta * w_t[idx] * dD
+    loss = base["loss"] + float(np.sum(w_t * (cfg.kl_beta * kl - cfg.ent_coef * ent)))
+    out = dict(base)
+    out.update(g=g, loss=loss, entropy=ent, kl=kl)
+    return out
+
+
+def grpo_loss_reg_bwd(cfg: Cfg, H, W, y, cs, keep, lse, g, entropy, w, grad_scale=1.0, dw_rows=None):
+    """Backward with the entropy bonus: with p = softmax(z_t) and e_t = ent_coef * w_i,
+        dz_tv = grad_scale * ( g_t (1[v = y_t] - p_tv) + e_t p_tv (log p_tv + H_t) ),
+    the second term being d(-e_t H_t)/dz_tv; then dH = dz W and dW = dz^T H as before."""
+    H = np.asarray(H, np.float64)
+    W = np.asarray(W, np.float64)
+    T, d = H.shape
+    V = W.shape[0]
+    owner = token_rollout(cs, T)
+    idx = np.nonzero(np.asarray(keep)[owner] != 0)[0]
+    dH = np.zeros((T, d))
+    rows = np.arange(V) if dw_rows is None else np.asarray(dw_rows, np.int64)
+    dW = np.zeros((len(rows), d))
+    if len(idx):
+        z = logits(H[idx], W)
+        logp_all = z - np.asarray(lse, np.float64)[idx][:, None]
+        p = np.exp(logp_all)
+        dz = -p * np.asarray(g, np.float64)[idx][:, None]
+        dz[np.arange(len(idx)), np.asarray(y, np.int64)[idx]] += np.asarray(g, np.float64)[idx]
+        e_t = cfg.ent_coef * np.asarray(w, np.float64)[owner[idx]]
+        dz += e_t[:, None] * p * (logp_all + np.asarray(entropy, np.float64)[idx][:, None])
+        dz *= grad_scale
         dH[idx] = dz @ W
         dW = dz[:, rows].T @ H[idx]
     return dH, dW

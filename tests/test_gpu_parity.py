@@ -278,6 +278,23 @@ def test_full_width_qwen_1p5b_shape(ctx):
     assert TL.rel_l2(dW.cpu().numpy()[rows], rdW) < GRAD_L2
 
 
+def test_full_width_qwen_7b_shape(ctx):
+    """Full d = 3584 and V = 152064 of the Qwen2.5-7B shaped workloads, AERO mode with ragged groups
+    and per-prompt priors, on a batch the oracle can finish.  Every output against the oracle; dW on
+    the target rows plus 512 random rows."""
+    wl = synth.scaled(synth.WORKLOADS[3], P=3, n_lo=2, n_hi=6, len_median=48.0, len_cap=120, seed=33)
+    batch = TL.Batch(wl, TL.cfg_for(wl))
+    assert batch.T >= 256 and batch.ref_g["keep"].sum() < batch.R
+    ref = batch.oracle_fwd()
+    cfg, dv, f, dH, dW = run_fwd_bwd(ctx, batch, "bf16")
+    assert ctx.last_status() == 0
+    check_fwd(batch, f, ref, LOGP_ABS, LOSS_REL, 2e-2)
+    rows = np.unique(np.concatenate([batch.st.y[:64], np.random.default_rng(2).integers(0, wl.V, 512)]))
+    rdH, rdW = batch.oracle_bwd(ref, dw_rows=rows)
+    assert TL.rel_l2(dH.float().cpu().numpy(), rdH) < GRAD_L2
+    assert TL.rel_l2(dW.cpu().numpy()[rows], rdW) < GRAD_L2
+
+
 def test_step_from_host_buffers_matches_device_calls(ctx):
     over, cover, _ = BF16_CASES["aero_dropped"]
     wl = synth.scaled(synth.WORKLOADS[1], **over)
@@ -305,18 +322,20 @@ def test_step_from_host_buffers_matches_device_calls(ctx):
     assert ctx.last_status() == 0
 
 
-def test_full_size_qwen_1p5b_in_bench_configuration(ctx):
-    """The whole Qwen2.5-Math-1.5B shaped workload (~283k tokens) in the launch configuration
-    bench.py times.  The oracle cannot produce all of it, so: the group stage is compared in
-    full; 96 sampled token rows are compared one by one (log-prob, lse, g, dH row); the loss and
-    sampled rows of dW are checked through identities that hold at any size."""
-    wl = synth.WORKLOADS[1]
+@pytest.mark.parametrize("config", [1, 2, 3, 4])
+def test_full_size_workload_in_bench_configuration(ctx, config):
+    """A whole benchmark workload (1: Qwen2.5-Math-1.5B shape, ~283k tokens; 2: Qwen2.5-7B shape,
+    ~850k; 3: the AERO-curated ragged batch; 4: the ~4.5M-token stress batch) in the launch
+    configuration bench.py times.  The oracle cannot produce all of it, so: the group stage is
+    compared in full; 96 sampled token rows are compared one by one (log-prob, lse, g, dH row);
+    the loss and sampled rows of dW are checked through identities that hold at any size."""
+    wl = synth.WORKLOADS[config]
     st = synth.make_structure(wl)
     P, R, T = len(st.go) - 1, len(st.reward), int(st.cs[-1])
     ocfg = TL.cfg_for(wl)
     cfg = TL.lib_cfg(ocfg, "bf16")
     H, W = synth.make_tensors(wl, T, device="cuda")
-    ref_g = O.group_stats(ocfg, st.go, st.reward, st.cs, key=st.key)
+    ref_g = O.group_stats(ocfg, st.go, st.reward, st.cs, key=st.key, alpha_in=st.alpha, beta_in=st.beta)
     gi, g = TL.run_group_gpu(ctx, cfg, st)
     TL.check_group(g, ref_g, R, P)
 
@@ -371,7 +390,7 @@ def test_full_size_qwen_1p5b_in_bench_configuration(ctx):
     kept = ref_g["keep"][owner] != 0
     A_t, w_t = adv32[owner], w32[owner]
     rho = np.exp(logp.astype(np.float64) - old.astype(np.float64))
-    surr = np.minimum(rho * A_t, np.clip(rho, 0.8, 1.2) * A_t)
+    surr = np.minimum(rho * A_t, np.clip(rho, 1 - ocfg.clip_lo, 1 + ocfg.clip_hi) * A_t)
     loss_re = -float(np.sum((w_t * surr)[kept]))
     assert abs(f["loss"].item() - loss_re) <= 1e-4 * abs(loss_re) + 1e-8
     assert (logp[kept] <= 1e-6).all() and not logp[~kept].any()
@@ -381,14 +400,17 @@ def test_full_size_qwen_1p5b_in_bench_configuration(ctx):
     # rows of dW from the definition, with the library's own lse and g (fp64 on the device)
     vrows = np.unique(np.concatenate([st.y[kept_rows[:8]], rng.integers(0, wl.V, 24)]))
     vr = torch.from_numpy(vrows).cuda()
-    H64 = H.double()
-    z = H64 @ W[vr].double().T
-    dz = -torch.exp(z - f["lse"][:T].double()[:, None])
-    dz += (y[:, None] == vr[None, :].to(y.dtype)).double()
-    dz *= f["g"][:T].double()[:, None]
-    ref_rows = (dz.T @ H64).cpu().numpy()
-    assert TL.rel_l2(dW[vr].cpu().numpy(), ref_rows) < GRAD_L2
-    del H64, z, dz
+    Wv = W[vr].double()
+    ref_rows = torch.zeros((len(vrows), wl.d), dtype=torch.float64, device="cuda")
+    for a in range(0, T, 1 << 18):                       # row blocks bound the fp64 copies of H
+        b = min(T, a + (1 << 18))
+        H64 = H[a:b].double()
+        dz = -torch.exp(H64 @ Wv.T - f["lse"][a:b].double()[:, None])
+        dz += (y[a:b, None] == vr[None, :].to(y.dtype)).double()
+        dz *= f["g"][a:b].double()[:, None]
+        ref_rows += dz.T @ H64
+        del H64, dz
+    assert TL.rel_l2(dW[vr].cpu().numpy(), ref_rows.cpu().numpy()) < GRAD_L2
     # a different chunking gives the same dH bits and the same dW up to fp32 summation order
     ws2 = torch.empty(ctx.bwd_workspace_bytes(T, wl.d, wl.V, R, 148 * 128), dtype=torch.uint8, device="cuda")
     dH2, dW2 = ctx.grpo_loss_bwd(cfg, H, W, y, cs, g["keep"], f["lse"], f["g"], workspace=ws2)

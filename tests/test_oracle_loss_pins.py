@@ -211,3 +211,83 @@ def test_loss_matches_scalar_loop_statement_of_eq2():
             J += acc / (cs[i + 1] - cs[i]) / 4
     J /= len(surviving)
     assert f["loss"] == pytest.approx(-J, rel=1e-12)
+
+
+# ---------------------------------------------------------------- regularisers (KL, entropy)
+def test_entropy_closed_forms_and_library_routine():
+    import scipy.stats
+    V = 17
+    assert np.allclose(O.entropy_rows(np.zeros((3, V))), math.log(V))           # uniform: log V
+    z = np.full((1, V), -800.0)
+    z[0, 5] = 0.0
+    assert O.entropy_rows(z)[0] == pytest.approx(0.0, abs=1e-300)               # one-hot: 0
+    rng = np.random.default_rng(3)
+    z = rng.standard_normal((6, V)) * 3
+    p = np.exp(z - z.max(axis=1, keepdims=True))
+    p /= p.sum(axis=1, keepdims=True)
+    assert np.allclose(O.entropy_rows(z), scipy.stats.entropy(p, axis=1), rtol=1e-12)
+    assert np.allclose(O.entropy_rows(z + 1000.0), O.entropy_rows(z), rtol=1e-9)  # shift invariance
+
+
+def test_kl_estimator_properties():
+    rng = np.random.default_rng(4)
+    logp = -np.abs(rng.standard_normal(50)) - 0.1
+    D, dD = O.kl_to_reference(logp, logp)
+    assert not D.any() and not dD.any()                                        # same policy: zero, flat
+    ref = logp + rng.standard_normal(50)
+    D, dD = O.kl_to_reference(logp, ref)
+    assert (D > 0).all()
+    h = 1e-6
+    Dp, _ = O.kl_to_reference(logp + h, ref)
+    Dm, _ = O.kl_to_reference(logp - h, ref)
+    assert np.allclose((Dp - Dm) / (2 * h), dD, rtol=1e-6, atol=1e-8)
+    # in expectation under pi_theta the estimator is the KL divergence: exact sum over a small vocabulary
+    z, zr = rng.standard_normal(9), rng.standard_normal(9)
+    lp, lr = z - np.log(np.exp(z).sum()), zr - np.log(np.exp(zr).sum())
+    D_all, _ = O.kl_to_reference(lp, lr)
+    assert np.sum(np.exp(lp) * D_all) == pytest.approx(np.sum(np.exp(lp) * (lp - lr)), rel=1e-12)
+
+
+@pytest.mark.parametrize("kl_beta,ent_coef", [(0.0, 0.0), (0.04, 0.0), (0.0, 1e-3), (0.3, 0.2)])
+def test_regularised_backward_equals_autograd_of_library_statement(kl_beta, ent_coef):
+    go, cs, reward, H, W, y, rng = _batch(7, d=12, V=23)
+    cfg = O.Cfg(eps_std=0.0, kl_beta=kl_beta, ent_coef=ent_coef)
+    gs, old = _with_old(cfg, go, cs, reward, H, W, y, rng, 0.3)
+    ref_lp = old + 0.2 * rng.standard_normal(len(old))
+    f = O.grpo_loss_reg_fwd(cfg, H, W, y, old, ref_lp, cs, gs["adv"], gs["w"], gs["keep"])
+    dH, dW = O.grpo_loss_reg_bwd(cfg, H, W, y, cs, gs["keep"], f["lse"], f["g"], f["entropy"], gs["w"])
+    if kl_beta == 0.0 and ent_coef == 0.0:            # reduces to the unregularised functions
+        f0 = O.grpo_loss_fwd(cfg, H, W, y, old, cs, gs["adv"], gs["w"], gs["keep"])
+        dH0, dW0 = O.grpo_loss_bwd(H, W, y, cs, gs["keep"], f0["lse"], f0["g"])
+        assert f["loss"] == f0["loss"]
+        assert np.allclose(dH, dH0, rtol=1e-12, atol=1e-15) and np.allclose(dW, dW0, rtol=1e-12, atol=1e-15)
+    # independent statement in torch: log_softmax, Categorical entropy, autograd
+    Ht = torch.tensor(H, requires_grad=True)
+    Wt = torch.tensor(W, requires_grad=True)
+    owner = torch.tensor(O.token_rollout(cs, H.shape[0]))
+    keep_t = torch.tensor(gs["keep"].astype(bool))[owner]
+    A = torch.tensor(gs["adv"])[owner]
+    w = torch.tensor(gs["w"])[owner]
+    lsm = torch.log_softmax(Ht @ Wt.T, dim=1)
+    lp = lsm[torch.arange(H.shape[0]), torch.tensor(y).long()]
+    rho = torch.exp(lp - torch.tensor(old))
+    surr = torch.minimum(rho * A, torch.clamp(rho, 0.8, 1.2) * A)
+    q = torch.tensor(ref_lp) - lp
+    ent = torch.distributions.Categorical(logits=lsm).entropy()
+    per_tok = -surr + kl_beta * (torch.exp(q) - q - 1) - ent_coef * ent
+    loss = (w * per_tok)[keep_t].sum()
+    loss.backward()
+    assert f["loss"] == pytest.approx(loss.item(), rel=1e-11, abs=1e-14)
+    assert np.allclose(dH, Ht.grad.numpy(), rtol=1e-9, atol=1e-13)
+    assert np.allclose(dW, Wt.grad.numpy(), rtol=1e-9, atol=1e-13)
+
+
+def test_regularised_gradient_invariants():
+    go, cs, reward, H, W, y, rng = _batch(8, d=10, V=19)
+    cfg = O.Cfg(eps_std=0.0, kl_beta=0.1, ent_coef=0.05)
+    gs, old = _with_old(cfg, go, cs, reward, H, W, y, rng, 0.2)
+    f = O.grpo_loss_reg_fwd(cfg, H, W, y, old, old, cs, gs["adv"], gs["w"], gs["keep"])
+    _, dW = O.grpo_loss_reg_bwd(cfg, H, W, y, cs, gs["keep"], f["lse"], f["g"], f["entropy"], gs["w"])
+    # each row of dz still sums to zero (sum_v p (log p + H) = 0), so the columns of dW do too
+    assert np.abs(dW.sum(axis=0)).max() < 1e-12
+    assert (f["entropy"] >= 0).all() and (f["kl"] >= 0).all()
