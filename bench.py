@@ -27,6 +27,11 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "rollout tokens/sec, fused GRPO logprob+loss fwd+bwd"
+# dram__bytes_read.sum + dram__bytes_write.sum of one lmhead_kernel<MODE_FWD> launch, from the ncu capture
+# summarised in profiles/lmhead_fwd_qwen1p5b_8prompts.md (a reduced batch of the same workload); the kernel's DRAM
+# traffic grows in proportion to the token rows it processes, so it is scaled by kept tokens.
+NCU_FWD_TRAFFIC = {"config": 1, "bytes": 1.117685e9, "tokens": 36784,
+                   "source": "ncu capture of a 36784-token batch (288 token tiles), scaled by kept tokens"}
 UNIT = "tokens/s"
 
 
@@ -275,10 +280,12 @@ def run_ours(args):
     fwd_ms = float(np.mean(fw))
     clocks = sampler.stop()
     flops_launch = 2.0 * T_kept * wl.d * wl.V
+    traffic = NCU_FWD_TRAFFIC["bytes"] * T_kept / NCU_FWD_TRAFFIC["tokens"] if args.config == NCU_FWD_TRAFFIC["config"] else None
     achieved = flops_launch / (fwd_ms * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "lmhead_kernel<MODE_FWD>", "achieved": achieved, "peak": pk["burst"],
                 "unit": "TFLOP/s", "frac": achieved / pk["burst"], "peak_source": pk["src"] + " burst bf16",
-                "traffic": None, "ms_per_launch": fwd_ms,
+                "traffic": traffic, "traffic_source": NCU_FWD_TRAFFIC["source"] if traffic else None,
+                "ms_per_launch": fwd_ms,
                 "step_executed_tflops": 8.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12,
                 "step_frac_of_sustained": 8.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12 / pk["sustained"]}
 

@@ -108,6 +108,10 @@ typedef struct aero_cfg {
   uint64_t seed;            /* seeds the default selection keys                  default 0   */
   int32_t dtype;            /* AERO_BF16 | AERO_FP32: type of H, W and dH        default BF16 */
   int32_t reserved;
+  float   kl_beta;          /* Eq. 2's beta (KL to a reference policy); read only by   default 0 */
+                            /* the *_reg_* calls                                                 */
+  float   ent_coef;         /* entropy bonus coefficient (Table 9: 1e-3); read only    default 0 */
+                            /* by the *_reg_* calls                                              */
 } aero_cfg;
 
 typedef struct aero_ctx aero_ctx;   /* opaque: device id, borrowed stream, status word */
@@ -276,6 +280,47 @@ int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d,
                        const float* lse, const float* g, float grad_scale,
                        void* dH, float* dW, int accumulate_dW,
                        void* workspace, size_t workspace_bytes);
+
+/* ------------------------------------------------------------------------------
+ * Stage (b) with the regularisers of Eq. 2 and Table 9.
+ *
+ * Per kept token of rollout i, with D_t = exp(q_t) - q_t - 1, q_t = ref_logp_t - logp_t
+ * (a non-negative per-token estimate of Eq. 2's D_KL[pi_theta || pi_ref]; the paper does
+ * not print the estimator, this is the one GRPO uses) and H_t = -sum_v p_tv log p_tv the
+ * entropy of the token's distribution (Table 9 "entropy coefficient"):
+ *   loss  = sum_t w_i ( -s_t + kl_beta D_t - ent_coef H_t )
+ *   g_t   = -w_i A_i rho_t [unclipped] + kl_beta w_i (1 - exp(q_t))
+ *   dz_tv = grad_scale ( g_t (1[v == y_t] - p_tv) + ent_coef w_i p_tv (log p_tv + H_t) )
+ * The entropy is carried through the same online pass as the log-sum-exp
+ * (H_t = lse_t - sum_v p_tv z_tv); nothing of size [T,V] is stored.
+ *
+ * aero_grpo_loss_reg_fwd: arguments of aero_grpo_loss_fwd plus ref_logp [T] f32 (NULL:
+ *   no KL term, kl_beta ignored) and entropy [T] f32 out (NULL: no entropy term,
+ *   ent_coef ignored).  With both NULL it is aero_grpo_loss_fwd.
+ * aero_grpo_loss_reg_bwd: arguments of aero_grpo_loss_bwd plus entropy [T] from the
+ *   forward and w [R] (both NULL: no entropy term).
+ * aero_logprob_fwd: the log-prob pass alone over all T rows (what produces old_logp and
+ *   ref_logp, Appendix C "Rollout"/"GRPO Training"): logp, lse [T] f32 and, if not NULL,
+ *   entropy [T] f32.  Workspace: aero_fwd_workspace_bytes(T, d, V, 0).
+ */
+int aero_grpo_loss_reg_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                           const void* H, const void* W, const int32_t* y, const float* old_logp,
+                           const float* ref_logp,
+                           const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                           float* logp, float* lse, float* g, float* entropy, float* loss, float* metrics,
+                           int accumulate, void* workspace, size_t workspace_bytes);
+
+int aero_grpo_loss_reg_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                           const void* H, const void* W, const int32_t* y,
+                           const int64_t* cs, const uint8_t* keep,
+                           const float* lse, const float* g, const float* entropy, const float* w,
+                           float grad_scale, void* dH, float* dW, int accumulate_dW,
+                           void* workspace, size_t workspace_bytes);
+
+int aero_logprob_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V,
+                     const void* H, const void* W, const int32_t* y,
+                     float* logp, float* lse, float* entropy,
+                     void* workspace, size_t workspace_bytes);
 
 /* ------------------------------------------------------------------------------
  * One whole step of the path from HOST buffers: stage (a), forward and backward

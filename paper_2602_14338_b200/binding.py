@@ -27,6 +27,7 @@ EXPORTS = [
     "aero_set_stream", "aero_last_status", "aero_group_workspace_bytes", "aero_group_stats",
     "aero_fwd_workspace_bytes", "aero_grpo_loss_fwd", "aero_bwd_workspace_bytes", "aero_grpo_loss_bwd",
     "aero_step_workspace_bytes", "aero_grpo_step_host", "aero_launch_count", "aero_group_stats_static",
+    "aero_grpo_loss_reg_fwd", "aero_grpo_loss_reg_bwd", "aero_logprob_fwd",
 ]
 
 
@@ -38,6 +39,7 @@ class AeroCfg(C.Structure):
         ("alpha0", C.c_float), ("beta0", C.c_float), ("eps_std", C.c_float),
         ("clip_lo", C.c_float), ("clip_hi", C.c_float),
         ("seed", C.c_uint64), ("dtype", C.c_int32), ("reserved", C.c_int32),
+        ("kl_beta", C.c_float), ("ent_coef", C.c_float),
     ]
 
 
@@ -77,6 +79,11 @@ def load_library():
     lib.aero_bwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i64]
     lib.aero_grpo_loss_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 7 + [f32] +
                                        [vp, vp, C.c_int, vp, sz])
+    lib.aero_grpo_loss_reg_fwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 15 +
+                                           [C.c_int, vp, sz])
+    lib.aero_grpo_loss_reg_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 9 + [f32] +
+                                           [vp, vp, C.c_int, vp, sz])
+    lib.aero_logprob_fwd.argtypes = [vp, C.POINTER(AeroCfg), i64, i32, i32] + [vp] * 6 + [vp, sz]
     lib.aero_step_workspace_bytes.restype = sz
     lib.aero_step_workspace_bytes.argtypes = [i32, i32, i64, i32, i32, i64, i32]
     lib.aero_grpo_step_host.argtypes = ([vp, C.POINTER(AeroCfg), i32, i32, i64, i32, i32] + [vp] * 12 + [C.c_int] +
@@ -250,6 +257,78 @@ class Context:
             _ptr(o["metrics"]), 1 if accumulate else 0, ws.data_ptr(), ws.numel())
         _check(rc, "aero_grpo_loss_fwd")
         return o
+
+    def grpo_loss_reg_fwd(self, cfg, H, W, y, old_logp, ref_logp, cs, adv, w, keep, out=None, accumulate=False,
+                          entropy=True):
+        """aero_grpo_loss_reg_fwd: the forward with Eq. 2's KL term (ref_logp not None) and the entropy
+        bonus (entropy=True adds the per-row entropy output 'entropy')."""
+        T, d = H.shape
+        V = W.shape[0]
+        R = cs.numel() - 1
+        dt = torch.bfloat16 if cfg.dtype == AERO_BF16 else torch.float32
+        o = out if out is not None else {}
+        names = ("logp", "lse", "g", "entropy") if entropy else ("logp", "lse", "g")
+        for name in names:
+            if name not in o:
+                o[name] = torch.empty(max(T, 1), dtype=torch.float32, device=self.device)
+        if "loss" not in o:
+            o["loss"] = torch.zeros(1, dtype=torch.float32, device=self.device)
+        if "metrics" not in o:
+            o["metrics"] = torch.zeros(4, dtype=torch.float32, device=self.device)
+        ws = self.workspace(self.fwd_workspace_bytes(T, d, V, R))
+        rc = self.lib.aero_grpo_loss_reg_fwd(
+            self.h, C.byref(cfg), T, d, V, R, _ptr(H, dt, T * d, "H"), _ptr(W, dt, V * d, "W"),
+            _ptr(y, torch.int32, T, "y"), _ptr(old_logp, torch.float32, T, "old_logp"),
+            _ptr(ref_logp, torch.float32, T, "ref_logp"),
+            _ptr(cs, torch.int64, R + 1, "cs"), _ptr(adv, torch.float32, R, "adv"), _ptr(w, torch.float32, R, "w"),
+            _ptr(keep, torch.uint8, R, "keep"), _ptr(o["logp"]), _ptr(o["lse"]), _ptr(o["g"]),
+            _ptr(o["entropy"]) if entropy else None, _ptr(o["loss"]),
+            _ptr(o["metrics"]), 1 if accumulate else 0, ws.data_ptr(), ws.numel())
+        _check(rc, "aero_grpo_loss_reg_fwd")
+        return o
+
+    def logprob_fwd(self, cfg, H, W, y, entropy=False, out=None):
+        """aero_logprob_fwd: log-probs (and optionally entropies) of the target tokens of all T rows."""
+        T, d = H.shape
+        V = W.shape[0]
+        dt = torch.bfloat16 if cfg.dtype == AERO_BF16 else torch.float32
+        o = out if out is not None else {}
+        names = ("logp", "lse", "entropy") if entropy else ("logp", "lse")
+        for name in names:
+            if name not in o:
+                o[name] = torch.empty(max(T, 1), dtype=torch.float32, device=self.device)
+        ws = self.workspace(self.fwd_workspace_bytes(T, d, V, 0))
+        rc = self.lib.aero_logprob_fwd(
+            self.h, C.byref(cfg), T, d, V, _ptr(H, dt, T * d, "H"), _ptr(W, dt, V * d, "W"),
+            _ptr(y, torch.int32, T, "y"), _ptr(o["logp"]), _ptr(o["lse"]),
+            _ptr(o["entropy"]) if entropy else None, ws.data_ptr(), ws.numel())
+        _check(rc, "aero_logprob_fwd")
+        return o
+
+    def grpo_loss_reg_bwd(self, cfg, H, W, y, cs, keep, lse, g, entropy, w, grad_scale=1.0, dH=None, dW=None,
+                          accumulate_dW=False, chunk_tokens=None, workspace=None):
+        """aero_grpo_loss_reg_bwd: the backward with the entropy term (entropy and w from the forward / group stage)."""
+        T, d = H.shape
+        V = W.shape[0]
+        R = cs.numel() - 1
+        dt = torch.bfloat16 if cfg.dtype == AERO_BF16 else torch.float32
+        if dH is None:
+            dH = torch.empty((max(T, 1), d), dtype=dt, device=self.device)[:T]
+        if dW is None:
+            dW = torch.empty((V, d), dtype=torch.float32, device=self.device)
+        if workspace is None:
+            if chunk_tokens is None:
+                chunk_tokens = min(max(128, (T + 127) // 128 * 128), 2 * 148 * 128)
+            workspace = self.workspace(self.bwd_workspace_bytes(T, d, V, R, chunk_tokens))
+        rc = self.lib.aero_grpo_loss_reg_bwd(
+            self.h, C.byref(cfg), T, d, V, R, _ptr(H, dt, T * d, "H"), _ptr(W, dt, V * d, "W"),
+            _ptr(y, torch.int32, T, "y"), _ptr(cs, torch.int64, R + 1, "cs"), _ptr(keep, torch.uint8, R, "keep"),
+            _ptr(lse, torch.float32, T, "lse"), _ptr(g, torch.float32, T, "g"),
+            _ptr(entropy, torch.float32, T, "entropy"), _ptr(w, torch.float32, R, "w"), C.c_float(grad_scale),
+            _ptr(dH, dt, T * d, "dH"), _ptr(dW, torch.float32, V * d, "dW"), 1 if accumulate_dW else 0,
+            workspace.data_ptr(), workspace.numel())
+        _check(rc, "aero_grpo_loss_reg_bwd")
+        return dH, dW
 
     def grpo_loss_bwd(self, cfg, H, W, y, cs, keep, lse, g, grad_scale=1.0, dH=None, dW=None,
                       accumulate_dW=False, chunk_tokens=None, workspace=None):

@@ -52,6 +52,8 @@ void aero_cfg_default(aero_cfg* cfg) {
   cfg->seed = 0;
   cfg->dtype = AERO_BF16;
   cfg->reserved = 0;
+  cfg->kl_beta = 0.f;
+  cfg->ent_coef = 0.f;
 }
 
 int aero_create(aero_ctx** out, int device, void* cuda_stream) {
@@ -133,40 +135,75 @@ size_t aero_fwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R) {
   return a > b ? a : b;
 }
 
-int aero_grpo_loss_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
-                       const void* H, const void* W, const int32_t* y, const float* old_logp,
-                       const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
-                       float* logp, float* lse, float* g, float* loss, float* metrics,
-                       int accumulate, void* workspace, size_t workspace_bytes) {
+static int fwd_dispatch(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                        const void* H, const void* W, const int32_t* y, const float* old_logp,
+                        const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                        float* logp, float* lse, float* g, float* loss, float* metrics,
+                        int accumulate, void* workspace, size_t workspace_bytes, const aero_fwd_extra& ex) {
   int rc = check_ctx(ctx);
   if (rc) return rc;
   if (!cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
-  if (!W || !cs || !loss) return AERO_ERR_INVALID;
-  if (T > 0 && (!H || !y || !old_logp || !logp || !lse || !g)) return AERO_ERR_INVALID;
-  if (R > 0 && (!adv || !w || !keep)) return AERO_ERR_INVALID;
+  if (!W) return AERO_ERR_INVALID;
+  if (T > 0 && (!H || !y || !logp || !lse)) return AERO_ERR_INVALID;
+  if (!ex.logprob_only) {
+    if (!cs || !loss) return AERO_ERR_INVALID;
+    if (T > 0 && (!old_logp || !g)) return AERO_ERR_INVALID;
+    if (R > 0 && (!adv || !w || !keep)) return AERO_ERR_INVALID;
+  }
   if (!workspace || !aligned256(workspace)) return AERO_ERR_INVALID;
   if (workspace_bytes < aero_fwd_workspace_bytes(T, d, V, R)) return AERO_ERR_WORKSPACE;
   if (cfg->dtype == AERO_FP32) {
     return aero_fwd_fp32(ctx, cfg, T, d, V, R, static_cast<const float*>(H), static_cast<const float*>(W),
-                         y, old_logp, cs, adv, w, keep, logp, lse, g, loss, metrics, accumulate, workspace);
+                         y, old_logp, cs, adv, w, keep, logp, lse, g, loss, metrics, accumulate, workspace, ex);
   }
   if (cfg->dtype != AERO_BF16) return AERO_ERR_UNSUPPORTED;
   if (d % 64 != 0) return AERO_ERR_UNSUPPORTED;
   if (!aligned16(H) || !aligned16(W)) return AERO_ERR_INVALID;
   return aero_fwd_tc(ctx, cfg, T, d, V, R, H, W, y, old_logp, cs, adv, w, keep, logp, lse, g, loss,
-                     metrics, accumulate, workspace);
+                     metrics, accumulate, workspace, ex);
+}
+
+int aero_grpo_loss_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                       const void* H, const void* W, const int32_t* y, const float* old_logp,
+                       const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                       float* logp, float* lse, float* g, float* loss, float* metrics,
+                       int accumulate, void* workspace, size_t workspace_bytes) {
+  const aero_fwd_extra ex = {nullptr, 0.f, 0.f, nullptr, 0};
+  return fwd_dispatch(ctx, cfg, T, d, V, R, H, W, y, old_logp, cs, adv, w, keep, logp, lse, g, loss, metrics,
+                      accumulate, workspace, workspace_bytes, ex);
+}
+
+int aero_grpo_loss_reg_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                           const void* H, const void* W, const int32_t* y, const float* old_logp,
+                           const float* ref_logp,
+                           const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                           float* logp, float* lse, float* g, float* entropy, float* loss, float* metrics,
+                           int accumulate, void* workspace, size_t workspace_bytes) {
+  if (!cfg) return AERO_ERR_INVALID;
+  const aero_fwd_extra ex = {ref_logp, ref_logp ? cfg->kl_beta : 0.f, entropy ? cfg->ent_coef : 0.f, entropy, 0};
+  return fwd_dispatch(ctx, cfg, T, d, V, R, H, W, y, old_logp, cs, adv, w, keep, logp, lse, g, loss, metrics,
+                      accumulate, workspace, workspace_bytes, ex);
+}
+
+int aero_logprob_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V,
+                     const void* H, const void* W, const int32_t* y,
+                     float* logp, float* lse, float* entropy,
+                     void* workspace, size_t workspace_bytes) {
+  const aero_fwd_extra ex = {nullptr, 0.f, 0.f, entropy, 1};
+  return fwd_dispatch(ctx, cfg, T, d, V, 0, H, W, y, nullptr, nullptr, nullptr, nullptr, nullptr, logp, lse, nullptr,
+                      nullptr, nullptr, 0, workspace, workspace_bytes, ex);
 }
 
 size_t aero_bwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R, int64_t chunk_tokens) {
   return aero_bwd_ws_bytes_tc(T, d, V, R, chunk_tokens);
 }
 
-int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
-                       const void* H, const void* W, const int32_t* y,
-                       const int64_t* cs, const uint8_t* keep,
-                       const float* lse, const float* g, float grad_scale,
-                       void* dH, float* dW, int accumulate_dW,
-                       void* workspace, size_t workspace_bytes) {
+static int bwd_dispatch(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                        const void* H, const void* W, const int32_t* y,
+                        const int64_t* cs, const uint8_t* keep,
+                        const float* lse, const float* g, float grad_scale,
+                        void* dH, float* dW, int accumulate_dW,
+                        void* workspace, size_t workspace_bytes, const aero_bwd_extra& ex) {
   int rc = check_ctx(ctx);
   if (rc) return rc;
   if (!cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
@@ -175,7 +212,7 @@ int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d,
   if (R > 0 && !keep) return AERO_ERR_INVALID;
   if (cfg->dtype == AERO_FP32) {
     return aero_bwd_fp32(ctx, cfg, T, d, V, R, static_cast<const float*>(H), static_cast<const float*>(W),
-                         y, cs, keep, lse, g, grad_scale, static_cast<float*>(dH), dW, accumulate_dW);
+                         y, cs, keep, lse, g, grad_scale, static_cast<float*>(dH), dW, accumulate_dW, ex);
   }
   if (cfg->dtype != AERO_BF16) return AERO_ERR_UNSUPPORTED;
   if (d % 64 != 0) return AERO_ERR_UNSUPPORTED;
@@ -183,7 +220,31 @@ int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d,
   if (!workspace || !aligned256(workspace)) return AERO_ERR_INVALID;
   if (workspace_bytes < aero_bwd_ws_bytes_tc(T, d, V, R, 128)) return AERO_ERR_WORKSPACE;
   return aero_bwd_tc(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, grad_scale, dH, dW, accumulate_dW,
-                     workspace, workspace_bytes);
+                     workspace, workspace_bytes, ex);
+}
+
+int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                       const void* H, const void* W, const int32_t* y,
+                       const int64_t* cs, const uint8_t* keep,
+                       const float* lse, const float* g, float grad_scale,
+                       void* dH, float* dW, int accumulate_dW,
+                       void* workspace, size_t workspace_bytes) {
+  const aero_bwd_extra ex = {nullptr, nullptr, 0.f};
+  return bwd_dispatch(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, grad_scale, dH, dW, accumulate_dW, workspace,
+                      workspace_bytes, ex);
+}
+
+int aero_grpo_loss_reg_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                           const void* H, const void* W, const int32_t* y,
+                           const int64_t* cs, const uint8_t* keep,
+                           const float* lse, const float* g, const float* entropy, const float* w,
+                           float grad_scale, void* dH, float* dW, int accumulate_dW,
+                           void* workspace, size_t workspace_bytes) {
+  if (!cfg) return AERO_ERR_INVALID;
+  if ((entropy == nullptr) != (w == nullptr)) return AERO_ERR_INVALID;
+  const aero_bwd_extra ex = {entropy, w, entropy ? cfg->ent_coef : 0.f};
+  return bwd_dispatch(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, grad_scale, dH, dW, accumulate_dW, workspace,
+                      workspace_bytes, ex);
 }
 
 }  // extern "C"

@@ -41,6 +41,21 @@ int aero_group_stats_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32
                             int32_t* kept_ids, int64_t* kept_tok_off, int64_t* counters,
                             float* metrics, void* ws);
 
+// Optional terms of the objective beyond the clipped surrogate: Eq. 2's KL to a reference
+// policy and the entropy bonus of Table 9.  All-zero / NULL means the plain objective.
+struct aero_fwd_extra {
+  const float* ref_logp;   // [T] or NULL (no KL term)
+  float kl_beta;
+  float ent_coef;          // used only when `entropy` is given
+  float* entropy;          // [T] out, or NULL (no entropy term)
+  int logprob_only;        // all T rows, log-probs (and entropy) only: cs/adv/w/keep/old_logp unused
+};
+struct aero_bwd_extra {
+  const float* entropy;    // [T] from the forward, or NULL
+  const float* w;          // [R] rollout weights (entropy term only)
+  float ent_coef;
+};
+
 // ---- stage (b): helpers shared by the fp32 and the tensor-core paths ---------------
 // Row-tile work list over maximal runs of consecutive kept rollouts.
 struct aero_tiles {
@@ -53,6 +68,8 @@ aero_tiles aero_carve_tiles(void* ws, int64_t T, int32_t R, int tile_rows);
 size_t aero_tiles_bytes(int64_t T, int32_t R, int tile_rows);
 int aero_build_tiles(aero_ctx* ctx, int64_t T, int32_t R, const int64_t* cs, const uint8_t* keep,
                      int tile_rows, aero_tiles tiles);
+// The same list over all T rows (one run): tile k starts at row k * tile_rows.
+int aero_build_dense_tiles(aero_ctx* ctx, int64_t T, int tile_rows, aero_tiles tiles);
 
 // Per-token surrogate terms and the fixed-order loss reduction.
 int aero_loss_finalize(aero_ctx* ctx, const double* partials, int n_partials, int stride,
@@ -63,19 +80,22 @@ size_t aero_fwd_ws_bytes_fp32(int64_t T, int32_t R);
 int aero_fwd_fp32(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                   const float* H, const float* W, const int32_t* y, const float* old_logp,
                   const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
-                  float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws);
+                  float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws,
+                  const aero_fwd_extra& ex);
 int aero_bwd_fp32(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                   const float* H, const float* W, const int32_t* y, const int64_t* cs, const uint8_t* keep,
-                  const float* lse, const float* g, float grad_scale, float* dH, float* dW, int accumulate_dW);
+                  const float* lse, const float* g, float grad_scale, float* dH, float* dW, int accumulate_dW,
+                  const aero_bwd_extra& ex);
 
 // ---- stage (b): tcgen05 / TMEM / TMA path (bf16) -------------------------------------
 size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t R);
 int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                 const void* H, const void* W, const int32_t* y, const float* old_logp,
                 const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
-                float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws);
+                float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws,
+                const aero_fwd_extra& ex);
 size_t aero_bwd_ws_bytes_tc(int64_t T, int32_t d, int32_t V, int32_t R, int64_t chunk_tokens);
 int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                 const void* H, const void* W, const int32_t* y, const int64_t* cs, const uint8_t* keep,
                 const float* lse, const float* g, float grad_scale, void* dH, float* dW, int accumulate_dW,
-                void* ws, size_t ws_bytes);
+                void* ws, size_t ws_bytes, const aero_bwd_extra& ex);

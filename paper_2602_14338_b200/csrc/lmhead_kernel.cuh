@@ -4,9 +4,14 @@
 // The logits never reach shared or global memory.
 //
 //   MODE_FWD : online log-sum-exp over vocabulary tiles + target pick, then the clipped
-//              surrogate of Eq. 2 per token (logp, lse, g, per-tile loss partials).
+//              surrogate of Eq. 2 per token (logp, lse, g, per-tile loss partials), with the
+//              KL-to-reference term when a reference log-prob is given; or, without old
+//              log-probs, the log-probs alone.
 //   MODE_DZ  : dz = coef_t * (1[v == y_t] - exp(z - lse_t)) rounded to bf16 and stored to
 //              the chunk's scratch block (Eq. 3 through the softmax).
+//   The _ENT variants add the entropy bonus (Table 9): the forward also carries
+//   sum_v exp(z - m) z, giving H_t = lse_t - E_p[z]; the backward adds
+//   e_t p_tv (z_tv - lse_t + H_t) to dz, e_t = ent_coef * w_i.
 //
 // CTAs work in pairs (a cluster of two, tcgen05 cta_group::2): the pair takes two token tiles,
 // one per CTA, and one MMA covers both (M = 256).  Each CTA stages its own 128 rows of H and
@@ -36,7 +41,8 @@ namespace lmhead {
 constexpr int BM = 128, BN = 256, BNH = BN / 2, BK = 64, STAGES = AERO_TC_STAGES, UMMA_K = 16;
 constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BNH * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
-constexpr int MODE_FWD = 0, MODE_DZ = 1;
+constexpr int MODE_FWD = 0, MODE_DZ = 1, MODE_FWD_ENT = 2, MODE_DZ_ENT = 3;   // bit 0: dz mode, bit 1: entropy term
+constexpr float kMasked = -1e30f;   // stands for -inf in columns past V (finite, so that 0 * z stays 0)
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 
 struct Ctl {
@@ -57,19 +63,23 @@ struct Params {
   int tile_begin, tile_end;     // this launch covers tiles [tile_begin, min(tile_end, *n_tiles))
   const int32_t* y;
   uint32_t* status;
-  // MODE_FWD
-  const float* old_logp;
   const int64_t* cs;
-  const float* adv;
   const float* w;
-  float clip_lo, clip_hi;
+  float ent_coef;
+  // forward modes
+  const float* old_logp;        // NULL: log-probs only, no objective
+  const float* ref_logp;        // NULL: no KL term
+  const float* adv;
+  float clip_lo, clip_hi, kl_beta;
   float* logp;
   float* lse_out;
   float* g_out;
+  float* ent_out;               // entropy per row (entropy modes)
   double* partials;             // [tile][4 epilogue warps][kPartialStride]
-  // MODE_DZ
+  // dz modes
   const float* lse_in;
   const float* g_in;
+  const float* ent_in;
   float grad_scale;
   __nv_bfloat16* dz;            // [(tile - tile_begin) * 128 + r][ldz]
   long long ldz;
@@ -90,6 +100,7 @@ template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW,
               const __grid_constant__ CUtensorMap tmDZ, const Params p) {
+  constexpr bool IS_DZ = (MODE & 1) != 0, ENT = (MODE & 2) != 0;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stg_all = smem + (size_t)STAGES * STAGE_BYTES;
@@ -191,10 +202,19 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
       if (bad_y) { aero_raise(p.status, AERO_ST_BAD_TARGET); yt = -1; }
       const bool live = valid_row && !bad_y;
 
-      float m2 = -INFINITY, l = 0.f, zy = 0.f;         // MODE_FWD running state (log2 domain)
-      float lse2 = 0.f, coef = 0.f;                    // MODE_DZ per-row constants
-      if (MODE == MODE_DZ) {
-        if (live) { lse2 = p.lse_in[row] * kLog2e; coef = p.g_in[row] * p.grad_scale; }
+      float m2 = -INFINITY, l = 0.f, zy = 0.f, sz = 0.f;   // forward running state (log2 domain); sz = sum e^(z-m) z
+      float lse2 = 0.f, coef = 0.f, et = 0.f, c0 = 0.f;     // dz per-row constants: dz = 1[y] coef + p (c0 + et z)
+      if (IS_DZ) {
+        if (live) {
+          const float ls = p.lse_in[row];
+          lse2 = ls * kLog2e;
+          coef = p.g_in[row] * p.grad_scale;
+          c0 = -coef;
+          if (ENT) {
+            et = p.ent_coef * p.w[aero_owner(p.cs, p.R, row)] * p.grad_scale;
+            c0 += et * (p.ent_in[row] - ls);
+          }
+        }
       }
       const int dz_row0 = (tile - p.tile_begin) * BM + warp * 32;   // first dz row of this warp
 
@@ -211,27 +231,33 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
           continue;
         }
         const int col_base = j * BN;
-        const int ncol = min(BN, (MODE == MODE_DZ ? (int)p.ldz : p.V) - col_base);
+        const int ncol = min(BN, (IS_DZ ? (int)p.ldz : p.V) - col_base);
         const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + buf * BN;
         // One 32-column chunk of this thread's row, already in registers.
         auto process = [&](const uint32_t (&r)[32], int c) {
           const int col0 = col_base + c * 32;
-          if (MODE == MODE_FWD) {
+          if (!IS_DZ) {
             float z[32];
 #pragma unroll
             for (int q = 0; q < 32; ++q) z[q] = __uint_as_float(r[q]);
             if (col0 + 32 > p.V) {
 #pragma unroll
-              for (int q = 0; q < 32; ++q) if (col0 + q >= p.V) z[q] = -INFINITY;
+              for (int q = 0; q < 32; ++q) if (col0 + q >= p.V) z[q] = kMasked;
             }
             float cmax = z[0];
 #pragma unroll
             for (int q = 1; q < 32; ++q) cmax = fmaxf(cmax, z[q]);
             const float m2n = fmaxf(m2, cmax * kLog2e);
-            float acc = 0.f;
+            float acc = 0.f, accz = 0.f;
 #pragma unroll
-            for (int q = 0; q < 32; ++q) acc += ex2(fmaf(z[q], kLog2e, -m2n));
-            l = fmaf(l, ex2(m2 - m2n), acc);
+            for (int q = 0; q < 32; ++q) {
+              const float e = ex2(fmaf(z[q], kLog2e, -m2n));
+              acc += e;
+              if (ENT) accz = fmaf(e, z[q], accz);
+            }
+            const float scale = ex2(m2 - m2n);
+            l = fmaf(l, scale, acc);
+            if (ENT) sz = fmaf(sz, scale, accz);
             m2 = m2n;
             if ((unsigned)(yt - col0) < 32u) {
               const int sel = yt - col0;
@@ -245,7 +271,11 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
             if (live && col0 + 32 <= p.V) {
               float v[32];
 #pragma unroll
-              for (int q = 0; q < 32; ++q) v[q] = -coef * ex2(fmaf(__uint_as_float(r[q]), kLog2e, -lse2));
+              for (int q = 0; q < 32; ++q) {
+                const float z = __uint_as_float(r[q]);
+                const float pr = ex2(fmaf(z, kLog2e, -lse2));
+                v[q] = ENT ? pr * fmaf(et, z, c0) : c0 * pr;
+              }
               if ((unsigned)(yt - col0) < 32u) {
                 const int sel = yt - col0;
 #pragma unroll
@@ -256,8 +286,9 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
             } else {
 #pragma unroll
               for (int q = 0; q < 32; q += 2) {
-                float v0 = -coef * ex2(fmaf(__uint_as_float(r[q]), kLog2e, -lse2));
-                float v1 = -coef * ex2(fmaf(__uint_as_float(r[q + 1]), kLog2e, -lse2));
+                const float z0 = __uint_as_float(r[q]), z1 = __uint_as_float(r[q + 1]);
+                float v0 = ex2(fmaf(z0, kLog2e, -lse2)) * (ENT ? fmaf(et, z0, c0) : c0);
+                float v1 = ex2(fmaf(z1, kLog2e, -lse2)) * (ENT ? fmaf(et, z1, c0) : c0);
                 if (col0 + q == yt) v0 += coef;
                 if (col0 + q + 1 == yt) v1 += coef;
                 if (!live || col0 + q >= p.V) v0 = 0.f;
@@ -310,23 +341,36 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
         if (lane == 0) tc::mbar_arrive_cluster(tc::mapa_shared(tc::smem_u32(&ctl->tempty[buf]), 0));
       }
 
-      if (MODE == MODE_FWD && ok && have_tile) {
+      if (!IS_DZ && ok && have_tile) {
         double part[kPartialStride] = {0.0, 0.0, 0.0, 0.0, 0.0};
         if (live) {
           const float ls = (m2 + __log2f(l)) * kLn2;
           const float lp = zy - ls;
-          const int i = aero_owner(p.cs, p.R, row);
-          const float old = p.old_logp[row];
-          const float wi = p.w[i];
-          const SurrogateOut so = aero_surrogate(lp, old, p.adv[i], wi, p.clip_lo, p.clip_hi);
+          const float ent = ENT ? ls - sz / l : 0.f;       // H = lse - E_p[z]
           p.logp[row] = lp;
           p.lse_out[row] = ls;
-          p.g_out[row] = so.g;
-          part[0] = (double)wi * (double)so.s;
-          part[1] = so.clipped;
-          part[2] = so.rho;
-          part[3] = (double)old - (double)lp;
-          part[4] = 1.0;
+          if (ENT) p.ent_out[row] = ent;
+          if (p.old_logp != nullptr) {
+            const int i = aero_owner(p.cs, p.R, row);
+            const float old = p.old_logp[row];
+            const float wi = p.w[i];
+            const SurrogateOut so = aero_surrogate(lp, old, p.adv[i], wi, p.clip_lo, p.clip_hi);
+            float g = so.g;
+            float obj = so.s;                              // per-token objective: s - beta D + c_H H
+            if (p.ref_logp != nullptr) {
+              const float q = p.ref_logp[row] - lp;
+              const float eq = __expf(q);
+              obj -= p.kl_beta * (eq - q - 1.f);
+              g += p.kl_beta * wi * (1.f - eq);
+            }
+            if (ENT) obj += p.ent_coef * ent;
+            p.g_out[row] = g;
+            part[0] = (double)wi * (double)obj;
+            part[1] = so.clipped;
+            part[2] = so.rho;
+            part[3] = (double)old - (double)lp;
+            part[4] = 1.0;
+          }
         }
         // fixed-shape reduction: a shuffle tree per warp; the four warps' records are
         // added later by the finalising kernel in a fixed order
@@ -342,7 +386,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
   }
 
   // ---------------- teardown ----------------
-  if (MODE == MODE_DZ && warp < 4 && lane == 0) tc::tma_store_wait_all<0>();   // own stores have landed
+  if (IS_DZ && warp < 4 && lane == 0) tc::tma_store_wait_all<0>();   // own stores have landed
   __syncwarp();
   if (*abort_flag) {
     // a wait gave up: let copies and MMAs already in flight land before shared memory and

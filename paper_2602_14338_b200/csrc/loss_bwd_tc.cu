@@ -37,7 +37,7 @@ size_t aero_bwd_ws_bytes_tc(int64_t T, int32_t d, int32_t V, int32_t R, int64_t 
 int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                 const void* H, const void* W, const int32_t* y, const int64_t* cs, const uint8_t* keep,
                 const float* lse, const float* g, float grad_scale, void* dH, float* dW, int accumulate_dW,
-                void* ws, size_t ws_bytes) {
+                void* ws, size_t ws_bytes, const aero_bwd_extra& ex) {
   (void)cfg;
   if (!accumulate_dW) AERO_CUDA_TRY(cudaMemsetAsync(dW, 0, (size_t)V * d * sizeof(float), ctx->stream));
   if (T == 0 || R == 0) return AERO_OK;
@@ -76,7 +76,8 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
   CUtensorMap tmDZ_st;
   if ((rc = aero_make_tmap_2d(ctx, &tmDZ_st, BF, 2, dz, dz_rows, ldz, ldz, 32, 64))) return rc;
 
-  auto k_dz = lmhead::lmhead_kernel<lmhead::MODE_DZ>;
+  const bool with_entropy = ex.entropy != nullptr && ex.ent_coef != 0.f;
+  auto k_dz = with_entropy ? lmhead::lmhead_kernel<lmhead::MODE_DZ_ENT> : lmhead::lmhead_kernel<lmhead::MODE_DZ>;
   auto k_dh = gemmbwd::gemm_kernel<gemmbwd::KIND_DH>;
   auto k_dw = gemmbwd::gemm_kernel<gemmbwd::KIND_DW>;
   AERO_CUDA_TRY(cudaFuncSetAttribute(k_dz, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lmhead::SMEM_BYTES));
@@ -92,6 +93,7 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     lp.tile_begin = (int)begin; lp.tile_end = (int)(begin + tpc);
     lp.y = y; lp.status = ctx->d_status;
     lp.lse_in = lse; lp.g_in = g; lp.grad_scale = grad_scale; lp.dz = dz; lp.ldz = ldz;
+    lp.cs = cs; lp.w = ex.w; lp.ent_in = ex.entropy; lp.ent_coef = ex.ent_coef;
     const long long max_pairs = ctx->sm_count / 2 > 0 ? ctx->sm_count / 2 : 1;
     const long long dz_pairs = (tpc + 1) / 2;
     const int grid_dz = 2 * (int)(dz_pairs < max_pairs ? dz_pairs : max_pairs);

@@ -97,6 +97,19 @@ __global__ void __launch_bounds__(1024) build_tiles_kernel(long long T, int R, c
   if (threadIdx.x == 0) *n_tiles = carry_tiles < max_tiles ? carry_tiles : max_tiles;
 }
 
+__global__ void __launch_bounds__(256) dense_tiles_kernel(long long T, int tile_rows, int32_t* __restrict__ tile_row,
+                                                          int32_t* __restrict__ tile_valid, int32_t* __restrict__ n_tiles,
+                                                          int max_tiles) {
+  const long long n = (T + tile_rows - 1) / tile_rows;
+  const int count = (int)(n < max_tiles ? n : max_tiles);
+  for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < count; k += gridDim.x * blockDim.x) {
+    const long long start = (long long)k * tile_rows;
+    tile_row[k] = (int32_t)start;
+    tile_valid[k] = (int32_t)(T - start < tile_rows ? T - start : tile_rows);
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) *n_tiles = count;
+}
+
 // Sum n partial records of `stride` doubles each in a fixed order: thread j adds records
 // j, j+1024, ... in increasing order, then a fixed shuffle/shared tree combines threads.
 __global__ void __launch_bounds__(1024) finalize_kernel(const double* __restrict__ part, int n, int stride,
@@ -148,6 +161,20 @@ aero_tiles aero_carve_tiles(void* ws, int64_t T, int32_t R, int tile_rows) {
   t.tile_valid = reinterpret_cast<int32_t*>(p);
   t.max_tiles = (int32_t)mt;
   return t;
+}
+
+int aero_build_dense_tiles(aero_ctx* ctx, int64_t T, int tile_rows, aero_tiles tiles) {
+  if (T == 0) {
+    AERO_CUDA_TRY(cudaMemsetAsync(tiles.n_tiles, 0, sizeof(int32_t), ctx->stream));
+    return AERO_OK;
+  }
+  const long long n = (T + tile_rows - 1) / tile_rows;
+  const int blocks = (int)((n + 255) / 256 < 1024 ? (n + 255) / 256 : 1024);
+  dense_tiles_kernel<<<blocks, 256, 0, ctx->stream>>>(T, tile_rows, tiles.tile_row, tiles.tile_valid, tiles.n_tiles,
+                                                       tiles.max_tiles);
+  ctx->launches += 1;
+  AERO_CUDA_TRY(cudaGetLastError());
+  return AERO_OK;
 }
 
 int aero_build_tiles(aero_ctx* ctx, int64_t T, int32_t R, const int64_t* cs, const uint8_t* keep,

@@ -32,60 +32,101 @@ fwd_fp32_kernel(aero_cfg cfg, long long T, int d, int V, int R,
                 const float* __restrict__ old_logp, const int64_t* __restrict__ cs,
                 const float* __restrict__ adv, const float* __restrict__ wgt, const uint8_t* __restrict__ keep,
                 float* __restrict__ logp, float* __restrict__ lse, float* __restrict__ g,
-                double* __restrict__ partials, uint32_t* status) {
+                double* __restrict__ partials, uint32_t* status, aero_fwd_extra ex) {
   const int lane = threadIdx.x & 31;
   const long long warp0 = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
   const long long nwarps = (long long)gridDim.x * kWarpsPerBlock;
   for (long long t = warp0; t < T; t += nwarps) {
     double* pr = partials + (size_t)t * kPartialStride;
-    const int i = aero_owner(cs, R, t);
+    const int i = ex.logprob_only ? 0 : aero_owner(cs, R, t);
+    const bool kp = ex.logprob_only ? true : keep[i] != 0;
     const int yt = y[t];
     const bool bad = yt < 0 || yt >= V;
-    if (bad && keep[i] && lane == 0) aero_raise(status, AERO_ST_BAD_TARGET);
-    if (!keep[i] || bad) {
+    if (bad && kp && lane == 0) aero_raise(status, AERO_ST_BAD_TARGET);
+    if (!kp || bad) {
       if (lane == 0) {
-        logp[t] = 0.f; lse[t] = 0.f; g[t] = 0.f;
+        logp[t] = 0.f; lse[t] = 0.f;
+        if (g) g[t] = 0.f;
+        if (ex.entropy) ex.entropy[t] = 0.f;
         for (int k = 0; k < kPartialStride; ++k) pr[k] = 0.0;
       }
       continue;
     }
     const float* h = H + (size_t)t * d;
-    float m = -INFINITY, l = 0.f;
+    float m = -INFINITY, l = 0.f, sz = 0.f;       // sz = sum_v exp(z_v - m) z_v, for the entropy
     for (int v = lane; v < V; v += 32) {
       const float z = dot_row(h, W + (size_t)v * d, d);
       const float mn = fmaxf(m, z);
-      l = l * __expf(m - mn) + __expf(z - mn);
+      const float sc = __expf(m - mn), e = __expf(z - mn);
+      l = l * sc + e;
+      sz = sz * sc + e * z;
       m = mn;
     }
     const float M = warp_max(m);
-    l = warp_sum(l * __expf(m - M));
+    const float sc = __expf(m - M);
+    l = warp_sum(l * sc);
+    sz = warp_sum(sz * sc);
     const float ls = M + __logf(l);
     if (lane == 0) {
       const float zy = dot_row(h, W + (size_t)yt * d, d);
       const float lp = zy - ls;
-      const SurrogateOut so = aero_surrogate(lp, old_logp[t], adv[i], wgt[i], cfg.clip_lo, cfg.clip_hi);
-      logp[t] = lp; lse[t] = ls; g[t] = so.g;
-      pr[0] = (double)wgt[i] * (double)so.s;
-      pr[1] = so.clipped;
-      pr[2] = so.rho;
-      pr[3] = (double)old_logp[t] - (double)lp;
-      pr[4] = 1.0;
+      const float ent = ls - sz / l;              // H = lse - E_p[z]
+      logp[t] = lp; lse[t] = ls;
+      if (ex.entropy) ex.entropy[t] = ent;
+      for (int k = 0; k < kPartialStride; ++k) pr[k] = 0.0;
+      if (!ex.logprob_only) {
+        const SurrogateOut so = aero_surrogate(lp, old_logp[t], adv[i], wgt[i], cfg.clip_lo, cfg.clip_hi);
+        float gt = so.g, obj = so.s;              // per-token objective: s - beta D + c_H H
+        if (ex.ref_logp) {
+          const float q = ex.ref_logp[t] - lp;
+          const float eq = __expf(q);
+          obj -= ex.kl_beta * (eq - q - 1.f);
+          gt += ex.kl_beta * wgt[i] * (1.f - eq);
+        }
+        if (ex.entropy) obj += ex.ent_coef * ent;
+        g[t] = gt;
+        pr[0] = (double)wgt[i] * (double)obj;
+        pr[1] = so.clipped;
+        pr[2] = so.rho;
+        pr[3] = (double)old_logp[t] - (double)lp;
+        pr[4] = 1.0;
+      }
     }
   }
+}
+
+// Per-row constants of dz = gs * (g (1[v=y] - p) + e p (z - lse + H)) = 1[v=y] coef + p (c0 + et z).
+struct RowDz { float coef, c0, et; };
+__device__ __forceinline__ RowDz row_dz(long long t, float gs, const float* __restrict__ g, const float* __restrict__ lse,
+                                        const int64_t* __restrict__ cs, int R, const uint8_t* __restrict__ keep,
+                                        const aero_bwd_extra& ex) {
+  RowDz r;
+  r.coef = g[t] * gs;
+  r.c0 = -r.coef;
+  r.et = 0.f;
+  if (ex.entropy && ex.ent_coef != 0.f) {
+    const int i = aero_owner(cs, R, t);
+    if (keep[i]) {
+      r.et = ex.ent_coef * ex.w[i] * gs;
+      r.c0 += r.et * (ex.entropy[t] - lse[t]);
+    }
+  }
+  return r;
 }
 
 // dH[t, :] = g_t * gs * (W[y_t, :] - sum_v p_tv W[v, :]), one warp per token row.
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 bwd_dh_fp32_kernel(long long T, int d, int V, const float* __restrict__ H, const float* __restrict__ W,
                    const int32_t* __restrict__ y, const float* __restrict__ lse, const float* __restrict__ g,
-                   float gs, float* __restrict__ dH) {
+                   float gs, float* __restrict__ dH, const int64_t* __restrict__ cs, int R,
+                   const uint8_t* __restrict__ keep, aero_bwd_extra ex) {
   const int lane = threadIdx.x & 31;
   const long long warp0 = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
   const long long nwarps = (long long)gridDim.x * kWarpsPerBlock;
   for (long long t = warp0; t < T; t += nwarps) {
-    const float gt = g[t] * gs;
+    const RowDz rd = row_dz(t, gs, g, lse, cs, R, keep, ex);
     float* out = dH + (size_t)t * d;
-    if (gt == 0.f) {
+    if (rd.coef == 0.f && rd.et == 0.f) {
       for (int k = lane; k < d; k += 32) out[k] = 0.f;
       continue;
     }
@@ -101,7 +142,7 @@ bwd_dh_fp32_kernel(long long T, int d, int V, const float* __restrict__ H, const
         float part = 0.f;
         for (int k = lane; k < d; k += 32) part = fmaf(h[k], wv[k], part);
         const float z = warp_sum(part);
-        const float dz = gt * ((v == yt ? 1.f : 0.f) - __expf(z - ls));
+        const float dz = (v == yt ? rd.coef : 0.f) + __expf(z - ls) * fmaf(rd.et, z, rd.c0);
 #pragma unroll
         for (int q = 0; q < kChunk / 32; ++q) {
           const int k = c0 + q * 32 + lane;
@@ -121,7 +162,8 @@ bwd_dh_fp32_kernel(long long T, int d, int V, const float* __restrict__ H, const
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 bwd_dw_fp32_kernel(long long T, int d, int V, const float* __restrict__ H, const float* __restrict__ W,
                    const int32_t* __restrict__ y, const float* __restrict__ lse, const float* __restrict__ g,
-                   float gs, float* __restrict__ dW, int accumulate) {
+                   float gs, float* __restrict__ dW, int accumulate, const int64_t* __restrict__ cs, int R,
+                   const uint8_t* __restrict__ keep, aero_bwd_extra ex) {
   const int lane = threadIdx.x & 31;
   const int warp0 = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
   const int nwarps = gridDim.x * kWarpsPerBlock;
@@ -133,13 +175,13 @@ bwd_dw_fp32_kernel(long long T, int d, int V, const float* __restrict__ H, const
 #pragma unroll
       for (int q = 0; q < kChunk / 32; ++q) acc[q] = 0.f;
       for (long long t = 0; t < T; ++t) {
-        const float gt = g[t] * gs;
-        if (gt == 0.f) continue;
+        const RowDz rd = row_dz(t, gs, g, lse, cs, R, keep, ex);
+        if (rd.coef == 0.f && rd.et == 0.f) continue;
         const float* h = H + (size_t)t * d;
         float part = 0.f;
         for (int k = lane; k < d; k += 32) part = fmaf(h[k], wv[k], part);
         const float z = warp_sum(part);
-        const float dz = gt * ((v == y[t] ? 1.f : 0.f) - __expf(z - lse[t]));
+        const float dz = (v == y[t] ? rd.coef : 0.f) + __expf(z - lse[t]) * fmaf(rd.et, z, rd.c0);
 #pragma unroll
         for (int q = 0; q < kChunk / 32; ++q) {
           const int k = c0 + q * 32 + lane;
@@ -165,33 +207,37 @@ size_t aero_fwd_ws_bytes_fp32(int64_t T, int32_t R) {
 int aero_fwd_fp32(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                   const float* H, const float* W, const int32_t* y, const float* old_logp,
                   const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
-                  float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws) {
+                  float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws,
+                  const aero_fwd_extra& ex) {
   double* partials = static_cast<double*>(ws);
-  if (T > 0 && R > 0) {
+  if (T > 0 && (R > 0 || ex.logprob_only)) {
     const long long blocks = (T + kWarpsPerBlock - 1) / kWarpsPerBlock;
     const int grid = (int)(blocks < 65535 ? blocks : 65535);
     fwd_fp32_kernel<<<grid, kWarpsPerBlock * 32, 0, ctx->stream>>>(*cfg, T, d, V, R, H, W, y, old_logp, cs, adv, w,
-                                                                   keep, logp, lse, g, partials, ctx->d_status);
+                                                                   keep, logp, lse, g, partials, ctx->d_status, ex);
     ctx->launches += 1;
     AERO_CUDA_TRY(cudaGetLastError());
   }
+  if (ex.logprob_only) return AERO_OK;
   return aero_loss_finalize(ctx, partials, (T > 0 && R > 0) ? (int)T : 0, kPartialStride, loss, metrics, accumulate);
 }
 
 int aero_bwd_fp32(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                   const float* H, const float* W, const int32_t* y, const int64_t* cs, const uint8_t* keep,
-                  const float* lse, const float* g, float grad_scale, float* dH, float* dW, int accumulate_dW) {
-  (void)cfg; (void)cs; (void)keep; (void)R;
+                  const float* lse, const float* g, float grad_scale, float* dH, float* dW, int accumulate_dW,
+                  const aero_bwd_extra& ex) {
+  (void)cfg;
   if (T > 0) {
     const long long blocks = (T + kWarpsPerBlock - 1) / kWarpsPerBlock;
     const int grid = (int)(blocks < 65535 ? blocks : 65535);
-    bwd_dh_fp32_kernel<<<grid, kWarpsPerBlock * 32, 0, ctx->stream>>>(T, d, V, H, W, y, lse, g, grad_scale, dH);
+    bwd_dh_fp32_kernel<<<grid, kWarpsPerBlock * 32, 0, ctx->stream>>>(T, d, V, H, W, y, lse, g, grad_scale, dH, cs, R,
+                                                                      keep, ex);
     ctx->launches += 1;
     AERO_CUDA_TRY(cudaGetLastError());
   }
   const int vblocks = (V + kWarpsPerBlock - 1) / kWarpsPerBlock;
   bwd_dw_fp32_kernel<<<vblocks < 65535 ? vblocks : 65535, kWarpsPerBlock * 32, 0, ctx->stream>>>(
-      T, d, V, H, W, y, lse, g, grad_scale, dW, accumulate_dW);
+      T, d, V, H, W, y, lse, g, grad_scale, dW, accumulate_dW, cs, R, keep, ex);
   ctx->launches += 1;
   AERO_CUDA_TRY(cudaGetLastError());
   return AERO_OK;

@@ -30,17 +30,20 @@ size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t R) {
 int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                 const void* H, const void* W, const int32_t* y, const float* old_logp,
                 const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
-                float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws) {
+                float* logp, float* lse, float* g, float* loss, float* metrics, int accumulate, void* ws,
+                const aero_fwd_extra& ex) {
   FwdWs f = carve_fwd(ws, T, R);
   AERO_CUDA_TRY(cudaMemsetAsync(f.partials, 0, f.n_partials * kPartialStride * sizeof(double), ctx->stream));
   if (T > 0) {
     AERO_CUDA_TRY(cudaMemsetAsync(logp, 0, (size_t)T * sizeof(float), ctx->stream));
     AERO_CUDA_TRY(cudaMemsetAsync(lse, 0, (size_t)T * sizeof(float), ctx->stream));
-    AERO_CUDA_TRY(cudaMemsetAsync(g, 0, (size_t)T * sizeof(float), ctx->stream));
+    if (g) AERO_CUDA_TRY(cudaMemsetAsync(g, 0, (size_t)T * sizeof(float), ctx->stream));
+    if (ex.entropy) AERO_CUDA_TRY(cudaMemsetAsync(ex.entropy, 0, (size_t)T * sizeof(float), ctx->stream));
   }
-  int rc = aero_build_tiles(ctx, T, R, cs, keep, lmhead::BM, f.tiles);
+  int rc = ex.logprob_only ? aero_build_dense_tiles(ctx, T, lmhead::BM, f.tiles)
+                           : aero_build_tiles(ctx, T, R, cs, keep, lmhead::BM, f.tiles);
   if (rc) return rc;
-  if (T > 0 && R > 0) {
+  if (T > 0 && (R > 0 || ex.logprob_only)) {
     CUtensorMap tmH, tmW;
     rc = aero_make_tmap_2d(ctx, &tmH, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, H, (uint64_t)T, (uint64_t)d, (uint64_t)d,
                            lmhead::BM, lmhead::BK);
@@ -53,10 +56,11 @@ int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     p.tile_row = f.tiles.tile_row; p.tile_valid = f.tiles.tile_valid; p.n_tiles = f.tiles.n_tiles;
     p.tile_begin = 0; p.tile_end = f.tiles.max_tiles;
     p.y = y; p.status = ctx->d_status;
-    p.old_logp = old_logp; p.cs = cs; p.adv = adv; p.w = w;
+    p.old_logp = ex.logprob_only ? nullptr : old_logp; p.cs = cs; p.adv = adv; p.w = w;
+    p.ref_logp = ex.ref_logp; p.kl_beta = ex.kl_beta; p.ent_coef = ex.ent_coef; p.ent_out = ex.entropy;
     p.clip_lo = cfg->clip_lo; p.clip_hi = cfg->clip_hi;
     p.logp = logp; p.lse_out = lse; p.g_out = g; p.partials = f.partials;
-    auto kern = lmhead::lmhead_kernel<lmhead::MODE_FWD>;
+    auto kern = ex.entropy ? lmhead::lmhead_kernel<lmhead::MODE_FWD_ENT> : lmhead::lmhead_kernel<lmhead::MODE_FWD>;
     AERO_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lmhead::SMEM_BYTES));
     // one CTA pair per two token tiles, at most one pair per two SMs
     const int64_t upper_pairs = (T / lmhead::BM + R + 2) / 2;
@@ -66,5 +70,6 @@ int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     ctx->launches += 1;
     AERO_CUDA_TRY(cudaGetLastError());
   }
+  if (ex.logprob_only) return AERO_OK;
   return aero_loss_finalize(ctx, f.partials, (int)f.n_partials, kPartialStride, loss, metrics, accumulate);
 }

@@ -17,7 +17,8 @@ def lib_cfg(ocfg, dtype):
                          rescue_S=ocfg.rescue_S, n_explore=ocfg.n_explore, n_keep_uniform=ocfg.n_keep_uniform,
                          stats_over=ocfg.stats_over, agg=ocfg.agg, denom=ocfg.denom, alpha0=ocfg.alpha0,
                          beta0=ocfg.beta0, eps_std=ocfg.eps_std, clip_lo=ocfg.clip_lo, clip_hi=ocfg.clip_hi,
-                         seed=ocfg.seed, dtype=B.AERO_BF16 if dtype == "bf16" else B.AERO_FP32)
+                         seed=ocfg.seed, dtype=B.AERO_BF16 if dtype == "bf16" else B.AERO_FP32,
+                         kl_beta=ocfg.kl_beta, ent_coef=ocfg.ent_coef)
 
 
 def cfg_for(wl, **over):

@@ -295,6 +295,94 @@ def test_full_width_qwen_7b_shape(ctx):
     assert TL.rel_l2(dW.cpu().numpy()[rows], rdW) < GRAD_L2
 
 
+REG_CASES = {
+    # name: (dtype, workload overrides, cfg overrides, peak, use reference log-probs)
+    "tiny_fp32_kl_entropy": ("fp32", dict(), dict(kl_beta=0.04, ent_coef=1e-3), 0.0, True),
+    "bf16_entropy_only": ("bf16", dict(P=6, n_lo=3, n_hi=9, d=128, V=1000, len_median=70.0, len_cap=300, dtype="bf16",
+                                       seed=41), dict(ent_coef=0.05), 0.0, False),
+    "bf16_kl_only": ("bf16", dict(P=6, n_lo=3, n_hi=9, d=128, V=3001, len_median=50.0, len_cap=200, dtype="bf16",
+                                  seed=42), dict(kl_beta=0.5), 0.0, True),
+    "bf16_peaked_kl_entropy": ("bf16", dict(P=6, n_lo=4, n_hi=8, d=128, V=4096, len_median=60.0, len_cap=200,
+                                            dtype="bf16", aero=True, seed=43),
+                               dict(kl_beta=0.2, ent_coef=0.3, uniform_policy=O.UNIFORM_BAYES, rejection=1), 45.0, True),
+}
+
+
+@pytest.mark.parametrize("name", list(REG_CASES))
+def test_regularised_objective(ctx, name):
+    """Eq. 2's KL term and the entropy bonus of Table 9 through aero_grpo_loss_reg_fwd / _bwd against
+    the oracle.  The coefficients are larger than the paper's so that both terms carry weight in
+    every tolerance; the peaked case makes the entropy gradient comparable to the policy gradient."""
+    dtype, over, cover, peak, use_ref = REG_CASES[name]
+    base = synth.WORKLOADS[0] if dtype == "fp32" else synth.WORKLOADS[1]
+    wl = synth.scaled(base, **over)
+    batch = TL.Batch(wl, O.Cfg(seed=wl.seed, **cover), peak=peak)
+    ocfg = batch.ocfg
+    rg = batch.ref_g
+    rng = np.random.default_rng(5)
+    ref_lp = (batch.old.astype(np.float64) + 0.3 * rng.standard_normal(batch.T)).astype(np.float32) if use_ref else None
+    adv32 = rg["adv"].astype(np.float32).astype(np.float64)
+    w32 = rg["w"].astype(np.float32).astype(np.float64)
+    ref = O.grpo_loss_reg_fwd(ocfg, batch.H, batch.W, batch.st.y, batch.old, ref_lp, batch.st.cs, adv32, w32, rg["keep"])
+    rdH, rdW = O.grpo_loss_reg_bwd(ocfg, batch.H, batch.W, batch.st.y, batch.st.cs, rg["keep"], ref["lse"], ref["g"],
+                                   ref["entropy"], w32)
+    cfg = TL.lib_cfg(ocfg, dtype)
+    dv = batch.to_device()
+    want_ent = ocfg.ent_coef != 0.0
+    f = ctx.grpo_loss_reg_fwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], TL.dev(ref_lp) if use_ref else None,
+                              dv["cs"], dv["adv"], dv["w"], dv["keep"], entropy=want_ent)
+    if want_ent:
+        dH, dW = ctx.grpo_loss_reg_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], dv["keep"], f["lse"], f["g"],
+                                       f["entropy"], dv["w"])
+    else:
+        dH, dW = ctx.grpo_loss_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], dv["keep"], f["lse"], f["g"])
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    tol = (1e-4, 1e-4, 1e-4) if dtype == "fp32" else (LOGP_ABS, LOSS_REL, GRAD_L2)
+    owner = O.token_rollout(batch.st.cs, batch.T)
+    kept = rg["keep"][owner] != 0
+    assert np.abs(f["logp"][:batch.T].cpu().numpy() - ref["logp"]).max() <= tol[0]
+    if want_ent:
+        ent = f["entropy"][:batch.T].cpu().numpy()
+        assert np.abs(ent - ref["entropy"]).max() <= tol[0] and not ent[~kept].any()
+        assert ref["entropy"][kept].min() > 0.05          # the term is not vacuous
+    assert abs(f["loss"].item() - ref["loss"]) <= tol[1] * abs(ref["loss"]) + 1e-7
+    rho = ref["rho"]
+    edge = (np.abs(rho - (1 + ocfg.clip_hi)) < 1e-3) | (np.abs(rho - (1 - ocfg.clip_lo)) < 1e-3)
+    np.testing.assert_allclose(f["g"][:batch.T].cpu().numpy()[~edge], ref["g"][~edge], rtol=2e-2, atol=1e-9)
+    assert TL.rel_l2(dH.float().cpu().numpy()[~edge], rdH[~edge]) < tol[2]
+    if not edge.any():
+        assert TL.rel_l2(dW.cpu().numpy(), rdW) < tol[2]
+    # the regulariser changes the answer by more than the tolerance: the test can see it
+    plain = O.grpo_loss_fwd(ocfg, batch.H, batch.W, batch.st.y, batch.old, batch.st.cs, adv32, w32, rg["keep"])
+    pdH, _ = O.grpo_loss_bwd(batch.H, batch.W, batch.st.y, batch.st.cs, rg["keep"], plain["lse"], plain["g"])
+    assert TL.rel_l2(pdH, rdH) > 5 * tol[2]
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_logprob_pass_alone(ctx, dtype):
+    """aero_logprob_fwd over all rows (no groups, no objective): the pass that produces old and
+    reference log-probs, against log_softmax of the oracle's logits; entropy output included."""
+    if dtype == "fp32":
+        wl = synth.WORKLOADS[0]
+    else:
+        wl = synth.scaled(synth.WORKLOADS[1], P=5, n_lo=2, n_hi=6, d=192, V=5003, len_median=45.0, len_cap=150, seed=51)
+    st = synth.make_structure(wl)
+    T = int(st.cs[-1])
+    H, W = synth.make_tensors(wl, T, device="cpu")
+    z = O.logits(H.double().numpy(), W.double().numpy())
+    lp, lse = O.log_softmax_pick(z, st.y)
+    cfg = B.cfg_default(dtype=B.AERO_BF16 if dtype == "bf16" else B.AERO_FP32)
+    o = ctx.logprob_fwd(cfg, H.cuda(), W.cuda(), TL.dev(st.y), entropy=True)
+    tol = 1e-4 if dtype == "fp32" else LOGP_ABS
+    assert np.abs(o["logp"][:T].cpu().numpy() - lp).max() <= tol
+    assert np.abs(o["lse"][:T].cpu().numpy() - lse).max() <= tol
+    assert np.abs(o["entropy"][:T].cpu().numpy() - O.entropy_rows(z)).max() <= tol
+    o2 = ctx.logprob_fwd(cfg, H.cuda(), W.cuda(), TL.dev(st.y))
+    assert torch.equal(o2["logp"][:T], o["logp"][:T])
+    assert ctx.last_status() == 0
+
+
 def test_step_from_host_buffers_matches_device_calls(ctx):
     over, cover, _ = BF16_CASES["aero_dropped"]
     wl = synth.scaled(synth.WORKLOADS[1], **over)
