@@ -299,7 +299,7 @@ REG_CASES = {
     # name: (dtype, workload overrides, cfg overrides, peak, use reference log-probs)
     "tiny_fp32_kl_entropy": ("fp32", dict(), dict(kl_beta=0.04, ent_coef=1e-3), 0.0, True),
     "bf16_entropy_only": ("bf16", dict(P=6, n_lo=3, n_hi=9, d=128, V=1000, len_median=70.0, len_cap=300, dtype="bf16",
-                                       seed=41), dict(ent_coef=0.05), 0.0, False),
+                                       seed=41), dict(ent_coef=0.5), 45.0, False),
     "bf16_kl_only": ("bf16", dict(P=6, n_lo=3, n_hi=9, d=128, V=3001, len_median=50.0, len_cap=200, dtype="bf16",
                                   seed=42), dict(kl_beta=0.5), 0.0, True),
     "bf16_peaked_kl_entropy": ("bf16", dict(P=6, n_lo=4, n_hi=8, d=128, V=4096, len_median=60.0, len_cap=200,
