@@ -107,7 +107,8 @@ typedef struct aero_cfg {
   float   clip_lo, clip_hi; /* clip(rho, 1-clip_lo, 1+clip_hi)                   default 0.2, 0.2 */
   uint64_t seed;            /* seeds the default selection keys                  default 0   */
   int32_t dtype;            /* AERO_BF16 | AERO_FP32: type of H, W and dH        default BF16 */
-  int32_t reserved;
+  int32_t reject_high;      /* 1 (with rejection): also cut the correct rollouts of a     default 0   */
+                            /* high-success mixed group to min(k*(n-c), c) (appendix ablation)       */
   float   kl_beta;          /* Eq. 2's beta (KL to a reference policy); read only by   default 0 */
                             /* the *_reg_* calls                                                 */
   float   ent_coef;         /* entropy bonus coefficient (Table 9: 1e-3); read only    default 0 */
@@ -148,7 +149,10 @@ int aero_last_status(aero_ctx* ctx, uint32_t* bits);
  *             smallest (key, index) (BAYES);  low-success mixed group with rejection:
  *             all correct + the min(k*c, n-c) incorrect of smallest (key, index),
  *             where low-success means Partial, or c*n_explore <= rescue_S*n when
- *             rescue_S > 0;  any other group: all present rollouts;
+ *             rescue_S > 0;  any other group: all present rollouts -- except that with
+ *             reject_high (the appendix ablation "Effect of Discarding High-Success
+ *             Rollouts") a mixed group that is not low-success keeps all incorrect + the
+ *             min(k*(n-c), c) correct of smallest (key, index);
  *   advantage (r enters as the bit r > 0.5; a reward other than 0 or 1 raises
  *             AERO_ST_BAD_REWARD)
  *             mixed group: (r - mean)/(std + eps_std) with the population std over

@@ -53,6 +53,8 @@ class Cfg:
     uniform_policy: int = UNIFORM_MASK
     rejection: int = 0
     k_ratio: int = 1            # Sec. 4.2 Strategy 3, m = k*c; paper uses k=1
+    reject_high: int = 0        # ablation "Effect of Discarding High-Success Rollouts": 1 = also
+                                # down-sample the correct rollouts of mixed groups with u >= 0.5
     rescue_S: int = 0           # Sec. 4.2 Strategy 1; paper uses S=0
     n_explore: int = 8
     n_keep_uniform: int = 4     # "typically 4 rollouts from n" (Strategy 2); <=0 keeps all
@@ -102,7 +104,11 @@ def group_stats(cfg: Cfg, go, reward, cs, key=None, keep_in=None,
          n_keep_uniform rollouts chosen by smallest key (BAYES); with
          rejection on, low-success mixed groups keep all c correct rollouts
          and the m = min(k*c, n-c) incorrect ones of smallest (key, index);
-         every other group keeps all        [Sec. 4.2 Strategies 2 and 3]
+         every other group keeps all        [Sec. 4.2 Strategies 2 and 3];
+         with reject_high also on, a mixed group that is not low-success keeps
+         all n-c incorrect rollouts and the min(k*(n-c), c) correct ones of
+         smallest (key, index) (the appendix ablation: 5 correct / 3 incorrect
+         under 1:1 keeps 3 and 3)
       5. advantage (r - mean)/std over the kept subset with population std
          (the proof of Theorem 4.1 uses sigma^2 = mu(1-mu)); uniform groups:
          0 under MASK, (r - u~)/sqrt(u~(1-u~)) under BAYES   [Eq. 1; Sec. 3.2]
@@ -172,6 +178,10 @@ def group_stats(cfg: Cfg, go, reward, cs, key=None, keep_in=None,
                 m = min(cfg.k_ratio * c, n - c)
                 order = sorted(wrong, key=lambda i: (int(key[i]), i))
                 kept = correct + order[:m]
+            elif cfg.rejection and cfg.reject_high:
+                m = min(cfg.k_ratio * (n - c), c)
+                order = sorted(correct, key=lambda i: (int(key[i]), i))
+                kept = sorted(order[:m] + wrong)
             else:
                 kept = members
         for i in kept:

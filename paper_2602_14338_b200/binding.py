@@ -38,7 +38,7 @@ class AeroCfg(C.Structure):
         ("stats_over", C.c_int32), ("agg", C.c_int32), ("denom", C.c_int32),
         ("alpha0", C.c_float), ("beta0", C.c_float), ("eps_std", C.c_float),
         ("clip_lo", C.c_float), ("clip_hi", C.c_float),
-        ("seed", C.c_uint64), ("dtype", C.c_int32), ("reserved", C.c_int32),
+        ("seed", C.c_uint64), ("dtype", C.c_int32), ("reject_high", C.c_int32),
         ("kl_beta", C.c_float), ("ent_coef", C.c_float),
     ]
 

@@ -51,7 +51,7 @@ void aero_cfg_default(aero_cfg* cfg) {
   cfg->clip_hi = 0.2f;
   cfg->seed = 0;
   cfg->dtype = AERO_BF16;
-  cfg->reserved = 0;
+  cfg->reject_high = 0;
   cfg->kl_beta = 0.f;
   cfg->ent_coef = 0.f;
 }

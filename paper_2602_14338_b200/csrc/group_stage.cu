@@ -135,7 +135,7 @@ struct PromptState {
   unsigned kb[kMaxPT];       // kept rollouts | kept correct ones << 16 (staged path)
   int quota[kMaxPT];
   uint8_t mode[kMaxPT];      // 0 keep all present, 1 keep none, 2 select by rank
-  uint8_t reject[kMaxPT];    // select among the incorrect only, keep every correct one
+  uint8_t reject[kMaxPT];    // 1: select among the incorrect only; 2: among the correct only; 0: among all
   uint8_t uniform[kMaxPT];
   float ut[kMaxPT];
   float mu[kMaxPT];
@@ -246,7 +246,9 @@ __device__ void chain_tile(const Workspace& ws, TileShared& sh, int tile, int ti
 struct Rule {
   int category, mode;
   long long quota;
-  bool reject, uniform;
+  int reject;          // 0: every present rollout is a candidate; 1: the incorrect ones (all correct kept);
+                       // 2: the correct ones (all incorrect kept)
+  bool uniform;
   float al, be, ut;
 };
 __device__ __forceinline__ Rule decide(const Args& a, int p, int n, int c) {
@@ -262,7 +264,7 @@ __device__ __forceinline__ Rule decide(const Args& a, int p, int n, int c) {
   r.uniform = (c == 0 || c == n);
   r.mode = 0;
   r.quota = 0;
-  r.reject = false;
+  r.reject = 0;
   if (n == 0) {
     r.mode = 1;
   } else if (r.uniform) {
@@ -273,7 +275,10 @@ __device__ __forceinline__ Rule decide(const Args& a, int p, int n, int c) {
                      (a.cfg.rescue_S > 0 && (long long)c * a.cfg.n_explore <= (long long)a.cfg.rescue_S * n);
     if (a.cfg.rejection && low) {
       const long long m = min((long long)a.cfg.k_ratio * c, (long long)(n - c));
-      if (m < n - c) { r.mode = 2; r.quota = m; r.reject = true; }
+      if (m < n - c) { r.mode = 2; r.quota = m; r.reject = 1; }
+    } else if (a.cfg.rejection && a.cfg.reject_high) {
+      const long long m = min((long long)a.cfg.k_ratio * (n - c), (long long)c);
+      if (m < c) { r.mode = 2; r.quota = m; r.reject = 2; }
     }
   }
   return r;
@@ -354,8 +359,10 @@ __device__ void run_tile_staged(const Args& a, const Workspace& ws, TileShared& 
     a.alpha_out[p] = ru.al;
     a.beta_out[p] = ru.be;
     ps.mode[tid] = (uint8_t)ru.mode;
-    ps.reject[tid] = ru.reject ? 1 : 0;
-    ps.quota[tid] = (int)ru.quota;
+    ps.reject[tid] = (uint8_t)ru.reject;
+    // every incorrect rollout orders before every correct one: when the correct ones are the
+    // candidates, the n - c incorrect ones are counted by each rank and the quota allows for them
+    ps.quota[tid] = (int)ru.quota + (ru.reject == 2 ? n - c : 0);
     ps.uniform[tid] = ru.uniform ? 1 : 0;
     ps.ut[tid] = ru.ut;
     mine.cat[ru.category] = 1;
@@ -368,7 +375,8 @@ __device__ void run_tile_staged(const Args& a, const Workspace& ws, TileShared& 
     const int mode = ps.mode[q];
     const uint8_t f = rs.flag[j];
     bool kp = (f & 1) && mode != 1;
-    if (kp && mode == 2 && !(ps.reject[q] && (f & 2))) {
+    const int rej = ps.reject[q];
+    if (kp && mode == 2 && !(rej == 1 && (f & 2)) && !(rej == 2 && !(f & 2))) {
       const unsigned long long mykey = rs.ck[j];
       const int lo = ps.lo[q], hi = ps.lo[q + 1];
       int rank = 0;
@@ -511,11 +519,12 @@ __device__ void run_tile_global(const Args& a, const Workspace& ws, TileShared& 
     for (int j = lo; j < hi; ++j) {
       const bool corr = a.reward[r0 + j] > 0.5f;
       bool kp = present(j) && ru.mode != 1;
-      if (kp && ru.mode == 2 && !(ru.reject && corr)) {
+      if (kp && ru.mode == 2 && !(ru.reject == 1 && corr) && !(ru.reject == 2 && !corr)) {
         const unsigned long long mykey = order_key(j);
         long long rank = 0;
         for (int k = lo; k < hi; ++k) {
-          if (ru.reject && a.reward[r0 + k] > 0.5f) continue;
+          const bool ck = a.reward[r0 + k] > 0.5f;
+          if ((ru.reject == 1 && ck) || (ru.reject == 2 && !ck)) continue;
           rank += order_key(k) < mykey ? 1 : 0;
         }
         kp = rank < ru.quota;

@@ -13,7 +13,7 @@ def oracle_cfg(**kw):
 
 
 def lib_cfg(ocfg, dtype):
-    return B.cfg_default(uniform_policy=ocfg.uniform_policy, rejection=ocfg.rejection, k_ratio=ocfg.k_ratio,
+    return B.cfg_default(uniform_policy=ocfg.uniform_policy, rejection=ocfg.rejection, k_ratio=ocfg.k_ratio, reject_high=ocfg.reject_high,
                          rescue_S=ocfg.rescue_S, n_explore=ocfg.n_explore, n_keep_uniform=ocfg.n_keep_uniform,
                          stats_over=ocfg.stats_over, agg=ocfg.agg, denom=ocfg.denom, alpha0=ocfg.alpha0,
                          beta0=ocfg.beta0, eps_std=ocfg.eps_std, clip_lo=ocfg.clip_lo, clip_hi=ocfg.clip_hi,

@@ -32,6 +32,8 @@ GROUP_MODES = [
     dict(uniform_policy=O.UNIFORM_BAYES, rejection=1, k_ratio=2, agg=O.AGG_SEQ_MEAN),
     dict(rejection=1, stats_over=O.STATS_ALL, denom=O.DENOM_ALL),
     dict(uniform_policy=O.UNIFORM_BAYES, rejection=1, rescue_S=4, n_keep_uniform=0, agg=O.AGG_SEQ_MEAN, denom=O.DENOM_ALL),
+    dict(uniform_policy=O.UNIFORM_BAYES, rejection=1, reject_high=1),
+    dict(rejection=1, reject_high=1, k_ratio=2, stats_over=O.STATS_ALL),
 ]
 
 
@@ -66,6 +68,30 @@ def test_group_stats_ties_and_small_groups(ctx):
     ref = O.group_stats(ocfg, st.go, st.reward, st.cs, key=st.key, alpha_in=st.alpha, beta_in=st.beta)
     _, out = TL.run_group_gpu(ctx, TL.lib_cfg(ocfg, "bf16"), st)
     TL.check_group(out, ref, len(st.reward), len(st.go) - 1)
+
+
+@pytest.mark.parametrize("high", [0, 1])
+def test_group_stats_groups_larger_than_a_tile(ctx, high):
+    """Groups of thousands of rollouts do not fit the shared-memory staging of a tile and take the
+    path that walks global memory; small groups around them take the staged path.  Heavy key ties."""
+    rng = np.random.default_rng(91)
+    sizes = np.concatenate([rng.integers(1, 9, 30), [2600], rng.integers(1, 9, 25), [3100, 2400, 2500], rng.integers(1, 9, 20)])
+    P, R = len(sizes), int(sizes.sum())
+    go = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    reward = (rng.random(R) < 0.5).astype(np.float32)
+    big = np.nonzero(sizes > 1000)[0]
+    reward[go[big[0]]:go[big[0] + 1]] = 0.0                                               # uniform: keep 4 of 2600
+    reward[go[big[1]]:go[big[1] + 1]] = (rng.random(sizes[big[1]]) < 0.1).astype(np.float32)   # low success: rejection
+    reward[go[big[2]]:go[big[2] + 1]] = (rng.random(sizes[big[2]]) < 0.8).astype(np.float32)   # high success
+    lens = rng.integers(1, 50, R)
+    cs = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    key = rng.integers(0, 200, R).astype(np.uint32)
+    st = synth.Structure(go, cs, reward, key, None, None, None, None)
+    ocfg = O.Cfg(uniform_policy=O.UNIFORM_BAYES, rejection=1, reject_high=high, agg=O.AGG_SEQ_MEAN if high else O.AGG_TOKEN_MEAN)
+    ref = O.group_stats(ocfg, go, reward, cs, key=key)
+    _, out = TL.run_group_gpu(ctx, TL.lib_cfg(ocfg, "bf16"), st)
+    TL.check_group(out, ref, R, P)
+    assert ctx.last_status() == 0
 
 
 def test_group_stats_empty_inputs_and_status_bits(ctx):

@@ -39,15 +39,21 @@ def test_splitmix64_published_vectors():
 
 @pytest.mark.parametrize("row", _rows("paper_worked_counts.txt"))
 def test_paper_kept_counts(row):
-    n, c, k, up, rej, expected = (int(v) for v in row)
-    cfg = O.Cfg(uniform_policy=up, rejection=rej, k_ratio=k, seed=7)
+    n, c, k, up, rej, expected = (int(v) for v in row[:6])
+    high = int(row[6]) if len(row) > 6 else 0
+    cfg = O.Cfg(uniform_policy=up, rejection=rej, k_ratio=k, reject_high=high, seed=7)
     go, reward, cs = _one_group(n, c)
     out = O.group_stats(cfg, go, reward, cs)
     assert int(out["keep"].sum()) == expected
     assert int(out["counters"][0]) == expected
-    # every correct rollout of a mixed group survives (Sec. 4.2 Strategy 3)
-    if 0 < c < n:
+    if 0 < c < n and not high:
+        # every correct rollout of a mixed group survives (Sec. 4.2 Strategy 3)
         assert out["keep"][:c].all()
+    if 0 < c < n and high and 2 * c >= n:
+        # the ablation keeps every incorrect rollout and as many correct ones: advantages are +-1
+        assert out["keep"][c:].all() and int(out["keep"][:c].sum()) == min(k * (n - c), c)
+        if k == 1 and n - c <= c:
+            assert np.allclose(np.abs(out["adv"][out["keep"] != 0]), 1.0, atol=1e-5)
 
 
 @pytest.mark.parametrize("row", _rows("paper_posterior.txt"))
@@ -274,3 +280,30 @@ def test_empty_group_and_empty_batch():
     assert out["u_tilde"][0] == pytest.approx(0.5)
     out = O.group_stats(O.Cfg(), np.array([0], np.int32), np.zeros(0, np.float32), np.array([0], np.int64))
     assert out["counters"][0] == 0 and out["counters"][1] == 0
+
+
+def test_high_success_downsampling_brute_force():
+    """reject_high: which correct rollouts survive, against a plain sort; low-success groups and
+    uniform groups are untouched by the switch."""
+    rng = np.random.default_rng(11)
+    for _ in range(40):
+        n = int(rng.integers(2, 14))
+        c = int(rng.integers(0, n + 1))
+        reward = np.zeros(n, np.float32)
+        reward[rng.permutation(n)[:c]] = 1.0
+        key = rng.integers(0, 5, n).astype(np.uint32)          # few distinct keys: ties by index matter
+        go = np.array([0, n], np.int32)
+        cs = np.arange(n + 1, dtype=np.int64) * 2
+        k = int(rng.integers(1, 3))
+        base = O.group_stats(O.Cfg(uniform_policy=O.UNIFORM_BAYES, rejection=1, k_ratio=k), go, reward, cs, key=key)
+        out = O.group_stats(O.Cfg(uniform_policy=O.UNIFORM_BAYES, rejection=1, k_ratio=k, reject_high=1), go, reward,
+                            cs, key=key)
+        if c == 0 or c == n or 2 * c < n:
+            assert np.array_equal(out["keep"], base["keep"])
+            continue
+        m = min(k * (n - c), c)
+        corr = sorted([i for i in range(n) if reward[i] > 0.5], key=lambda i: (int(key[i]), i))[:m]
+        expect = np.zeros(n, np.uint8)
+        expect[corr] = 1
+        expect[reward < 0.5] = 1
+        assert np.array_equal(out["keep"], expect)
