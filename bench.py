@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-group-leg", action="store_true")
+    ap.add_argument("--no-variants-leg", action="store_true",
+                    help="skip the timings of the regularised step (KL + entropy) and of the log-prob pass alone")
     ap.add_argument("--only-group-leg", action="store_true",
                     help="run only the large-input group-stage measurement (for profiling that stage alone)")
     return ap.parse_args()
@@ -232,10 +234,8 @@ def run_ours(args):
     chunk = min(args.chunk_tokens, (T + 127) // 128 * 128)
     ws_b = torch.empty(ctx.bwd_workspace_bytes(T, wl.d, wl.V, R, chunk), dtype=torch.uint8, device=dev)
 
-    # old log-probs: the current policy's own log-probs plus seeded noise (a first forward pass)
-    g0 = ctx.group_stats(cfg, go, reward, cs, key=key, alpha_in=alpha, beta_in=beta, out=gbuf)
-    all_keep = torch.ones(R, dtype=torch.uint8, device=dev)
-    f0 = ctx.grpo_loss_fwd(cfg, H, W, y, torch.zeros(T, device=dev), cs, g0["adv"], g0["w"], all_keep)
+    # old log-probs: the current policy's own log-probs (the log-prob pass alone) plus seeded noise
+    f0 = ctx.logprob_fwd(cfg, H, W, y)
     old = (f0["logp"][:T] + noise).contiguous()
     del f0
 
@@ -302,6 +302,8 @@ def run_ours(args):
         "roofline": roofline,
     }
 
+    if rank == 0 and world == 1 and not args.no_variants_leg:
+        line["variants"] = variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, gbuf, dH, dW, ws_b, T_kept, pk)
     if rank == 0 and world == 1 and not args.no_group_leg:
         line["group_stage"] = group_stage_leg(ctx, pk, dev)
     if rank == 0 and not args.no_e2e:
@@ -312,6 +314,44 @@ def run_ours(args):
     if rank == 0:
         print(json.dumps(line), flush=True)
     D.barrier()
+
+
+def variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, g, dH, dW, ws_b, T_kept, pk):
+    """The step with Eq. 2's KL term and the entropy bonus (aero_grpo_loss_reg_fwd/_bwd), and the
+    log-prob pass alone (aero_logprob_fwd) that produces old / reference log-probs."""
+    import copy
+    import torch
+
+    T = H.shape[0]
+    rcfg = copy.copy(cfg)
+    rcfg.kl_beta, rcfg.ent_coef = 0.04, 1e-3
+    ref = (old + 0.5 * noise).contiguous()
+    fb, lb = {}, {}
+
+    def timed(fn, n=3):
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    def reg_step():
+        f = ctx.grpo_loss_reg_fwd(rcfg, H, W, y, old, ref, cs, g["adv"], g["w"], g["keep"], out=fb)
+        ctx.grpo_loss_reg_bwd(rcfg, H, W, y, cs, g["keep"], f["lse"], f["g"], f["entropy"], g["w"], dH=dH, dW=dW,
+                              workspace=ws_b)
+
+    ms_reg = timed(reg_step)
+    ms_lp = timed(lambda: ctx.logprob_fwd(rcfg, H, W, y, out=lb))
+    fl = 2.0 * wl.d * wl.V
+    return {"regularised_step": {"kl_beta": 0.04, "ent_coef": 1e-3, "ms": ms_reg, "tokens_per_s": T_kept / (ms_reg * 1e-3),
+                                 "executed_tflops": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12,
+                                 "frac_of_sustained": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12 / pk["sustained"]},
+            "logprob_pass": {"rows": T, "ms": ms_lp, "tokens_per_s": T / (ms_lp * 1e-3),
+                             "tflops": fl * T / (ms_lp * 1e-3) / 1e12, "frac_of_burst": fl * T / (ms_lp * 1e-3) / 1e12 / pk["burst"]}}
 
 
 def group_stage_leg(ctx, pk, dev):
