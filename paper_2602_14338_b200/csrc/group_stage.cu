@@ -666,20 +666,22 @@ __global__ void __launch_bounds__(kThreads, 4) curate_kernel(Args a, Workspace w
   if (tile < ntiles) {
     const int p0 = tile * pt;
     const int npt = min(pt, a.P - p0);
-    // rollout range of the tile and of each of its prompts (clamped if the offsets are bad)
+    // rollout range of the tile and of each of its prompts (clamped if the offsets are bad), later made
+    // relative to the tile's first rollout
     for (int q = tid; q <= npt; q += kThreads) {
       int v = a.go[p0 + q];
       const int prev = q > 0 ? a.go[p0 + q - 1] : v;
       if (v < 0 || v > a.R || v < prev) st |= AERO_ST_BAD_OFFSETS;
       sh.ps.lo[q] = min(max(v, 0), a.R);
     }
-    __syncthreads();
-    if (tid == 0) {
-      // make the ranges non-decreasing, then relative to the tile's first rollout
-      int run = sh.ps.lo[0];
-      for (int q = 1; q <= npt; ++q) { run = max(run, sh.ps.lo[q]); sh.ps.lo[q] = run; }
+    // bad offsets only: make the ranges non-decreasing (serial, so kept off the normal path)
+    if (__syncthreads_or((st & AERO_ST_BAD_OFFSETS) != 0)) {
+      if (tid == 0) {
+        int run = sh.ps.lo[0];
+        for (int q = 1; q <= npt; ++q) { run = max(run, sh.ps.lo[q]); sh.ps.lo[q] = run; }
+      }
+      __syncthreads();
     }
-    __syncthreads();
     const int r0 = sh.ps.lo[0];
     const int nroll = sh.ps.lo[npt] - r0;
     __syncthreads();
