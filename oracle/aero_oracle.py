@@ -418,3 +418,93 @@ def grpo_loss_reg_bwd(cfg: Cfg, H, W, y, cs, keep, lse, g, entropy, w, grad_scal
         dH[idx] = dz @ W
         dW = dz[:, rows].T @ H[idx]
     return dH, dW
+
+
+# ----------------------------------------------------------------------------
+# rollout allocation controller of one training step, simulated on prompts with
+# hidden success rates (Algorithm 1; Sec. 4.2 Strategy 1; Appendix C "AERO")
+# ----------------------------------------------------------------------------
+@dataclasses.dataclass
+class AllocCfg:
+    n_extra: int = 2       # rescue increment Delta n (Strategy 1: "n_extra, e.g., 2"; Appendix C: Delta n = 2)
+    k_max: int = 10        # Appendix C: up to K_max = 10 iterations
+    n_max: int = 32        # Appendix C: n_p <= n_max = 32
+    n_budget: int = 16     # Appendix C: sum_p n_p <= n_budget * |P|
+
+
+def curated_size(cfg: Cfg, n: int, c: int) -> int:
+    """Number of rollouts the curation rule of group_stats keeps from a group with n rollouts, c correct."""
+    if n == 0:
+        return 0
+    if c == 0 or c == n:
+        if cfg.uniform_policy == UNIFORM_MASK:
+            return 0
+        return n if cfg.n_keep_uniform <= 0 else min(cfg.n_keep_uniform, n)
+    low = (2 * c < n) or (cfg.rescue_S > 0 and c * cfg.n_explore <= cfg.rescue_S * n)
+    if cfg.rejection and low:
+        return c + min(cfg.k_ratio * c, n - c)
+    if cfg.rejection and cfg.reject_high:
+        return (n - c) + min(cfg.k_ratio * (n - c), c)
+    return n
+
+
+def allocate_sim(cfg: Cfg, acfg: AllocCfg, thr):
+    """One step of the allocation controller over P simulated prompts.
+
+    Rollout j (in generation order) of prompt p is correct iff the draw
+    default_key(cfg.seed, p * n_max + j) < thr[p]; thr[p] = floor(u_p * 2^32) encodes the
+    hidden success rate u_p.  Steps:
+      1. exploration: n_explore rollouts per prompt, c_p correct        [Algorithm 1, Stage 1]
+      2. rescue set: c_p <= rescue_S.  For up to k_max iterations every prompt still in the
+         set asks for min(n_extra, n_max - n_p) more rollouts (asking for none leaves the
+         set); requests are granted in prompt order while their running sum stays within the
+         budget left of n_budget * P; a granted prompt draws its rollouts and leaves the set
+         as soon as one of them is correct ("early exit upon first success")
+                                                [Sec. 4.2 Strategy 1; Appendix C items 2-3]
+      3. curated training size per prompt by the rule of group_stats        [Sec. 4.4]
+    The paper does not say how a short budget is shared: prompt order is a reading.
+    Returns n_gen, c, n_train per prompt and counters
+    [rollouts generated, rollouts kept for training, zero-accuracy prompts after exploration,
+     zero-accuracy prompts at the end, prompts rescued, iterations run, budget left, P]."""
+    thr = np.asarray(thr, dtype=np.uint64)
+    P = len(thr)
+    n = np.full(P, cfg.n_explore, dtype=np.int64)
+    c = np.zeros(P, dtype=np.int64)
+    for p in range(P):
+        for j in range(cfg.n_explore):
+            c[p] += 1 if default_key(cfg.seed, p * acfg.n_max + j) < int(thr[p]) else 0
+    zero_before = int((c == 0).sum())
+    rescue = c <= cfg.rescue_S
+    rescued = np.zeros(P, dtype=bool)          # left the rescue set by drawing a correct rollout
+    remaining = max(acfg.n_budget * P - cfg.n_explore * P, 0)
+    iters = 0
+    for _ in range(acfg.k_max):
+        running = 0
+        granted_any = False
+        for p in range(P):
+            if not rescue[p]:
+                continue
+            req = min(acfg.n_extra, acfg.n_max - int(n[p]))
+            if req <= 0:
+                rescue[p] = False
+                continue
+            running += req
+            if running > remaining:
+                continue                      # not granted this iteration; stays in the set
+            granted_any = True
+            new_c = 0
+            for j in range(int(n[p]), int(n[p]) + req):
+                new_c += 1 if default_key(cfg.seed, p * acfg.n_max + j) < int(thr[p]) else 0
+            n[p] += req
+            c[p] += new_c
+            if new_c > 0:
+                rescue[p] = False
+                rescued[p] = True
+        if not granted_any:
+            break
+        iters += 1
+        remaining = acfg.n_budget * P - int(n.sum())
+    n_train = np.array([curated_size(cfg, int(n[p]), int(c[p])) for p in range(P)], dtype=np.int64)
+    counters = np.array([int(n.sum()), int(n_train.sum()), zero_before, int((c == 0).sum()), int(rescued.sum()), iters,
+                         acfg.n_budget * P - int(n.sum()), P], dtype=np.int64)
+    return dict(n_gen=n.astype(np.int32), c=c.astype(np.int32), n_train=n_train.astype(np.int32), counters=counters)
