@@ -346,8 +346,21 @@ def variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, g, dH, dW, ws_b, T_kept,
 
     ms_reg = timed(reg_step)
     ms_lp = timed(lambda: ctx.logprob_fwd(rcfg, H, W, y, out=lb))
+    # allocation controller on 2^22 simulated prompts with success rates ~ Beta(0.5, 0.5)
+    from paper_2602_14338_b200 import binding as B
+    from paper_2602_14338_b200 import synth
+    Pn = 1 << 22
+    thr = torch.from_numpy(synth.success_thresholds(Pn, 0.5, 0.5, seed=4301).view(np.int32)).to(H.device)
+    acfg = B.cfg_default(uniform_policy=B.AERO_UNIFORM_BAYES, rejection=1, k_ratio=1, seed=4302)
+    ab = {}
+    ms_alloc = timed(lambda: ctx.allocate_sim(acfg, B.alloc_cfg_default(), thr, out=ab), n=5)
+    cnt = ab["counters"].cpu().tolist()
     fl = 2.0 * wl.d * wl.V
-    return {"regularised_step": {"kl_beta": 0.04, "ent_coef": 1e-3, "ms": ms_reg, "tokens_per_s": T_kept / (ms_reg * 1e-3),
+    return {"allocation_sim": {"prompts": Pn, "ms": ms_alloc, "prompts_per_s": Pn / (ms_alloc * 1e-3),
+                               "launches": 23, "mean_rollouts_generated": cnt[0] / Pn, "mean_rollouts_trained": cnt[1] / Pn,
+                               "zero_accuracy_before": cnt[2] / Pn, "zero_accuracy_after": cnt[3] / Pn,
+                               "iterations": cnt[5]},
+            "regularised_step": {"kl_beta": 0.04, "ent_coef": 1e-3, "ms": ms_reg, "tokens_per_s": T_kept / (ms_reg * 1e-3),
                                  "executed_tflops": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12,
                                  "frac_of_sustained": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12 / pk["sustained"]},
             "logprob_pass": {"rows": T, "ms": ms_lp, "tokens_per_s": T / (ms_lp * 1e-3),

@@ -354,6 +354,42 @@ int aero_grpo_step_host(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R
                         float* loss_h, int64_t* counters_h, float* metrics_h,
                         void* workspace, size_t workspace_bytes);
 
+/* ------------------------------------------------------------------------------
+ * Rollout allocation controller of one training step, simulated on P prompts with hidden
+ * success rates (Algorithm 1; Sec. 4.2 Strategy 1; Appendix C "AERO": categorisation,
+ * iterative rejection sampling with increment 2 for at most 10 iterations, n_p <= 32,
+ * sum_p n_p <= 16 |P|).  No language model is involved: rollout j (in generation order) of
+ * prompt p is correct iff the draw -- the high 32 bits of SplitMix64 applied to
+ * cfg->seed + (p * n_max + j + 1) * 0x9E3779B97F4A7C15 -- is below thr[p]
+ * (thr[p] = floor(u_p * 2^32) for success rate u_p).
+ *   1. exploration: cfg->n_explore rollouts per prompt, c_p of them correct;
+ *   2. rescue set: c_p <= cfg->rescue_S.  In each of up to k_max iterations every prompt
+ *      still in the set asks for min(n_extra, n_max - n_p) more rollouts (asking for none
+ *      leaves the set); requests are granted in prompt order while their running sum stays
+ *      within what is left of n_budget * P (the paper does not say how a short budget is
+ *      shared); a granted prompt draws its rollouts and leaves the set as soon as one is
+ *      correct;
+ *   3. n_train[p]: the number of rollouts the curation rule of aero_group_stats keeps from
+ *      a group with n_p rollouts of which c_p are correct.
+ * Inputs   thr [P] u32.   Outputs  n_gen, c, n_train [P] i32; counters [8] i64: rollouts
+ *          generated, rollouts kept for training, zero-accuracy prompts after exploration,
+ *          zero-accuracy prompts at the end, prompts rescued, iterations that granted
+ *          anything, budget left, P.  All outputs are integers and exact.
+ * workspace: at least aero_allocate_workspace_bytes(P) bytes, 256-byte aligned.
+ */
+typedef struct aero_alloc_cfg {
+  int32_t n_extra;    /* rescue increment (Strategy 1 "n_extra, e.g., 2")        default 2  */
+  int32_t k_max;      /* iterations (Appendix C)                                  default 10 */
+  int32_t n_max;      /* per-prompt cap (Appendix C)                              default 32 */
+  int32_t n_budget;   /* mean rollouts per prompt the step may spend (Appendix C) default 16 */
+} aero_alloc_cfg;
+
+void aero_alloc_cfg_default(aero_alloc_cfg* ac);
+size_t aero_allocate_workspace_bytes(int32_t P);
+int aero_allocate_sim(aero_ctx* ctx, const aero_cfg* cfg, const aero_alloc_cfg* ac, int32_t P, const uint32_t* thr,
+                      int32_t* n_gen, int32_t* c, int32_t* n_train, int64_t* counters,
+                      void* workspace, size_t workspace_bytes);
+
 /* Number of kernels the library has launched through this context since it was created
  * (copies and memsets are not counted).  Host-side counter, no synchronisation. */
 int64_t aero_launch_count(aero_ctx* ctx);

@@ -28,6 +28,7 @@ EXPORTS = [
     "aero_fwd_workspace_bytes", "aero_grpo_loss_fwd", "aero_bwd_workspace_bytes", "aero_grpo_loss_bwd",
     "aero_step_workspace_bytes", "aero_grpo_step_host", "aero_launch_count", "aero_group_stats_static",
     "aero_grpo_loss_reg_fwd", "aero_grpo_loss_reg_bwd", "aero_logprob_fwd",
+    "aero_alloc_cfg_default", "aero_allocate_workspace_bytes", "aero_allocate_sim",
 ]
 
 
@@ -41,6 +42,10 @@ class AeroCfg(C.Structure):
         ("seed", C.c_uint64), ("dtype", C.c_int32), ("reject_high", C.c_int32),
         ("kl_beta", C.c_float), ("ent_coef", C.c_float),
     ]
+
+
+class AeroAllocCfg(C.Structure):
+    _fields_ = [("n_extra", C.c_int32), ("k_max", C.c_int32), ("n_max", C.c_int32), ("n_budget", C.c_int32)]
 
 
 class AeroError(RuntimeError):
@@ -84,6 +89,11 @@ def load_library():
     lib.aero_grpo_loss_reg_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 9 + [f32] +
                                            [vp, vp, C.c_int, vp, sz])
     lib.aero_logprob_fwd.argtypes = [vp, C.POINTER(AeroCfg), i64, i32, i32] + [vp] * 6 + [vp, sz]
+    lib.aero_alloc_cfg_default.restype = None
+    lib.aero_alloc_cfg_default.argtypes = [C.POINTER(AeroAllocCfg)]
+    lib.aero_allocate_workspace_bytes.restype = sz
+    lib.aero_allocate_workspace_bytes.argtypes = [i32]
+    lib.aero_allocate_sim.argtypes = [vp, C.POINTER(AeroCfg), C.POINTER(AeroAllocCfg), i32] + [vp] * 5 + [vp, sz]
     lib.aero_step_workspace_bytes.restype = sz
     lib.aero_step_workspace_bytes.argtypes = [i32, i32, i64, i32, i32, i64, i32]
     lib.aero_grpo_step_host.argtypes = ([vp, C.POINTER(AeroCfg), i32, i32, i64, i32, i32] + [vp] * 12 + [C.c_int] +
@@ -108,6 +118,16 @@ def cfg_default(**over) -> AeroCfg:
             raise AttributeError(k)
         setattr(cfg, k, v)
     return cfg
+
+
+def alloc_cfg_default(**over) -> AeroAllocCfg:
+    ac = AeroAllocCfg()
+    load_library().aero_alloc_cfg_default(C.byref(ac))
+    for k, v in over.items():
+        if not hasattr(ac, k):
+            raise AttributeError(k)
+        setattr(ac, k, v)
+    return ac
 
 
 def _ptr(t, dtype=None, numel=None, name="tensor"):
@@ -352,6 +372,26 @@ class Context:
             workspace.data_ptr(), workspace.numel())
         _check(rc, "aero_grpo_loss_bwd")
         return dH, dW
+
+    # ---- allocation controller, simulated ----------------------------------------------------
+    def allocate_sim(self, cfg, acfg, thr, out=None):
+        """aero_allocate_sim: thr is a 32-bit integer CUDA tensor (bits read as unsigned) of per-prompt
+        success thresholds; returns n_gen, c, n_train [P] int32 and counters [8] int64."""
+        P = thr.numel()
+        if thr.dtype not in (torch.int32, torch.uint32):
+            raise AeroError("thr must be a 32-bit integer tensor (its bits are read as unsigned)")
+        o = out if out is not None else {}
+        for name in ("n_gen", "c", "n_train"):
+            if name not in o:
+                o[name] = torch.empty(max(P, 1), dtype=torch.int32, device=self.device)
+        if "counters" not in o:
+            o["counters"] = torch.zeros(8, dtype=torch.int64, device=self.device)
+        ws = self.workspace(self.lib.aero_allocate_workspace_bytes(P))
+        rc = self.lib.aero_allocate_sim(self.h, C.byref(cfg), C.byref(acfg), P, _ptr(thr, None, P, "thr"),
+                                        _ptr(o["n_gen"]), _ptr(o["c"]), _ptr(o["n_train"]), _ptr(o["counters"]),
+                                        ws.data_ptr(), ws.numel())
+        _check(rc, "aero_allocate_sim")
+        return o
 
     # ---- whole step from host buffers ---------------------------------------------------
     def launch_count(self) -> int:

@@ -120,3 +120,11 @@ def peak_hidden(H, W, y, strength: float):
     Wy = W[torch.as_tensor(y, device=W.device).long()].float()
     Wy = Wy / Wy.norm(dim=1, keepdim=True).clamp_min(1e-12)
     return (strength * Wy + 0.25 * H.float()).to(H.dtype)
+
+
+def success_thresholds(P: int, beta_a: float, beta_b: float, seed: int) -> np.ndarray:
+    """Hidden per-prompt success rates u ~ Beta(beta_a, beta_b) as 32-bit thresholds floor(u * 2^32)
+    (inputs of the allocation-controller simulation; a draw below the threshold is a correct rollout)."""
+    rng = np.random.default_rng(seed)
+    u = rng.beta(beta_a, beta_b, size=P)
+    return np.minimum(np.floor(u * 2.0 ** 32), 2.0 ** 32 - 1).astype(np.uint32)

@@ -144,6 +144,55 @@ def test_group_stats_large_properties(ctx):
         assert g["cat"][p] == ref["cat"][0]
 
 
+# ------------------------------------------------------------------ allocation controller (simulated)
+ALLOC_CASES = [
+    # P, Beta(a, b) of the hidden success rates, cfg overrides, alloc overrides
+    (1000, 0.5, 0.5, dict(uniform_policy=O.UNIFORM_BAYES, rejection=1), dict()),
+    (777, 0.3, 2.0, dict(uniform_policy=O.UNIFORM_BAYES, rejection=1, k_ratio=2), dict(n_budget=10)),       # budget binds
+    (513, 0.4, 1.5, dict(rejection=1, reject_high=1, rescue_S=2), dict(n_extra=3, k_max=4, n_max=17)),
+    (300, 5.0, 0.2, dict(uniform_policy=O.UNIFORM_BAYES), dict(k_max=0)),
+    (257, 0.05, 5.0, dict(uniform_policy=O.UNIFORM_BAYES, rejection=1, n_explore=4), dict(n_budget=5, n_extra=1)),
+]
+
+
+@pytest.mark.parametrize("case", range(len(ALLOC_CASES)))
+def test_allocation_controller_matches_oracle(ctx, case):
+    P, ba, bb, cover, aover = ALLOC_CASES[case]
+    thr = synth.success_thresholds(P, ba, bb, seed=600 + case)
+    ocfg = O.Cfg(seed=900 + case, **cover)
+    oa = O.AllocCfg(**aover)
+    ref = O.allocate_sim(ocfg, oa, thr)
+    out = ctx.allocate_sim(TL.lib_cfg(ocfg, "bf16"), B.alloc_cfg_default(**aover), TL.dev(thr.view(np.int32)))
+    for k in ("n_gen", "c", "n_train"):
+        assert np.array_equal(out[k][:P].cpu().numpy(), ref[k]), k
+    assert out["counters"].cpu().tolist() == ref["counters"].tolist()
+    if case == 1:
+        assert ref["counters"][6] < 2                 # the budget really ran out
+    assert ctx.last_status() == 0
+
+
+def test_allocation_controller_large_properties(ctx):
+    """2^20 prompts: budget and cap invariants, and the geometric closed forms of the rescue process."""
+    P, u = 1 << 20, 0.12
+    thr = np.full(P, int(u * 2 ** 32), np.uint32)
+    ocfg = O.Cfg(seed=77, uniform_policy=O.UNIFORM_BAYES, rejection=1)
+    out = ctx.allocate_sim(TL.lib_cfg(ocfg, "bf16"), B.alloc_cfg_default(), TL.dev(thr.view(np.int32)))
+    n, c, nt = (out[k][:P].cpu().numpy().astype(np.int64) for k in ("n_gen", "c", "n_train"))
+    cnt = out["counters"].cpu().numpy()
+    assert n.min() >= 8 and n.max() <= 32 and n.sum() <= 16 * P and (nt <= n).all()
+    assert cnt[0] == n.sum() and cnt[1] == nt.sum() and cnt[3] == (c == 0).sum() and cnt[6] == 16 * P - n.sum()
+    p0 = (1 - u) ** 8
+    assert abs(cnt[2] / P - p0) < 5 * np.sqrt(p0 * (1 - p0) / P)
+    pr = 1 - (1 - u) ** 20
+    assert abs(cnt[4] / cnt[2] - pr) < 5 * np.sqrt(pr * (1 - pr) / cnt[2])
+    sample = np.random.default_rng(1).integers(0, P, 300)
+    for p in sample:                                   # sampled prompts, draw by draw
+        draws = [O.default_key(ocfg.seed, int(p) * 32 + j) < int(thr[p]) for j in range(int(n[p]))]
+        assert sum(draws) == c[p] and nt[p] == O.curated_size(ocfg, int(n[p]), int(c[p]))
+        if n[p] > 8:
+            assert not any(draws[:int(n[p]) - 2])
+
+
 # ------------------------------------------------------------------ stage (b)
 def run_fwd_bwd(ctx, batch, dtype, grad_scale=1.0, chunk_tokens=None):
     cfg = TL.lib_cfg(batch.ocfg, dtype)
