@@ -42,7 +42,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1, help="workload index 0..4")
-    ap.add_argument("--chunk-tokens", type=int, default=2 * 148 * 128)
+    ap.add_argument("--chunk-tokens", type=int, default=4 * 148 * 128)
     ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (reduced runs for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -355,11 +355,23 @@ def variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, g, dH, dW, ws_b, T_kept,
     ab = {}
     ms_alloc = timed(lambda: ctx.allocate_sim(acfg, B.alloc_cfg_default(), thr, out=ab), n=5)
     cnt = ab["counters"].cpu().tolist()
+    # down-sampling ratio k = 1..4 on the AERO-curated batch (workload 3): what the backward has to process
+    st3 = synth.make_structure(synth.WORKLOADS[3])
+    t3 = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(H.device)
+    go3, rw3, cs3, key3 = t3(st3.go), t3(st3.reward), t3(st3.cs), t3(st3.key.view(np.int32))
+    al3, be3 = t3(st3.alpha), t3(st3.beta)
+    ksweep = {}
+    for k in (1, 2, 3, 4):
+        kc = B.cfg_default(uniform_policy=B.AERO_UNIFORM_BAYES, rejection=1, k_ratio=k, seed=synth.WORKLOADS[3].seed)
+        gk = ctx.group_stats(kc, go3, rw3, cs3, key=key3, alpha_in=al3, beta_in=be3)
+        ck = gk["counters"].cpu().tolist()
+        ksweep[str(k)] = {"kept_rollouts": ck[0], "kept_tokens": ck[1], "kept_token_fraction": ck[1] / max(ck[7], 1)}
     fl = 2.0 * wl.d * wl.V
     return {"allocation_sim": {"prompts": Pn, "ms": ms_alloc, "prompts_per_s": Pn / (ms_alloc * 1e-3),
                                "launches": 23, "mean_rollouts_generated": cnt[0] / Pn, "mean_rollouts_trained": cnt[1] / Pn,
                                "zero_accuracy_before": cnt[2] / Pn, "zero_accuracy_after": cnt[3] / Pn,
                                "iterations": cnt[5]},
+            "k_ratio_sweep_workload3": ksweep,
             "regularised_step": {"kl_beta": 0.04, "ent_coef": 1e-3, "ms": ms_reg, "tokens_per_s": T_kept / (ms_reg * 1e-3),
                                  "executed_tflops": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12,
                                  "frac_of_sustained": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12 / pk["sustained"]},

@@ -519,7 +519,7 @@ def test_full_size_workload_in_bench_configuration(ctx, config):
 
     y, cs, oldd = TL.dev(st.y), TL.dev(st.cs), TL.dev(old)
     f = ctx.grpo_loss_fwd(cfg, H, W, y, oldd, cs, g["adv"], g["w"], g["keep"])
-    chunk = 2 * 148 * 128
+    chunk = 4 * 148 * 128
     ws = torch.empty(ctx.bwd_workspace_bytes(T, wl.d, wl.V, R, chunk), dtype=torch.uint8, device="cuda")
     dH, dW = ctx.grpo_loss_bwd(cfg, H, W, y, cs, g["keep"], f["lse"], f["g"], workspace=ws)
     torch.cuda.synchronize()
