@@ -130,8 +130,8 @@ int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
 }
 
 size_t aero_fwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R) {
-  (void)d; (void)V;
-  size_t a = aero_fwd_ws_bytes_fp32(T, R), b = aero_fwd_ws_bytes_tc(T, R);
+  (void)V;
+  size_t a = aero_fwd_ws_bytes_fp32(T, R), b = aero_fwd_ws_bytes_tc(T, d, R);
   return a > b ? a : b;
 }
 

@@ -6,6 +6,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <stdlib.h>
 
 #include "../../include/aero.h"
 
@@ -88,7 +89,25 @@ int aero_bwd_fp32(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int3
                   const aero_bwd_extra& ex);
 
 // ---- stage (b): tcgen05 / TMEM / TMA path (bf16) -------------------------------------
-size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t R);
+// Number of CTA pairs that share a pair of token tiles and split the vocabulary between them:
+// the smallest power of two that brings the H tiles all 148 CTAs keep re-reading from L2
+// (148 * 128 * d * 2 bytes) under 72 MB, a bit over half of the 126 MB L2.
+static inline int aero_vsplit(int32_t d) {
+  if (const char* e = getenv("AERO_VSPLIT")) {          // override for tests and tuning: 1, 2, 4 or 8
+    const int v = atoi(e);
+    if (v == 1 || v == 2 || v == 4 || v == 8) return v;
+  }
+  const double live = 148.0 * 128.0 * (double)d * 2.0;
+  int s = 1;
+  while (live / s > 72.0 * 1024 * 1024 && s < 8) s *= 2;
+  return s;
+}
+// Meeting points per unit of the lm_head kernel's producers (0 switches the pacing off).
+static inline int aero_nsync() {
+  if (const char* e = getenv("AERO_NSYNC")) return atoi(e) > 0 ? atoi(e) : 0;
+  return 8;
+}
+size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t d, int32_t R);
 int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                 const void* H, const void* W, const int32_t* y, const float* old_logp,
                 const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,

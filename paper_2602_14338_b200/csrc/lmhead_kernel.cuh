@@ -63,6 +63,19 @@ struct Params {
   int tile_begin, tile_end;     // this launch covers tiles [tile_begin, min(tile_end, *n_tiles))
   const int32_t* y;
   uint32_t* status;
+  // Vocabulary split: `vsplit` CTA pairs share a pair of token tiles and walk 1/vsplit of the
+  // vocabulary tiles each, so that the H tiles all CTAs re-read from L2 (148 * 128 * d * 2 bytes,
+  // 136 MB at d = 3584) shrink to what L2 holds.  Forward modes then leave the per-row running
+  // state in xstate [vsplit][T] for merge_kernel instead of finishing the row.
+  int vsplit;
+  float4* xstate;
+  // Pacing: all CTAs re-read the same W tiles from L2, which only works while they walk the
+  // vocabulary in step; small rate differences between SMs add up over a long launch.  The
+  // producers therefore meet at `nsync` points per unit on a counter in global memory
+  // (zeroed before the launch).  The wait is short and bounded: a CTA that is not there in time
+  // is simply not waited for.
+  unsigned int* sync_ctr;
+  int nsync;
   const int64_t* cs;
   const float* w;
   float ent_coef;
@@ -94,6 +107,78 @@ __device__ __forceinline__ float ex2(float x) {
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// End of a token row in the forward modes: log-sum-exp, log-prob, entropy, then Eq. 2 (with the
+// KL term when a reference is given) and the warp's record of loss partials.  Called by the four
+// epilogue warps of a tile (warp = 0..3), with the merged running state of the row.
+__device__ __forceinline__ void finish_rows(const Params& p, bool ent_mode, bool live, long long row, int tile, int warp,
+                                            int lane, float m2, float l, float zy, float sz) {
+  double part[kPartialStride] = {0.0, 0.0, 0.0, 0.0, 0.0};
+  if (live) {
+    const float ls = (m2 + __log2f(l)) * kLn2;
+    const float lp = zy - ls;
+    const float ent = ent_mode ? ls - sz / l : 0.f;       // H = lse - E_p[z]
+    p.logp[row] = lp;
+    p.lse_out[row] = ls;
+    if (ent_mode) p.ent_out[row] = ent;
+    if (p.old_logp != nullptr) {
+      const int i = aero_owner(p.cs, p.R, row);
+      const float old = p.old_logp[row];
+      const float wi = p.w[i];
+      const SurrogateOut so = aero_surrogate(lp, old, p.adv[i], wi, p.clip_lo, p.clip_hi);
+      float g = so.g;
+      float obj = so.s;                              // per-token objective: s - beta D + c_H H
+      if (p.ref_logp != nullptr) {
+        const float q = p.ref_logp[row] - lp;
+        const float eq = __expf(q);
+        obj -= p.kl_beta * (eq - q - 1.f);
+        g += p.kl_beta * wi * (1.f - eq);
+      }
+      if (ent_mode) obj += p.ent_coef * ent;
+      p.g_out[row] = g;
+      part[0] = (double)wi * (double)obj;
+      part[1] = so.clipped;
+      part[2] = so.rho;
+      part[3] = (double)old - (double)lp;
+      part[4] = 1.0;
+    }
+  }
+  // fixed-shape reduction: a shuffle tree per warp; the four warps' records are
+  // added later by the finalising kernel in a fixed order
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+    for (int k = 0; k < kPartialStride; ++k) part[k] += __shfl_xor_sync(0xffffffffu, part[k], o);
+  if (lane == 0)
+    for (int k = 0; k < kPartialStride; ++k) p.partials[((size_t)tile * 4 + warp) * kPartialStride + k] = part[k];
+}
+
+// Forward modes with a vocabulary split: one block of 128 threads per token tile merges the
+// vsplit running states of each row and finishes it.
+static __global__ void __launch_bounds__(BM) merge_kernel(const Params p, int ent_mode) {
+  const int n_tiles = min(*p.n_tiles, p.tile_end);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int tile = p.tile_begin + blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    const long long row = (long long)p.tile_row[tile] + threadIdx.x;
+    const bool valid_row = (int)threadIdx.x < p.tile_valid[tile] && row < p.T;
+    int yt = -1;
+    if (valid_row) yt = p.y[row];
+    const bool live = valid_row && yt >= 0 && yt < p.V;      // a bad target was reported by the lm_head kernel
+    float m2 = -INFINITY, l = 0.f, zy = 0.f, sz = 0.f;
+    if (live) {
+      for (int s = 0; s < p.vsplit; ++s) {
+        const float4 o = p.xstate[(size_t)s * p.T + row];
+        const float mm = fmaxf(m2, o.x);
+        const float sa = ex2(m2 - mm), sb = ex2(o.x - mm);
+        l = l * sa + o.y * sb;
+        sz = sz * sa + o.w * sb;
+        zy += o.z;
+        m2 = mm;
+      }
+    }
+    finish_rows(p, ent_mode != 0, live, row, tile, warp, lane, m2, l, zy, sz);
+  }
 }
 
 template <int MODE>
@@ -129,18 +214,38 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
   const int nkb = p.d / BK;
   const int nvt = (p.V + BN - 1) / BN;
   // The pair's k-th unit is token tiles first, first + 1 (the second may not exist: its CTA
-  // then stages the first tile's rows again and discards the result).
-  auto unit_first = [&](int k) { return p.tile_begin + 2 * (pair + k * npairs); };
+  // then stages the first tile's rows again and discards the result) and one of the vsplit
+  // ranges of vocabulary tiles; the pairs that share tiles are neighbours.
+  const int vsplit = p.vsplit;
+  auto unit_first = [&](int k) { return p.tile_begin + 2 * ((pair + k * npairs) / vsplit); };
+  auto unit_j0 = [&](int k) { return (int)((long long)((pair + k * npairs) % vsplit) * nvt / vsplit); };
+  auto unit_j1 = [&](int k) { return (int)((long long)((pair + k * npairs) % vsplit + 1) * nvt / vsplit); };
 
   if (warp == 4) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
+      unsigned int meetings = 0;
+      // every CTA takes part in the same number of meetings: units of the longest schedule x nsync
+      const int total_units = ((n_tiles - p.tile_begin + 1) / 2) * vsplit;
+      const int max_units = total_units > 0 ? (total_units + npairs - 1) / npairs : 0;
       for (int k = 0; ok && unit_first(k) < n_tiles; ++k) {
         const int mine = unit_first(k) + (int)rank;
         const int row0 = p.tile_row[mine < n_tiles ? mine : unit_first(k)];
-        for (int j = 0; ok && j < nvt; ++j) {
+        int next_meet = 0;
+        for (int j = unit_j0(k), j0 = j, j1 = unit_j1(k); ok && j < j1; ++j) {
+          if (p.nsync > 0 && next_meet < p.nsync && j - j0 >= (int)((long long)next_meet * (j1 - j0) / p.nsync)) {
+            ++next_meet;
+            ++meetings;
+            atomicAdd(p.sync_ctr, 1u);
+            const unsigned int target = meetings * gridDim.x;
+            const unsigned long long t0 = tc::globaltimer_ns();
+            while (*reinterpret_cast<volatile unsigned int*>(p.sync_ctr) < target) {
+              if (tc::globaltimer_ns() - t0 > 200000ull) break;       // 0.2 ms: go on alone
+              __nanosleep(200);
+            }
+          }
           for (int kb = 0; kb < nkb; ++kb, ++it) {
             const int s = it % STAGES;
             const uint32_t ph = (it / STAGES) & 1u;
@@ -152,7 +257,15 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
             tc::tma_load_2d_pair(a_s + A_BYTES, &tmW, kb * BK, j * BN + (int)rank * BNH, full0);
           }
         }
+        // a unit whose range has fewer vocabulary tiles than meeting points still counts them all
+        if (p.nsync > 0 && next_meet < p.nsync) {
+          atomicAdd(p.sync_ctr, (unsigned)(p.nsync - next_meet));
+          meetings += (unsigned)(p.nsync - next_meet);
+        }
       }
+      // out of units: stand in for the meetings the longest schedule still has
+      if (p.nsync > 0 && meetings < (unsigned)(max_units * p.nsync))
+        atomicAdd(p.sync_ctr, (unsigned)(max_units * p.nsync) - meetings);
     }
   } else if (warp == 5) {
     // ---------------- MMA issuer ----------------
@@ -161,7 +274,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
       uint32_t it = 0, at = 0;
       bool ok = true;
       for (int k = 0; ok && unit_first(k) < n_tiles; ++k) {
-        for (int j = 0; ok && j < nvt; ++j, ++at) {
+        for (int j = unit_j0(k), j1 = unit_j1(k); ok && j < j1; ++j, ++at) {
           const uint32_t buf = at & 1u, aph = (at >> 1) & 1u;
           if (!tc::mbar_wait(&ctl->tempty[buf], aph ^ 1u, abort_flag)) { ok = false; break; }
           tc::tc_fence_after();
@@ -218,7 +331,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
       }
       const int dz_row0 = (tile - p.tile_begin) * BM + warp * 32;   // first dz row of this warp
 
-      for (int j = 0; ok && j < nvt; ++j, ++at) {
+      for (int j = unit_j0(k), j1 = unit_j1(k); ok && j < j1; ++j, ++at) {
         const uint32_t buf = at & 1u, aph = (at >> 1) & 1u;
         // the TMEM loads below are warp-collective: take the decision for the whole warp
         if (!__all_sync(0xffffffffu, tc::mbar_wait(&ctl->tfull[buf], aph, abort_flag))) { ok = false; break; }
@@ -342,45 +455,11 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
       }
 
       if (!IS_DZ && ok && have_tile) {
-        double part[kPartialStride] = {0.0, 0.0, 0.0, 0.0, 0.0};
-        if (live) {
-          const float ls = (m2 + __log2f(l)) * kLn2;
-          const float lp = zy - ls;
-          const float ent = ENT ? ls - sz / l : 0.f;       // H = lse - E_p[z]
-          p.logp[row] = lp;
-          p.lse_out[row] = ls;
-          if (ENT) p.ent_out[row] = ent;
-          if (p.old_logp != nullptr) {
-            const int i = aero_owner(p.cs, p.R, row);
-            const float old = p.old_logp[row];
-            const float wi = p.w[i];
-            const SurrogateOut so = aero_surrogate(lp, old, p.adv[i], wi, p.clip_lo, p.clip_hi);
-            float g = so.g;
-            float obj = so.s;                              // per-token objective: s - beta D + c_H H
-            if (p.ref_logp != nullptr) {
-              const float q = p.ref_logp[row] - lp;
-              const float eq = __expf(q);
-              obj -= p.kl_beta * (eq - q - 1.f);
-              g += p.kl_beta * wi * (1.f - eq);
-            }
-            if (ENT) obj += p.ent_coef * ent;
-            p.g_out[row] = g;
-            part[0] = (double)wi * (double)obj;
-            part[1] = so.clipped;
-            part[2] = so.rho;
-            part[3] = (double)old - (double)lp;
-            part[4] = 1.0;
-          }
+        if (vsplit > 1) {
+          if (live) p.xstate[(size_t)((pair + k * npairs) % vsplit) * p.T + row] = make_float4(m2, l, zy, sz);
+        } else {
+          finish_rows(p, ENT, live, row, tile, warp, lane, m2, l, zy, sz);
         }
-        // fixed-shape reduction: a shuffle tree per warp; the four warps' records are
-        // added later by the finalising kernel in a fixed order
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1)
-#pragma unroll
-          for (int k = 0; k < kPartialStride; ++k) part[k] += __shfl_xor_sync(0xffffffffu, part[k], o);
-        if (lane == 0)
-          for (int k = 0; k < kPartialStride; ++k)
-            p.partials[((size_t)tile * 4 + warp) * kPartialStride + k] = part[k];
       }
     }
   }

@@ -31,7 +31,7 @@ size_t aero_bwd_ws_bytes_tc(int64_t T, int32_t d, int32_t V, int32_t R, int64_t 
   (void)d;
   if (chunk_tokens < 128) chunk_tokens = 128;
   const size_t rows = (size_t)((chunk_tokens + 127) / 128 * 128);
-  return aero_tiles_bytes(T, R, lmhead::BM) + aero_align_up(rows * (size_t)ldz_of(V) * 2, 256);
+  return aero_tiles_bytes(T, R, lmhead::BM) + 256 + aero_align_up(rows * (size_t)ldz_of(V) * 2, 256);
 }
 
 int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
@@ -44,7 +44,9 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
 
   const long long ldz = ldz_of(V);
   aero_tiles tiles = aero_carve_tiles(ws, T, R, lmhead::BM);
-  const size_t tiles_bytes = aero_tiles_bytes(T, R, lmhead::BM);
+  // tile list, then the pacing counter of the lm_head kernel, then the dz block
+  const size_t tiles_bytes = aero_tiles_bytes(T, R, lmhead::BM) + 256;
+  unsigned int* sync_ctr = reinterpret_cast<unsigned int*>(static_cast<char*>(ws) + tiles_bytes - 256);
   __nv_bfloat16* dz = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + tiles_bytes);
   long long tpc = (long long)((ws_bytes - tiles_bytes) / ((size_t)lmhead::BM * (size_t)ldz * 2));
   if (tpc < 1) return AERO_ERR_WORKSPACE;
@@ -94,8 +96,11 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     lp.y = y; lp.status = ctx->d_status;
     lp.lse_in = lse; lp.g_in = g; lp.grad_scale = grad_scale; lp.dz = dz; lp.ldz = ldz;
     lp.cs = cs; lp.w = ex.w; lp.ent_in = ex.entropy; lp.ent_coef = ex.ent_coef;
+    lp.vsplit = aero_vsplit(d);
+    lp.sync_ctr = sync_ctr; lp.nsync = aero_nsync();
+    AERO_CUDA_TRY(cudaMemsetAsync(sync_ctr, 0, 256, ctx->stream));
     const long long max_pairs = ctx->sm_count / 2 > 0 ? ctx->sm_count / 2 : 1;
-    const long long dz_pairs = (tpc + 1) / 2;
+    const long long dz_pairs = (tpc + 1) / 2 * lp.vsplit;
     const int grid_dz = 2 * (int)(dz_pairs < max_pairs ? dz_pairs : max_pairs);
     k_dz<<<grid_dz, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH_k, tmW_k, tmDZ_st, lp);
 

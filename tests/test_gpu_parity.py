@@ -293,6 +293,50 @@ def test_bf16_tensor_core_path(ctx, name):
         assert TL.rel_l2(dW2.cpu().numpy()[never_hit], rdW[never_hit]) < GRAD_L2
 
 
+@pytest.mark.parametrize("vsplit", ["2", "4"])
+def test_vocabulary_split_between_cta_pairs(ctx, vsplit, monkeypatch):
+    """At large d several CTA pairs share a token tile and split the vocabulary (running states merged by
+    a second kernel).  Forced here on small shapes: all forward modes and the backward against the
+    oracle, and bit-identical log-probs between a split and an unsplit run of the log-prob pass."""
+    over, cover, peak = BF16_CASES["peaked"]
+    wl = synth.scaled(synth.WORKLOADS[1], **over)
+    batch = TL.Batch(wl, O.Cfg(seed=wl.seed, kl_beta=0.1, ent_coef=0.2, **cover), peak=peak)
+    ocfg, rg = batch.ocfg, batch.ref_g
+    adv32 = rg["adv"].astype(np.float32).astype(np.float64)
+    w32 = rg["w"].astype(np.float32).astype(np.float64)
+    ref_lp = (batch.old + 0.2).astype(np.float32)
+    ref = O.grpo_loss_reg_fwd(ocfg, batch.H, batch.W, batch.st.y, batch.old, ref_lp, batch.st.cs, adv32, w32, rg["keep"])
+    rdH, rdW = O.grpo_loss_reg_bwd(ocfg, batch.H, batch.W, batch.st.y, batch.st.cs, rg["keep"], ref["lse"], ref["g"],
+                                   ref["entropy"], w32)
+    cfg = TL.lib_cfg(ocfg, "bf16")
+    dv = batch.to_device()
+    plain = ctx.logprob_fwd(cfg, dv["H"], dv["W"], dv["y"], entropy=True)
+    monkeypatch.setenv("AERO_VSPLIT", vsplit)
+    f = ctx.grpo_loss_reg_fwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], TL.dev(ref_lp), dv["cs"], dv["adv"], dv["w"],
+                              dv["keep"])
+    dH, dW = ctx.grpo_loss_reg_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], dv["keep"], f["lse"], f["g"], f["entropy"],
+                                   dv["w"])
+    f0 = ctx.grpo_loss_fwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"], dv["keep"])
+    split = ctx.logprob_fwd(cfg, dv["H"], dv["W"], dv["y"], entropy=True)
+    torch.cuda.synchronize()
+    monkeypatch.delenv("AERO_VSPLIT")
+    assert ctx.last_status() == 0
+    T = batch.T
+    assert np.abs(f["logp"][:T].cpu().numpy() - ref["logp"]).max() <= LOGP_ABS
+    assert np.abs(f["entropy"][:T].cpu().numpy() - ref["entropy"]).max() <= LOGP_ABS
+    assert abs(f["loss"].item() - ref["loss"]) <= LOSS_REL * abs(ref["loss"]) + 1e-7
+    rho = ref["rho"]
+    edge = (np.abs(rho - 1.2) < 1e-3) | (np.abs(rho - 0.8) < 1e-3)
+    assert TL.rel_l2(dH.float().cpu().numpy()[~edge], rdH[~edge]) < GRAD_L2
+    if not edge.any():
+        assert TL.rel_l2(dW.cpu().numpy(), rdW) < GRAD_L2
+    check_fwd(batch, f0, O.grpo_loss_fwd(O.Cfg(seed=wl.seed, **cover), batch.H, batch.W, batch.st.y, batch.old,
+                                          batch.st.cs, adv32, w32, rg["keep"]), LOGP_ABS, LOSS_REL, 2e-2)
+    # the split changes only the order in which a row's tiles are merged
+    assert np.abs((split["logp"][:T] - plain["logp"][:T]).cpu().numpy()).max() < 1e-5
+    assert np.abs((split["entropy"][:T] - plain["entropy"][:T]).cpu().numpy()).max() < 1e-4
+
+
 def test_bwd_chunking_and_accumulation(ctx):
     over, cover, _ = BF16_CASES["aero_dropped"]
     wl = synth.scaled(synth.WORKLOADS[1], **over)
