@@ -105,7 +105,7 @@ static inline int aero_vsplit(int32_t d) {
 // Meeting points per unit of the lm_head kernel's producers (0 switches the pacing off).
 static inline int aero_nsync() {
   if (const char* e = getenv("AERO_NSYNC")) return atoi(e) > 0 ? atoi(e) : 0;
-  return 8;
+  return 32;
 }
 size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t d, int32_t R);
 int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
