@@ -27,12 +27,10 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "rollout tokens/sec, fused GRPO logprob+loss fwd+bwd"
-# dram__bytes_read.sum + dram__bytes_write.sum of one lmhead_kernel<MODE_FWD> launch, from the ncu capture
-# summarised in profiles/lmhead_fwd_qwen1p5b_8prompts.md (a reduced batch of the same workload); the kernel's DRAM
-# traffic grows in proportion to the token rows it processes, so it is scaled by kept tokens.
-NCU_FWD_TRAFFIC = {"config": 1, "bytes": 1.117685e9, "tokens": 36784,
-                   "source": "ncu capture of a 36784-token batch (288 token tiles), scaled by kept tokens"}
-UNIT = "tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one lmhead_kernel<MODE_FWD> launch on the full-size workload,
+# from the one-pass ncu captures summarised in profiles/lmhead_fwd_full_size_dram.md (per workload index).
+NCU_FWD_TRAFFIC = {1: {"bytes": 5.795e9, "tokens": 204780}, 2: {"bytes": 85.26e9, "tokens": 468700}}
+NCU_FWD_TRAFFIC_SOURCE = "ncu capture of the full-size launch (dram__bytes_read.sum + dram__bytes_write.sum)"
 
 
 def parse_args():
@@ -280,11 +278,12 @@ def run_ours(args):
     fwd_ms = float(np.mean(fw))
     clocks = sampler.stop()
     flops_launch = 2.0 * T_kept * wl.d * wl.V
-    traffic = NCU_FWD_TRAFFIC["bytes"] * T_kept / NCU_FWD_TRAFFIC["tokens"] if args.config == NCU_FWD_TRAFFIC["config"] else None
+    cap = NCU_FWD_TRAFFIC.get(args.config) if args.prompts == 0 else None
+    traffic = cap["bytes"] * T_kept / cap["tokens"] if cap else None
     achieved = flops_launch / (fwd_ms * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "lmhead_kernel<MODE_FWD>", "achieved": achieved, "peak": pk["burst"],
                 "unit": "TFLOP/s", "frac": achieved / pk["burst"], "peak_source": pk["src"] + " burst bf16",
-                "traffic": traffic, "traffic_source": NCU_FWD_TRAFFIC["source"] if traffic else None,
+                "traffic": traffic, "traffic_source": NCU_FWD_TRAFFIC_SOURCE if traffic else None,
                 "ms_per_launch": fwd_ms,
                 "step_executed_tflops": 8.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12,
                 "step_frac_of_sustained": 8.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12 / pk["sustained"]}
