@@ -32,10 +32,6 @@
 #include "loss_common.cuh"
 #include "tc_ptx.cuh"
 
-#ifndef AERO_L2_HINTS
-#define AERO_L2_HINTS 0
-#endif
-
 namespace lmhead {
 
 #ifndef AERO_TC_STAGES
@@ -231,10 +227,6 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
       uint32_t it = 0;
       bool ok = true;
       unsigned int meetings = 0;
-#if AERO_L2_HINTS
-      // H tiles are re-read for every vocabulary tile: keep them; a W tile is used once per wave
-      const uint64_t pol_h = tc::l2_policy_evict_last(), pol_w = tc::l2_policy_evict_first();
-#endif
       // every CTA takes part in the same number of meetings: units of the longest schedule x nsync
       const int total_units = ((n_tiles - p.tile_begin + 1) / 2) * vsplit;
       const int max_units = total_units > 0 ? (total_units + npairs - 1) / npairs : 0;
@@ -261,13 +253,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
             uint8_t* a_s = smem + (size_t)s * STAGE_BYTES;
             const uint32_t full0 = tc::mapa_shared(tc::smem_u32(&ctl->full[s]), 0);
             if (rank == 0) tc::mbar_arrive_expect_tx(&ctl->full[s], 2 * STAGE_BYTES);
-#if AERO_L2_HINTS
-            tc::tma_load_2d_pair_hint(a_s, &tmH, kb * BK, row0, full0, pol_h);
-            tc::tma_load_2d_pair_hint(a_s + A_BYTES, &tmW, kb * BK, j * BN + (int)rank * BNH, full0, pol_w);
-#else
             tc::tma_load_2d_pair(a_s, &tmH, kb * BK, row0, full0);
             tc::tma_load_2d_pair(a_s + A_BYTES, &tmW, kb * BK, j * BN + (int)rank * BNH, full0);
-#endif
           }
         }
         // a unit whose range has fewer vocabulary tiles than meeting points still counts them all
@@ -439,11 +426,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
               tc::fence_proxy_async();
               __syncwarp();
               if (lane == 0) {
-#if AERO_L2_HINTS
-                tc::tma_store_2d_hint(&tmDZ, stg, col0 - 32, dz_row0, tc::l2_policy_evict_first());
-#else
                 tc::tma_store_2d(&tmDZ, stg, col0 - 32, dz_row0);
-#endif
                 tc::tma_store_commit();
               }
               ++nstore;
