@@ -4,7 +4,8 @@
 //   KIND_DH : dH[rows of the chunk, :]  = dz[rows, V] * W[V, d]       (reduce over vocabulary)
 //   KIND_DW : dW[V, d]                 += dz[rows, V]^T * H[rows, d]  (reduce over the chunk's rows)
 //
-// dz is the chunk's scratch block written by the lm_head kernel in dz mode.  W and H are
+// dz is the chunk's scratch block written by the lm_head kernel in dz mode, stored as contiguous
+// [128 rows][64 columns] tiles (tile-major, then column block).  W and H are
 // used as stored (row-major, d contiguous), i.e. as MN-major B operands; dz is a K-major
 // A operand for dH and an MN-major A operand for dW, so nothing is transposed in memory.
 // Output tiles are 128 x 256; a unit is one output tile, units are numbered row-tile-major
@@ -98,7 +99,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           if (KIND == KIND_DH) {
             // A: dz rows of the tile (K-major, K = vocabulary); B: W rows kb*64.. as four
             // 64-column blocks (MN-major, blocked view)
-            tc::tma_load_2d(a_s, &tmA, kb * BK, mt * BM, &ctl->full[s]);
+            tc::tma_load_4d(a_s, &tmA, 0, 0, kb, mt, &ctl->full[s]);
             tc::tma_load_3d(b_s, &tmB, 0, kb * BK, nt * (BN / 64), &ctl->full[s]);
           } else {
             // A: two 64-column blocks of dz over 64 chunk rows (MN-major);
@@ -110,7 +111,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               row_next = nxt < chunk_tiles ? __ldg(p.tile_row + p.tile_begin + nxt) : 0;
             }
             const int hrow = row_cur + (kb % (BM / BK)) * BK;
-            tc::tma_load_3d(a_s, &tmA, 0, kb * BK, mt * (BM / 64), &ctl->full[s]);
+            tc::tma_load_4d(a_s, &tmA, 0, (kb % (BM / BK)) * BK, mt * (BM / 64), kb / (BM / BK), &ctl->full[s]);
             tc::tma_load_3d(b_s, &tmB, 0, hrow, nt * (BN / 64), &ctl->full[s]);
           }
         }

@@ -94,7 +94,7 @@ struct Params {
   const float* g_in;
   const float* ent_in;
   float grad_scale;
-  __nv_bfloat16* dz;            // [(tile - tile_begin) * 128 + r][ldz]
+  __nv_bfloat16* dz;            // tiled: [tile - tile_begin][ldz / 64][128 rows][64 columns]
   long long ldz;
 };
 
@@ -329,7 +329,6 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
           }
         }
       }
-      const int dz_row0 = (tile - p.tile_begin) * BM + warp * 32;   // first dz row of this warp
 
       for (int j = unit_j0(k), j1 = unit_j1(k); ok && j < j1; ++j, ++at) {
         const uint32_t buf = at & 1u, aph = (at >> 1) & 1u;
@@ -426,7 +425,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
               tc::fence_proxy_async();
               __syncwarp();
               if (lane == 0) {
-                tc::tma_store_2d(&tmDZ, stg, col0 - 32, dz_row0);
+                tc::tma_store_4d(&tmDZ, stg, 0, warp * 32, (col0 - 32) / 64, tile - p.tile_begin);
                 tc::tma_store_commit();
               }
               ++nstore;

@@ -65,18 +65,17 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
 
   const CUtensorMapDataType BF = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
   CUtensorMap tmH_k, tmW_k, tmDZ_k, tmW_mn, tmDZ_mn, tmH_mn;
-  const uint64_t dz_rows = (uint64_t)tpc * lmhead::BM;
   // K-major views (inner extent 64 = one 128-byte swizzle row) for the recompute and for dz as A of dH
   if ((rc = aero_make_tmap_2d(ctx, &tmH_k, BF, 2, H, T, d, d, lmhead::BM, 64))) return rc;
   if ((rc = aero_make_tmap_2d(ctx, &tmW_k, BF, 2, W, V, d, d, lmhead::BNH, 64))) return rc;
-  if ((rc = aero_make_tmap_2d(ctx, &tmDZ_k, BF, 2, dz, dz_rows, ldz, ldz, gemmbwd::BM, 64))) return rc;
+  if ((rc = aero_make_tmap_dz(ctx, &tmDZ_k, dz, (uint64_t)tpc, (uint64_t)(ldz / 64), gemmbwd::BM, 1))) return rc;
   // MN-major operands: blocked views, one box = 64 rows x (4 or 2) column blocks of 64
   if ((rc = aero_make_tmap_blocked(ctx, &tmW_mn, W, V, d, d, 64, gemmbwd::BN / 64))) return rc;
-  if ((rc = aero_make_tmap_blocked(ctx, &tmDZ_mn, dz, dz_rows, ldz, ldz, 64, gemmbwd::BM / 64))) return rc;
+  if ((rc = aero_make_tmap_dz(ctx, &tmDZ_mn, dz, (uint64_t)tpc, (uint64_t)(ldz / 64), 64, gemmbwd::BM / 64))) return rc;
   if ((rc = aero_make_tmap_blocked(ctx, &tmH_mn, H, T, d, d, 64, gemmbwd::BN / 64))) return rc;
   // store view of the dz block for the lm_head kernel's epilogue: 32 rows x 64 columns per copy
   CUtensorMap tmDZ_st;
-  if ((rc = aero_make_tmap_2d(ctx, &tmDZ_st, BF, 2, dz, dz_rows, ldz, ldz, 32, 64))) return rc;
+  if ((rc = aero_make_tmap_dz(ctx, &tmDZ_st, dz, (uint64_t)tpc, (uint64_t)(ldz / 64), 32, 1))) return rc;
 
   const bool with_entropy = ex.entropy != nullptr && ex.ent_coef != 0.f;
   auto k_dz = with_entropy ? lmhead::lmhead_kernel<lmhead::MODE_DZ_ENT> : lmhead::lmhead_kernel<lmhead::MODE_DZ>;
