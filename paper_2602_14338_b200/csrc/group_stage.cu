@@ -380,6 +380,7 @@ __device__ void run_tile_staged(const Args& a, const Workspace& ws, TileShared& 
       const unsigned long long mykey = rs.ck[j];
       const int lo = ps.lo[q], hi = ps.lo[q + 1];
       int rank = 0;
+#pragma unroll 4
       for (int k = lo; k < hi; ++k) rank += rs.ck[k] < mykey ? 1 : 0;
       kp = rank < ps.quota[q];
     }
@@ -419,10 +420,20 @@ __device__ void run_tile_staged(const Args& a, const Workspace& ws, TileShared& 
     const bool kp = j < nroll && (rs.flag[j] & 4);
     const unsigned kept_mask = __ballot_sync(0xffffffffu, kp);
     long long tok = kp ? rs.len[j] : 0;
+    if (__reduce_max_sync(0xffffffffu, (unsigned)tok) < (1u << 26)) {      // 32 lengths below 2^26: a 32-bit scan
+      unsigned t32 = (unsigned)tok;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const long long t2 = __shfl_up_sync(0xffffffffu, tok, o);
-      if (lane >= o) tok += t2;
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t2 = __shfl_up_sync(0xffffffffu, t32, o);
+        if (lane >= o) t32 += t2;
+      }
+      tok = t32;
+    } else {
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const long long t2 = __shfl_up_sync(0xffffffffu, tok, o);
+        if (lane >= o) tok += t2;
+      }
     }
     if (kp) {
       rs.ck[j] = (unsigned long long)(tok - rs.len[j]);
@@ -433,8 +444,17 @@ __device__ void run_tile_staged(const Args& a, const Workspace& ws, TileShared& 
   reduce_partial(sh, mine);
   __syncthreads();
 
-  // ---- warp 0: exclusive prefixes over the chunks, then the chained scan across tiles ----
-  if (tid < 32) {
+  // ---- warp 0: exclusive prefixes over the chunks, then the chained scan across tiles; meanwhile
+  // the other warps write what does not depend on it: advantage and keep flag per rollout ----
+  if (tid >= 32) {
+    for (int j = tid - 32; j < nroll; j += kThreads - 32) {
+      const int q = rs.pid[j];
+      const uint8_t f = rs.flag[j];
+      const bool kp = (f & 4) != 0;
+      a.adv[r0 + j] = kp ? (((f & 2) ? 1.f : 0.f) - ps.mu[q]) * ps.inv[q] : 0.f;
+      a.keep[r0 + j] = kp ? 1 : 0;
+    }
+  } else {
     const int nchunks = (nroll + 31) >> 5;
     int run_cnt = 0;
     long long run_tok = 0;
@@ -462,17 +482,12 @@ __device__ void run_tile_staged(const Args& a, const Workspace& ws, TileShared& 
   const int base_roll = sh.base_roll;
   const long long base_tok = sh.base_tok;
 
-  // ---- per rollout: advantage, keep flag, compacted id and token offset ----
-  for (int j = tid; j < nroll; j += kThreads) {
-    const int i = r0 + j;
-    const int q = rs.pid[j];
-    const uint8_t f = rs.flag[j];
-    const bool kp = (f & 4) != 0;
-    a.adv[i] = kp ? (((f & 2) ? 1.f : 0.f) - ps.mu[q]) * ps.inv[q] : 0.f;
-    a.keep[i] = kp ? 1 : 0;
-    if (kp && !failed) {
+  // ---- per kept rollout: compacted id and token offset ----
+  if (!failed) {
+    for (int j = tid; j < nroll; j += kThreads) {
+      if (!(rs.flag[j] & 4)) continue;
       const int pos = base_roll + rs.chunk_cnt[j >> 5] + rs.len[j];
-      a.kept_ids[pos] = i;
+      a.kept_ids[pos] = r0 + j;
       a.kept_tok_off[pos] = base_tok + rs.chunk_tok[j >> 5] + (long long)rs.ck[j];
     }
   }
