@@ -231,7 +231,8 @@ def run_ours(args):
     dH = torch.empty_like(H)
     dW = torch.empty((wl.V, wl.d), dtype=torch.float32, device=dev)
     chunk = min(args.chunk_tokens, (T + 127) // 128 * 128)
-    ws_b = torch.empty(ctx.bwd_workspace_bytes(T, wl.d, wl.V, R, chunk), dtype=torch.uint8, device=dev)
+    ws_b = torch.empty(max(ctx.bwd_workspace_bytes(T, wl.d, wl.V, R, chunk), ctx.fwd_bwd_workspace_bytes(T, wl.d, wl.V, R, chunk)),
+                       dtype=torch.uint8, device=dev)
 
     # old log-probs: the current policy's own log-probs (the log-prob pass alone) plus seeded noise
     f0 = ctx.logprob_fwd(cfg, H, W, y)
@@ -239,10 +240,17 @@ def run_ours(args):
     del f0
 
     def step():
+        # group stage, then forward and backward of stage (b) in one call (no recompute of the logits)
+        g = ctx.group_stats(cfg, go, reward, cs, key=key, alpha_in=alpha, beta_in=beta, out=gbuf)
+        f, _, _ = ctx.grpo_loss_fwd_bwd(cfg, H, W, y, old, cs, g["adv"], g["w"], g["keep"], out=fbuf, dH=dH, dW=dW,
+                                        workspace=ws_b)
+        return g, f
+
+    def step_two_calls():
+        # the same step through the separate forward and backward calls (the backward recomputes the logits)
         g = ctx.group_stats(cfg, go, reward, cs, key=key, alpha_in=alpha, beta_in=beta, out=gbuf)
         f = ctx.grpo_loss_fwd(cfg, H, W, y, old, cs, g["adv"], g["w"], g["keep"], out=fbuf)
         ctx.grpo_loss_bwd(cfg, H, W, y, cs, g["keep"], f["lse"], f["g"], dH=dH, dW=dW, workspace=ws_b)
-        return g, f
 
     for _ in range(max(args.warmup, 1)):
         g, f = step()
@@ -286,8 +294,21 @@ def run_ours(args):
                 "unit": "TFLOP/s", "frac": achieved / pk["burst"], "peak_source": pk["src"] + " burst bf16",
                 "traffic": traffic, "traffic_source": NCU_FWD_TRAFFIC_SOURCE if traffic else None,
                 "ms_per_launch": fwd_ms,
-                "step_executed_tflops": 8.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12,
-                "step_frac_of_sustained": 8.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12 / pk["sustained"]}
+                "step_executed_tflops": 6.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12,
+                "step_frac_of_sustained": 6.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12 / pk["sustained"]}
+    # the two-call step (8 d V executed FLOPs per token), for comparison
+    step_two_calls()
+    torch.cuda.synchronize()
+    a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a2.record()
+    for _ in range(2):
+        step_two_calls()
+    b2.record()
+    torch.cuda.synchronize()
+    ms2 = a2.elapsed_time(b2) / 2
+    roofline["two_call_step"] = {"ms": ms2, "tokens_per_s": T_kept / (ms2 * 1e-3),
+                                 "executed_tflops": 8.0 * T_kept * wl.d * wl.V / (ms2 * 1e-3) / 1e12,
+                                 "frac_of_sustained": 8.0 * T_kept * wl.d * wl.V / (ms2 * 1e-3) / 1e12 / pk["sustained"]}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -61,6 +61,9 @@ extern "C" {
 #define AERO_ST_BAD_REWARD     4u   /* reward not exactly 0 or 1                       */
 #define AERO_ST_EMPTY_ROLLOUT  8u   /* cs[i+1] == cs[i] for a present rollout          */
 #define AERO_ST_TIMEOUT       16u   /* a bounded wait inside a kernel ran out          */
+#define AERO_ST_RANGE         32u   /* aero_grpo_loss_fwd_bwd: a logit lies more than 125 octaves above  */
+                                    /* the shift taken from the row's first logits; that row's gradient   */
+                                    /* is saturated (use aero_grpo_loss_fwd + aero_grpo_loss_bwd instead) */
 
 /* ---- enumerations ------------------------------------------------------------- */
 #define AERO_UNIFORM_MASK   0   /* all-correct / all-incorrect groups are dropped (Sec. 3.2)      */
@@ -286,6 +289,31 @@ int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d,
                        void* workspace, size_t workspace_bytes);
 
 /* ------------------------------------------------------------------------------
+ * Stage (b), forward and backward in one call (Eq. 2, Eq. 3; same results as
+ * aero_grpo_loss_fwd followed by aero_grpo_loss_bwd, same arguments).
+ *
+ * The two separate calls must recompute the logits in the backward (8 d V FLOP per token).
+ * Called together, the forward of each chunk of token rows also leaves
+ * p~_tv = exp(z_tv - c_t) in bf16 in the chunk's scratch block, c_t being a per-row shift taken
+ * from the row's first logits; when lse_t and g_t are known the block is rescaled in place to
+ * dz_tv = grad_scale (g_t 1[v == y_t] - g_t exp(c_t - lse_t) p~_tv), and dH, dW follow as in
+ * aero_grpo_loss_bwd: 6 d V FLOP per token.  bf16 shares fp32's exponent range, so p~ carries the
+ * same 2^-9 relative rounding dz has in the two-call path.  Neither the logits nor anything of
+ * size [T,V] is stored: the scratch block is one chunk of rows, as in the backward.
+ *
+ * workspace: at least aero_fwd_bwd_workspace_bytes(T, d, V, R, chunk_tokens), 256-byte aligned.
+ * fp32 inputs run the two plain calls one after the other.
+ */
+size_t aero_fwd_bwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R, int64_t chunk_tokens);
+
+int aero_grpo_loss_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                           const void* H, const void* W, const int32_t* y, const float* old_logp,
+                           const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                           float* logp, float* lse, float* g, float* loss, float* metrics,
+                           float grad_scale, void* dH, float* dW, int accumulate_dW,
+                           void* workspace, size_t workspace_bytes);
+
+/* ------------------------------------------------------------------------------
  * Stage (b) with the regularisers of Eq. 2 and Table 9.
  *
  * Per kept token of rollout i, with D_t = exp(q_t) - q_t - 1, q_t = ref_logp_t - logp_t
@@ -330,7 +358,7 @@ int aero_logprob_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, i
  * One whole step of the path from HOST buffers: stage (a), forward and backward
  * (the same operations and citations as the three calls above), for callers whose
  * rollout batch lives in host memory.  The call copies the batch to the device,
- * runs aero_group_stats, aero_grpo_loss_fwd and aero_grpo_loss_bwd on the context's
+ * runs aero_group_stats and aero_grpo_loss_fwd_bwd on the context's
  * stream, copies the scalars back and synchronises the stream before returning.
  *
  * HOST inputs (pinned memory makes the copies asynchronous): go_h [P+1] i32,

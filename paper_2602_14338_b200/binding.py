@@ -21,6 +21,7 @@ AERO_TOKEN_MEAN, AERO_SEQ_MEAN = 0, 1
 AERO_DENOM_SURVIVING, AERO_DENOM_ALL = 0, 1
 AERO_BF16, AERO_FP32 = 0, 1
 AERO_ST_BAD_TARGET, AERO_ST_BAD_OFFSETS, AERO_ST_BAD_REWARD, AERO_ST_EMPTY_ROLLOUT, AERO_ST_TIMEOUT = 1, 2, 4, 8, 16
+AERO_ST_RANGE = 32
 
 EXPORTS = [
     "aero_version", "aero_error_string", "aero_cfg_default", "aero_create", "aero_destroy",
@@ -29,6 +30,7 @@ EXPORTS = [
     "aero_step_workspace_bytes", "aero_grpo_step_host", "aero_launch_count", "aero_group_stats_static",
     "aero_grpo_loss_reg_fwd", "aero_grpo_loss_reg_bwd", "aero_logprob_fwd",
     "aero_alloc_cfg_default", "aero_allocate_workspace_bytes", "aero_allocate_sim",
+    "aero_fwd_bwd_workspace_bytes", "aero_grpo_loss_fwd_bwd",
 ]
 
 
@@ -94,6 +96,10 @@ def load_library():
     lib.aero_allocate_workspace_bytes.restype = sz
     lib.aero_allocate_workspace_bytes.argtypes = [i32]
     lib.aero_allocate_sim.argtypes = [vp, C.POINTER(AeroCfg), C.POINTER(AeroAllocCfg), i32] + [vp] * 5 + [vp, sz]
+    lib.aero_fwd_bwd_workspace_bytes.restype = sz
+    lib.aero_fwd_bwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i64]
+    lib.aero_grpo_loss_fwd_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 13 + [f32] +
+                                           [vp, vp, C.c_int, vp, sz])
     lib.aero_step_workspace_bytes.restype = sz
     lib.aero_step_workspace_bytes.argtypes = [i32, i32, i64, i32, i32, i64, i32]
     lib.aero_grpo_step_host.argtypes = ([vp, C.POINTER(AeroCfg), i32, i32, i64, i32, i32] + [vp] * 12 + [C.c_int] +
@@ -349,6 +355,43 @@ class Context:
             workspace.data_ptr(), workspace.numel())
         _check(rc, "aero_grpo_loss_reg_bwd")
         return dH, dW
+
+    def fwd_bwd_workspace_bytes(self, T, d, V, R, chunk_tokens):
+        return self.lib.aero_fwd_bwd_workspace_bytes(T, d, V, R, chunk_tokens)
+
+    def grpo_loss_fwd_bwd(self, cfg, H, W, y, old_logp, cs, adv, w, keep, out=None, grad_scale=1.0, dH=None, dW=None,
+                          accumulate_dW=False, chunk_tokens=None, workspace=None):
+        """aero_grpo_loss_fwd_bwd: forward and backward of stage (b) in one call (no recompute of the logits).
+        Returns (forward outputs dict, dH, dW)."""
+        T, d = H.shape
+        V = W.shape[0]
+        R = cs.numel() - 1
+        dt = torch.bfloat16 if cfg.dtype == AERO_BF16 else torch.float32
+        o = out if out is not None else {}
+        for name in ("logp", "lse", "g"):
+            if name not in o:
+                o[name] = torch.empty(max(T, 1), dtype=torch.float32, device=self.device)
+        if "loss" not in o:
+            o["loss"] = torch.zeros(1, dtype=torch.float32, device=self.device)
+        if "metrics" not in o:
+            o["metrics"] = torch.zeros(4, dtype=torch.float32, device=self.device)
+        if dH is None:
+            dH = torch.empty((max(T, 1), d), dtype=dt, device=self.device)[:T]
+        if dW is None:
+            dW = torch.empty((V, d), dtype=torch.float32, device=self.device)
+        if workspace is None:
+            if chunk_tokens is None:
+                chunk_tokens = min(max(128, (T + 127) // 128 * 128), 2 * 148 * 128)
+            workspace = self.workspace(self.fwd_bwd_workspace_bytes(T, d, V, R, chunk_tokens))
+        rc = self.lib.aero_grpo_loss_fwd_bwd(
+            self.h, C.byref(cfg), T, d, V, R, _ptr(H, dt, T * d, "H"), _ptr(W, dt, V * d, "W"),
+            _ptr(y, torch.int32, T, "y"), _ptr(old_logp, torch.float32, T, "old_logp"),
+            _ptr(cs, torch.int64, R + 1, "cs"), _ptr(adv, torch.float32, R, "adv"), _ptr(w, torch.float32, R, "w"),
+            _ptr(keep, torch.uint8, R, "keep"), _ptr(o["logp"]), _ptr(o["lse"]), _ptr(o["g"]), _ptr(o["loss"]),
+            _ptr(o["metrics"]), C.c_float(grad_scale), _ptr(dH, dt, T * d, "dH"), _ptr(dW, torch.float32, V * d, "dW"),
+            1 if accumulate_dW else 0, workspace.data_ptr(), workspace.numel())
+        _check(rc, "aero_grpo_loss_fwd_bwd")
+        return o, dH, dW
 
     def grpo_loss_bwd(self, cfg, H, W, y, cs, keep, lse, g, grad_scale=1.0, dH=None, dW=None,
                       accumulate_dW=False, chunk_tokens=None, workspace=None):

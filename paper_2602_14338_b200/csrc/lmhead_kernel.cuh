@@ -9,6 +9,14 @@
 //              log-probs, the log-probs alone.
 //   MODE_DZ  : dz = coef_t * (1[v == y_t] - exp(z - lse_t)) rounded to bf16 and stored to
 //              the chunk's scratch block (Eq. 3 through the softmax).
+//   MODE_FWD_P : the forward of a fused step.  Besides the log-probs it stores, for its chunk of
+//              token tiles, p~ = exp(z - c_t) in bf16 into the block the dz mode would write,
+//              with one shift c_t per row and vocabulary split (the row's first logits plus a
+//              margin: bf16 has fp32's exponent range, so any c_t within ~85 of the row's
+//              log-sum-exp loses nothing but the usual 2^-9 relative rounding).  Once lse_t and
+//              g_t are known, dz = g_t 1[v=y_t] - g_t exp(c_t - lse_t) p~ is an element-wise
+//              rescale of that block (scale_dz_kernel), which replaces the recompute of the
+//              logits in the backward: 6 d V instead of 8 d V FLOP per token.
 //   The _ENT variants add the entropy bonus (Table 9): the forward also carries
 //   sum_v exp(z - m) z, giving H_t = lse_t - E_p[z]; the backward adds
 //   e_t p_tv (z_tv - lse_t + H_t) to dz, e_t = ent_coef * w_i.
@@ -41,7 +49,9 @@ namespace lmhead {
 constexpr int BM = 128, BN = 256, BNH = BN / 2, BK = 64, STAGES = AERO_TC_STAGES, UMMA_K = 16;
 constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BNH * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
-constexpr int MODE_FWD = 0, MODE_DZ = 1, MODE_FWD_ENT = 2, MODE_DZ_ENT = 3;   // bit 0: dz mode, bit 1: entropy term
+// bit 0: dz mode, bit 1: entropy term, bit 2: the forward also stores exp(z - c_t) of the chunk (see MODE_FWD_P)
+constexpr int MODE_FWD = 0, MODE_DZ = 1, MODE_FWD_ENT = 2, MODE_DZ_ENT = 3, MODE_FWD_P = 4;
+constexpr float kShiftMargin = 40.f;   // c_t = (largest logit of the row's first 32 columns) + this margin
 constexpr float kMasked = -1e30f;   // stands for -inf in columns past V (finite, so that 0 * z stays 0)
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 
@@ -88,6 +98,7 @@ struct Params {
   float* lse_out;
   float* g_out;
   float* ent_out;               // entropy per row (entropy modes)
+  float* shift_out;             // MODE_FWD_P: c_t * log2(e) per split and row, [vsplit][T]
   double* partials;             // [tile][4 epilogue warps][kPartialStride]
   // dz modes
   const float* lse_in;
@@ -185,7 +196,8 @@ template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW,
               const __grid_constant__ CUtensorMap tmDZ, const Params p) {
-  constexpr bool IS_DZ = (MODE & 1) != 0, ENT = (MODE & 2) != 0;
+  constexpr bool IS_DZ = (MODE & 1) != 0, ENT = (MODE & 2) != 0, STORE_P = (MODE & 4) != 0;
+  constexpr bool STORES = IS_DZ || STORE_P;       // the epilogue writes a tile of the chunk's block
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* stg_all = smem + (size_t)STAGES * STAGE_BYTES;
@@ -316,6 +328,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
       const bool live = valid_row && !bad_y;
 
       float m2 = -INFINITY, l = 0.f, zy = 0.f, sz = 0.f;   // forward running state (log2 domain); sz = sum e^(z-m) z
+      float c2 = 0.f;                                      // MODE_FWD_P: shift of the stored exponentials, log2 domain
       float lse2 = 0.f, coef = 0.f, et = 0.f, c0 = 0.f;     // dz per-row constants: dz = 1[y] coef + p (c0 + et z)
       if (IS_DZ) {
         if (live) {
@@ -343,8 +356,35 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
           continue;
         }
         const int col_base = j * BN;
-        const int ncol = min(BN, (IS_DZ ? (int)p.ldz : p.V) - col_base);
+        const int ncol = min(BN, (STORES ? (int)p.ldz : p.V) - col_base);
         const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + buf * BN;
+        // 32 columns of this thread's row as 16 packed words -> half of the row's 128-byte line in the
+        // staging buffer (16-byte chunks XOR-swizzled with the row, matching the store's tensor map);
+        // every second call sends the 32 x 64 buffer to the chunk's block.
+        auto stage_store = [&](const uint32_t (&pk)[16], int c, int col0) {
+          const int half = c & 1;
+          if (half == 0) {
+            // the buffer is free once the store issued two blocks ago has read it
+            if (lane == 0) tc::tma_store_wait_read<1>();
+            __syncwarp();
+          }
+          uint8_t* stg = stg_warp + (nstore & 1u) * STG_BUF_BYTES;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int chunk = (half * 4 + q) ^ (lane & 7);
+            *reinterpret_cast<uint4*>(stg + lane * 128 + chunk * 16) =
+                make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
+          }
+          if (half == 1) {
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tc::tma_store_4d(&tmDZ, stg, 0, warp * 32, (col0 - 32) / 64, tile - p.tile_begin);
+              tc::tma_store_commit();
+            }
+            ++nstore;
+          }
+        };
         // One 32-column chunk of this thread's row, already in registers.
         auto process = [&](const uint32_t (&r)[32], int c) {
           const int col0 = col_base + c * 32;
@@ -360,12 +400,28 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
 #pragma unroll
             for (int q = 1; q < 32; ++q) cmax = fmaxf(cmax, z[q]);
             const float m2n = fmaxf(m2, cmax * kLog2e);
+            if (STORE_P && m2 == -INFINITY) c2 = fmaf(cmax + kShiftMargin, kLog2e, 0.f);   // first chunk of the row
             float acc = 0.f, accz = 0.f;
+            if (STORE_P) {
+              // e^(z - c) = e^(z - m) * 2^(m2 - c2): one extra multiply per logit
+              const float d2 = m2n - c2;
+              if (live && d2 > 126.f) aero_raise(p.status, AERO_ST_RANGE);
+              const float sc = live ? ex2(fminf(d2, 126.f)) : 0.f;
+              uint32_t pk[16];
 #pragma unroll
-            for (int q = 0; q < 32; ++q) {
-              const float e = ex2(fmaf(z[q], kLog2e, -m2n));
-              acc += e;
-              if (ENT) accz = fmaf(e, z[q], accz);
+              for (int q = 0; q < 32; q += 2) {
+                const float e0 = ex2(fmaf(z[q], kLog2e, -m2n)), e1 = ex2(fmaf(z[q + 1], kLog2e, -m2n));
+                acc += e0 + e1;
+                pk[q >> 1] = pack_bf16(e0 * sc, e1 * sc);
+              }
+              stage_store(pk, c, col0);
+            } else {
+#pragma unroll
+              for (int q = 0; q < 32; ++q) {
+                const float e = ex2(fmaf(z[q], kLog2e, -m2n));
+                acc += e;
+                if (ENT) accz = fmaf(e, z[q], accz);
+              }
             }
             const float scale = ex2(m2 - m2n);
             l = fmaf(l, scale, acc);
@@ -408,28 +464,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
                 pk[q >> 1] = pack_bf16(v0, v1);
               }
             }
-            const int half = c & 1;
-            if (half == 0) {
-              // the buffer is free once the store issued two blocks ago has read it
-              if (lane == 0) tc::tma_store_wait_read<1>();
-              __syncwarp();
-            }
-            uint8_t* stg = stg_warp + (nstore & 1u) * STG_BUF_BYTES;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const int chunk = (half * 4 + q) ^ (lane & 7);
-              *reinterpret_cast<uint4*>(stg + lane * 128 + chunk * 16) =
-                  make_uint4(pk[4 * q], pk[4 * q + 1], pk[4 * q + 2], pk[4 * q + 3]);
-            }
-            if (half == 1) {
-              tc::fence_proxy_async();
-              __syncwarp();
-              if (lane == 0) {
-                tc::tma_store_4d(&tmDZ, stg, 0, warp * 32, (col0 - 32) / 64, tile - p.tile_begin);
-                tc::tma_store_commit();
-              }
-              ++nstore;
-            }
+            stage_store(pk, c, col0);
           }
         };
         // TMEM loads are software-pipelined: the load of chunk c+1 is in flight while chunk c
@@ -453,6 +488,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
         if (lane == 0) tc::mbar_arrive_cluster(tc::mapa_shared(tc::smem_u32(&ctl->tempty[buf]), 0));
       }
 
+      if (STORE_P && ok && have_tile && live) p.shift_out[(size_t)((pair + k * npairs) % vsplit) * p.T + row] = c2;
       if (!IS_DZ && ok && have_tile) {
         if (vsplit > 1) {
           if (live) p.xstate[(size_t)((pair + k * npairs) % vsplit) * p.T + row] = make_float4(m2, l, zy, sz);
@@ -464,7 +500,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
   }
 
   // ---------------- teardown ----------------
-  if (IS_DZ && warp < 4 && lane == 0) tc::tma_store_wait_all<0>();   // own stores have landed
+  if (STORES && warp < 4 && lane == 0) tc::tma_store_wait_all<0>();   // own stores have landed
   __syncwarp();
   if (*abort_flag) {
     // a wait gave up: let copies and MMAs already in flight land before shared memory and

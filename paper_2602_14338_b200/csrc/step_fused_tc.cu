@@ -1,0 +1,226 @@
+// Stage (b), forward and backward in one call on the tensor-core path.  Token tiles are processed
+// in chunks; per chunk:
+//   lmhead_kernel<MODE_FWD_P>  logits, online log-sum-exp, Eq. 2, and p~ = exp(z - c_t) in bf16 into
+//                              the chunk's tiled block (instead of recomputing the logits later)
+//   merge_kernel               (large d only) merges the running states of the vocabulary splits
+//   scale_dz_kernel            dz = gs (g_t 1[v = y_t] - g_t exp(c_t - lse_t) p~), in place
+//   gemm_kernel<DH>, <DW>      dH rows of the chunk, dW += dz^T H
+// and once at the end the fixed-order reduction of the loss partials.
+#include "gemm_bwd_kernel.cuh"
+#include "lmhead_kernel.cuh"
+#include "tmap.cuh"
+
+namespace {
+
+inline long long ldz_of(int32_t V) { return ((long long)V + 63) / 64 * 64; }
+
+struct ScaleArgs {
+  __nv_bfloat16* dz;        // tiled: [tile - tile_begin][ldz / 64][128][64]
+  int nblk;                 // ldz / 64
+  const int32_t* tile_row;
+  const int32_t* tile_valid;
+  const int32_t* n_tiles;
+  int tile_begin, tile_end;
+  long long T;
+  int V, vsplit, nvt;
+  const int32_t* y;
+  const float* lse;
+  const float* g;
+  const float* shift;       // [vsplit][T], log2 domain
+  float grad_scale;
+};
+
+constexpr int kBlocksPerCta = 8;     // 64-column blocks one CTA rescales for its token tile
+
+// One CTA: one token tile x kBlocksPerCta column blocks of the chunk's block, 16 bytes per thread
+// and step.  Rows past the tile's run, or whose g is 0, come out as zeros (p~ is 0 or g is).
+__global__ void __launch_bounds__(256) scale_dz_kernel(ScaleArgs a) {
+  const int n_tiles = min(*a.n_tiles, a.tile_end);
+  const int tile = a.tile_begin + blockIdx.y;
+  if (tile >= n_tiles) return;
+  const int row0 = a.tile_row[tile], valid = a.tile_valid[tile];
+  const int b0 = blockIdx.x * kBlocksPerCta;
+  const int nb = min(kBlocksPerCta, a.nblk - b0);
+  constexpr float kLog2e = 1.4426950408889634f;
+  for (int e = threadIdx.x; e < nb * 128 * 8; e += 256) {
+    const int blk = e / (128 * 8), r = (e / 8) % 128, seg = e % 8;
+    const int b = b0 + blk;
+    const long long row = (long long)row0 + r;
+    uint4* ptr = reinterpret_cast<uint4*>(a.dz + (((size_t)blockIdx.y * a.nblk + b) * 128 + r) * 64 + seg * 8);
+    float coef = 0.f, sc = 0.f;
+    int yt = -1;
+    if (r < valid && row < a.T) {
+      coef = a.g[row] * a.grad_scale;
+      yt = a.y[row];
+      if (coef != 0.f) {
+        // the vocabulary split that produced this column block, and its shift
+        const int j = b / (lmhead::BN / 64);
+        int s = 0;
+        while (s + 1 < a.vsplit && j >= (int)((long long)(s + 1) * a.nvt / a.vsplit)) ++s;
+        sc = -coef * exp2f(a.shift[(size_t)s * a.T + row] - a.lse[row] * kLog2e);
+      }
+    }
+    uint4 v = *ptr;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
+    const int col0 = b * 64 + seg * 8;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float2 f = __bfloat1622float2(h[q]);
+      f.x = (col0 + 2 * q == yt ? coef : 0.f) + sc * f.x;
+      f.y = (col0 + 2 * q + 1 == yt ? coef : 0.f) + sc * f.y;
+      h[q] = __floats2bfloat162_rn(f.x, f.y);
+    }
+    *ptr = v;
+  }
+}
+
+// dH rows of dropped rollouts are defined to be zero; one warp per row.
+__global__ void __launch_bounds__(256) zero_dropped_rows_fused(long long T, int d, int R, const int64_t* __restrict__ cs,
+                                                               const uint8_t* __restrict__ keep,
+                                                               __nv_bfloat16* __restrict__ dH) {
+  const int lane = threadIdx.x & 31;
+  const long long warp0 = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const long long nwarps = (long long)gridDim.x * 8;
+  for (long long t = warp0; t < T; t += nwarps) {
+    const int i = aero_owner(cs, R, t);
+    if (keep[i]) continue;
+    uint4* row = reinterpret_cast<uint4*>(dH + t * d);
+    for (int k = lane; k < d / 8; k += 32) row[k] = make_uint4(0, 0, 0, 0);
+  }
+}
+
+struct FusedWs {
+  aero_tiles tiles;
+  double* partials;
+  size_t n_partials;
+  unsigned int* sync_ctr;
+  float4* xstate;
+  float* shift;
+  __nv_bfloat16* dz;
+  size_t head_bytes;
+};
+
+size_t partials_bytes(int64_t T, int32_t R) {
+  const size_t mt = (size_t)(T / lmhead::BM) + (size_t)R + 2;
+  return aero_align_up(mt * 4 * kPartialStride * sizeof(double), 256);
+}
+
+FusedWs carve(void* ws, int64_t T, int32_t d, int32_t R) {
+  FusedWs f;
+  const int vs = aero_vsplit(d);
+  const size_t Tn = (size_t)(T > 0 ? T : 1);
+  char* p = static_cast<char*>(ws);
+  f.tiles = aero_carve_tiles(ws, T, R, lmhead::BM);
+  size_t off = aero_tiles_bytes(T, R, lmhead::BM);
+  f.partials = reinterpret_cast<double*>(p + off);             off += partials_bytes(T, R);
+  f.n_partials = (size_t)f.tiles.max_tiles * 4;
+  f.sync_ctr = reinterpret_cast<unsigned int*>(p + off);       off += 256;
+  f.xstate = reinterpret_cast<float4*>(p + off);               off += vs > 1 ? aero_align_up(vs * Tn * sizeof(float4), 256) : 0;
+  f.shift = reinterpret_cast<float*>(p + off);                 off += aero_align_up(vs * Tn * sizeof(float), 256);
+  f.dz = reinterpret_cast<__nv_bfloat16*>(p + off);
+  f.head_bytes = off;
+  return f;
+}
+
+}  // namespace
+
+size_t aero_fwd_bwd_ws_bytes_tc(int64_t T, int32_t d, int32_t V, int32_t R, int64_t chunk_tokens) {
+  if (chunk_tokens < 128) chunk_tokens = 128;
+  const size_t rows = (size_t)((chunk_tokens + 127) / 128 * 128);
+  return carve(nullptr, T, d, R).head_bytes + aero_align_up(rows * (size_t)ldz_of(V) * 2, 256);
+}
+
+int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                    const void* H, const void* W, const int32_t* y, const float* old_logp,
+                    const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                    float* logp, float* lse, float* g, float* loss, float* metrics,
+                    float grad_scale, void* dH, float* dW, int accumulate_dW, void* ws, size_t ws_bytes) {
+  FusedWs f = carve(ws, T, d, R);
+  AERO_CUDA_TRY(cudaMemsetAsync(f.partials, 0, f.n_partials * kPartialStride * sizeof(double), ctx->stream));
+  if (T > 0) {
+    AERO_CUDA_TRY(cudaMemsetAsync(logp, 0, (size_t)T * sizeof(float), ctx->stream));
+    AERO_CUDA_TRY(cudaMemsetAsync(lse, 0, (size_t)T * sizeof(float), ctx->stream));
+    AERO_CUDA_TRY(cudaMemsetAsync(g, 0, (size_t)T * sizeof(float), ctx->stream));
+  }
+  if (!accumulate_dW) AERO_CUDA_TRY(cudaMemsetAsync(dW, 0, (size_t)V * d * sizeof(float), ctx->stream));
+  int rc = aero_build_tiles(ctx, T, R, cs, keep, lmhead::BM, f.tiles);
+  if (rc) return rc;
+  if (T > 0 && R > 0) {
+    const long long ldz = ldz_of(V);
+    long long tpc = (long long)((ws_bytes - f.head_bytes) / ((size_t)lmhead::BM * (size_t)ldz * 2));
+    if (tpc < 1) return AERO_ERR_WORKSPACE;
+    if (tpc > f.tiles.max_tiles) tpc = f.tiles.max_tiles;
+    if (tpc > 32768) tpc = 32768;                                          // grid.y of the rescaling kernel
+    if (tpc > ctx->sm_count) tpc = tpc / ctx->sm_count * ctx->sm_count;   // whole waves of token tiles
+    {
+      const long long blocks = (T + 7) / 8;
+      zero_dropped_rows_fused<<<(int)(blocks < 4096 ? blocks : 4096), 256, 0, ctx->stream>>>(
+          T, d, R, cs, keep, static_cast<__nv_bfloat16*>(dH));
+      ctx->launches += 1;
+    }
+    const CUtensorMapDataType BF = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    CUtensorMap tmH_k, tmW_k, tmDZ_st, tmDZ_k, tmDZ_mn, tmW_mn, tmH_mn;
+    const uint64_t nblk = (uint64_t)(ldz / 64);
+    if ((rc = aero_make_tmap_2d(ctx, &tmH_k, BF, 2, H, T, d, d, lmhead::BM, 64))) return rc;
+    if ((rc = aero_make_tmap_2d(ctx, &tmW_k, BF, 2, W, V, d, d, lmhead::BNH, 64))) return rc;
+    if ((rc = aero_make_tmap_dz(ctx, &tmDZ_st, f.dz, (uint64_t)tpc, nblk, 32, 1))) return rc;
+    if ((rc = aero_make_tmap_dz(ctx, &tmDZ_k, f.dz, (uint64_t)tpc, nblk, gemmbwd::BM, 1))) return rc;
+    if ((rc = aero_make_tmap_dz(ctx, &tmDZ_mn, f.dz, (uint64_t)tpc, nblk, 64, gemmbwd::BM / 64))) return rc;
+    if ((rc = aero_make_tmap_blocked(ctx, &tmW_mn, W, V, d, d, 64, gemmbwd::BN / 64))) return rc;
+    if ((rc = aero_make_tmap_blocked(ctx, &tmH_mn, H, T, d, d, 64, gemmbwd::BN / 64))) return rc;
+
+    auto k_fwd = lmhead::lmhead_kernel<lmhead::MODE_FWD_P>;
+    auto k_dh = gemmbwd::gemm_kernel<gemmbwd::KIND_DH>;
+    auto k_dw = gemmbwd::gemm_kernel<gemmbwd::KIND_DW>;
+    AERO_CUDA_TRY(cudaFuncSetAttribute(k_fwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lmhead::SMEM_BYTES));
+    AERO_CUDA_TRY(cudaFuncSetAttribute(k_dh, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::SMEM_BYTES));
+    AERO_CUDA_TRY(cudaFuncSetAttribute(k_dw, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::SMEM_BYTES));
+
+    const int vs = aero_vsplit(d);
+    const int nvt = (V + lmhead::BN - 1) / lmhead::BN;
+    const int n_nt = (d + gemmbwd::BN - 1) / gemmbwd::BN;
+    const long long dw_units = (long long)((V + gemmbwd::BM - 1) / gemmbwd::BM) * n_nt;
+    const long long max_pairs = ctx->sm_count / 2 > 0 ? ctx->sm_count / 2 : 1;
+    for (long long begin = 0; begin < f.tiles.max_tiles; begin += tpc) {
+      lmhead::Params p = {};
+      p.T = T; p.d = d; p.V = V; p.R = R;
+      p.tile_row = f.tiles.tile_row; p.tile_valid = f.tiles.tile_valid; p.n_tiles = f.tiles.n_tiles;
+      p.tile_begin = (int)begin; p.tile_end = (int)(begin + tpc);
+      p.y = y; p.status = ctx->d_status;
+      p.vsplit = vs; p.xstate = f.xstate; p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync();
+      p.old_logp = old_logp; p.cs = cs; p.adv = adv; p.w = w;
+      p.clip_lo = cfg->clip_lo; p.clip_hi = cfg->clip_hi;
+      p.logp = logp; p.lse_out = lse; p.g_out = g; p.partials = f.partials;
+      p.shift_out = f.shift; p.dz = f.dz; p.ldz = ldz;
+      AERO_CUDA_TRY(cudaMemsetAsync(f.sync_ctr, 0, 256, ctx->stream));
+      const long long pairs = (tpc + 1) / 2 * vs;
+      const int grid = 2 * (int)(pairs < max_pairs ? pairs : max_pairs);
+      k_fwd<<<grid, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH_k, tmW_k, tmDZ_st, p);
+      ctx->launches += 1;
+      if (vs > 1) {
+        lmhead::merge_kernel<<<(int)(tpc < 8 * ctx->sm_count ? tpc : 8 * ctx->sm_count), lmhead::BM, 0, ctx->stream>>>(p, 0);
+        ctx->launches += 1;
+      }
+      ScaleArgs sa;
+      sa.dz = f.dz; sa.nblk = (int)nblk; sa.tile_row = f.tiles.tile_row; sa.tile_valid = f.tiles.tile_valid;
+      sa.n_tiles = f.tiles.n_tiles; sa.tile_begin = (int)begin; sa.tile_end = (int)(begin + tpc);
+      sa.T = T; sa.V = V; sa.vsplit = vs; sa.nvt = nvt; sa.y = y; sa.lse = lse; sa.g = g; sa.shift = f.shift;
+      sa.grad_scale = grad_scale;
+      scale_dz_kernel<<<dim3((unsigned)((nblk + kBlocksPerCta - 1) / kBlocksPerCta), (unsigned)tpc), 256, 0, ctx->stream>>>(sa);
+
+      gemmbwd::Params gp = {};
+      gp.T = T; gp.d = d; gp.V = V; gp.ldz = ldz;
+      gp.tile_row = f.tiles.tile_row; gp.tile_valid = f.tiles.tile_valid; gp.n_tiles = f.tiles.n_tiles;
+      gp.tile_begin = (int)begin; gp.tpc = (int)tpc;
+      gp.dH = static_cast<__nv_bfloat16*>(dH); gp.dW = dW; gp.status = ctx->d_status;
+      const long long dh_units = tpc * n_nt;
+      k_dh<<<(int)(dh_units < ctx->sm_count ? dh_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
+             ctx->stream>>>(tmDZ_k, tmW_mn, gp);
+      k_dw<<<(int)(dw_units < ctx->sm_count ? dw_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
+             ctx->stream>>>(tmDZ_mn, tmH_mn, gp);
+      ctx->launches += 3;
+      AERO_CUDA_TRY(cudaGetLastError());
+    }
+  }
+  return aero_loss_finalize(ctx, f.partials, (int)f.n_partials, kPartialStride, loss, metrics, 0);
+}

@@ -42,7 +42,7 @@ StepWs carve_step(void* base, int32_t P, int32_t R, int64_t T, int32_t d, int32_
   s.logp = c.take<float>(T); s.lse = c.take<float>(T); s.g = c.take<float>(T); s.loss = c.take<float>(1);
   size_t sub = aero_group_workspace_bytes(P, R);
   const size_t f = aero_fwd_workspace_bytes(T, d, V, R);
-  const size_t b = dtype == AERO_FP32 ? 256 : aero_bwd_workspace_bytes(T, d, V, R, chunk_tokens);
+  const size_t b = dtype == AERO_FP32 ? 256 : aero_fwd_bwd_workspace_bytes(T, d, V, R, chunk_tokens);
   if (f > sub) sub = f;
   if (b > sub) sub = b;
   s.sub = c.take<char>(sub);
@@ -108,11 +108,8 @@ int aero_grpo_step_host(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R
                             s.cat, s.u, s.ao, s.bo, s.kept_ids, s.kept_tok_off, s.counters, s.metrics, s.sub,
                             s.sub_bytes);
   if (rc) return rc;
-  rc = aero_grpo_loss_fwd(ctx, cfg, T, d, V, R, s.H, W, s.y, s.old_logp, s.cs, s.adv, s.w, s.keep, s.logp, s.lse,
-                          s.g, s.loss, s.metrics + 4, 0, s.sub, s.sub_bytes);
-  if (rc) return rc;
-  rc = aero_grpo_loss_bwd(ctx, cfg, T, d, V, R, s.H, W, s.y, s.cs, s.keep, s.lse, s.g, 1.0f, dH, dW, accumulate_dW,
-                          s.sub, s.sub_bytes);
+  rc = aero_grpo_loss_fwd_bwd(ctx, cfg, T, d, V, R, s.H, W, s.y, s.old_logp, s.cs, s.adv, s.w, s.keep, s.logp, s.lse,
+                              s.g, s.loss, s.metrics + 4, 1.0f, dH, dW, accumulate_dW, s.sub, s.sub_bytes);
   if (rc) return rc;
   if (loss_h) AERO_CUDA_TRY(cudaMemcpyAsync(loss_h, s.loss, 4, D2H, st));
   if (counters_h) AERO_CUDA_TRY(cudaMemcpyAsync(counters_h, s.counters, 64, D2H, st));

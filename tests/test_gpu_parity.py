@@ -337,6 +337,53 @@ def test_vocabulary_split_between_cta_pairs(ctx, vsplit, monkeypatch):
     assert np.abs((split["entropy"][:T] - plain["entropy"][:T]).cpu().numpy()).max() < 1e-4
 
 
+@pytest.mark.parametrize("name", list(BF16_CASES) + ["tiny_fp32"])
+def test_forward_and_backward_in_one_call(ctx, name):
+    """aero_grpo_loss_fwd_bwd (the forward leaves exp(z - c_t) of each chunk, the backward rescales it
+    instead of recomputing the logits) against the oracle, in one chunk and in 128-row chunks, with and
+    without a forced vocabulary split."""
+    if name == "tiny_fp32":
+        wl, cover, peak, dtype = synth.WORKLOADS[0], {}, 0.0, "fp32"
+    else:
+        over, cover, peak = BF16_CASES[name]
+        wl = synth.scaled(synth.WORKLOADS[0] if name == "tiny_bf16" else synth.WORKLOADS[1], **over)
+        dtype = "bf16"
+    batch = TL.Batch(wl, O.Cfg(seed=wl.seed, **cover), peak=peak)
+    ref = batch.oracle_fwd()
+    rdH, rdW = batch.oracle_bwd(ref, 0.75)
+    cfg = TL.lib_cfg(batch.ocfg, dtype)
+    dv = batch.to_device()
+    tol = (1e-4, 1e-4, 1e-4) if dtype == "fp32" else (LOGP_ABS, LOSS_REL, GRAD_L2)
+    rho = ref["rho"]
+    edge = (np.abs(rho - (1 + batch.ocfg.clip_hi)) < 1e-3) | (np.abs(rho - (1 - batch.ocfg.clip_lo)) < 1e-3)
+    import os
+    for chunk, vsplit in ((None, None), (128, None), (128, "2")):
+        if vsplit:
+            os.environ["AERO_VSPLIT"] = vsplit
+        try:
+            ws = None
+            if chunk:
+                ws = torch.empty(ctx.fwd_bwd_workspace_bytes(batch.T, wl.d, wl.V, batch.R, chunk), dtype=torch.uint8, device="cuda")
+            f, dH, dW = ctx.grpo_loss_fwd_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"],
+                                              dv["keep"], grad_scale=0.75, workspace=ws)
+            torch.cuda.synchronize()
+        finally:
+            os.environ.pop("AERO_VSPLIT", None)
+        assert ctx.last_status() == 0
+        check_fwd(batch, f, ref, tol[0], tol[1], 2e-2 if dtype == "bf16" else 1e-3)
+        assert TL.rel_l2(dH.float().cpu().numpy()[~edge], rdH[~edge]) < tol[2]
+        if not edge.any():
+            assert TL.rel_l2(dW.cpu().numpy(), rdW) < tol[2]
+        owner = O.token_rollout(batch.st.cs, batch.T)
+        assert not dH.float().cpu().numpy()[batch.ref_g["keep"][owner] == 0].any()
+        if peak > 0:          # the softmax part alone
+            g = ref["g"] * 0.75
+            soft_ref = rdH - g[:, None] * batch.W[batch.st.y]
+            soft_gpu = dH.float().cpu().numpy() - g[:, None] * batch.W[batch.st.y]
+            live = (g != 0) & ~edge
+            assert TL.rel_l2(soft_gpu[live], soft_ref[live]) < 3e-2
+
+
 def test_bwd_chunking_and_accumulation(ctx):
     over, cover, _ = BF16_CASES["aero_dropped"]
     wl = synth.scaled(synth.WORKLOADS[1], **over)
@@ -510,8 +557,7 @@ def test_step_from_host_buffers_matches_device_calls(ctx):
     cfg = TL.lib_cfg(batch.ocfg, "bf16")
     dv = batch.to_device()
     gi, g = TL.run_group_gpu(ctx, cfg, st)
-    f = ctx.grpo_loss_fwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], g["adv"], g["w"], g["keep"])
-    dH, dW = ctx.grpo_loss_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], g["keep"], f["lse"], f["g"])
+    f, dH, dW = ctx.grpo_loss_fwd_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], g["adv"], g["w"], g["keep"])
     l0 = ctx.launch_count()
     dH2, dW2 = torch.empty_like(dH), torch.empty_like(dW)
     ws = torch.empty(ctx.step_workspace_bytes(batch.P, batch.R, batch.T, wl.d, wl.V, 1024, cfg.dtype),
