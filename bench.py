@@ -30,6 +30,8 @@ METRIC = "rollout tokens/sec, fused GRPO logprob+loss fwd+bwd"
 # dram__bytes_read.sum + dram__bytes_write.sum of one lmhead_kernel<MODE_FWD> launch on the full-size workload,
 # from the one-pass ncu captures summarised in profiles/lmhead_fwd_full_size_dram.md (per workload index).
 NCU_FWD_TRAFFIC = {1: {"bytes": 5.795e9, "tokens": 204780}, 2: {"bytes": 85.26e9, "tokens": 468700}}
+# the same for the launches of lmhead_kernel<MODE_FWD_P> of one step (they also write the chunk blocks)
+NCU_FWDP_TRAFFIC = {1: {"bytes": 76.8e9, "tokens": 204780}}
 NCU_FWD_TRAFFIC_SOURCE = "ncu capture of the full-size launch (dram__bytes_read.sum + dram__bytes_write.sum)"
 UNIT = "tokens/s"
 
@@ -275,7 +277,15 @@ def run_ours(args):
     ms_step = ms_total / args.steps
     value = units / (ms_total * 1e-3)
 
-    # dominant kernel: the fused lm_head kernel (forward mode), timed alone over its call
+    # dominant kernel of the timed step: lmhead_kernel<MODE_FWD_P> (one launch per chunk), timed with CUDA events
+    # that the library records around its launches, over three more steps
+    ctx.enable_kernel_timing(True)
+    for _ in range(3):
+        step()
+    fp_total_ms, fp_launches = ctx.kernel_timing_ms()
+    ctx.enable_kernel_timing(False)
+    fwdp_ms_step = fp_total_ms / 3.0
+    # the plain forward kernel (MODE_FWD, used by the separate forward call and the log-prob pass), timed over its call
     fw = []
     for _ in range(max(3, min(args.steps, 10))):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -289,11 +299,16 @@ def run_ours(args):
     flops_launch = 2.0 * T_kept * wl.d * wl.V
     cap = NCU_FWD_TRAFFIC.get(args.config) if args.prompts == 0 else None
     traffic = cap["bytes"] * T_kept / cap["tokens"] if cap else None
-    achieved = flops_launch / (fwd_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "lmhead_kernel<MODE_FWD>", "achieved": achieved, "peak": pk["burst"],
+    achieved = flops_launch / (fwdp_ms_step * 1e-3) / 1e12
+    capp = NCU_FWDP_TRAFFIC.get(args.config) if args.prompts == 0 else None
+    roofline = {"bound": "tensor", "kernel": "lmhead_kernel<MODE_FWD_P>", "achieved": achieved, "peak": pk["burst"],
                 "unit": "TFLOP/s", "frac": achieved / pk["burst"], "peak_source": pk["src"] + " burst bf16",
-                "traffic": traffic, "traffic_source": NCU_FWD_TRAFFIC_SOURCE if traffic else None,
-                "ms_per_launch": fwd_ms,
+                "traffic": capp["bytes"] * T_kept / capp["tokens"] if capp else None,
+                "traffic_source": NCU_FWD_TRAFFIC_SOURCE.replace("launch", "launches of one step") if capp else None,
+                "launches_per_step": fp_launches / 3.0, "ms_per_step_all_launches": fwdp_ms_step,
+                "plain_forward_kernel": {"kernel": "lmhead_kernel<MODE_FWD>", "ms_per_launch": fwd_ms,
+                                         "achieved": flops_launch / (fwd_ms * 1e-3) / 1e12,
+                                         "frac": flops_launch / (fwd_ms * 1e-3) / 1e12 / pk["burst"], "traffic": traffic},
                 "step_executed_tflops": 6.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12,
                 "step_frac_of_sustained": 6.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12 / pk["sustained"]}
     # the two-call step (8 d V executed FLOPs per token), for comparison

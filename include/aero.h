@@ -418,6 +418,14 @@ int aero_allocate_sim(aero_ctx* ctx, const aero_cfg* cfg, const aero_alloc_cfg* 
                       int32_t* n_gen, int32_t* c, int32_t* n_train, int64_t* counters,
                       void* workspace, size_t workspace_bytes);
 
+/* Optional timing of the dominant kernel.  With timing on, aero_grpo_loss_fwd_bwd records a pair of
+ * CUDA events on the context's stream around each launch of its lm_head kernel (up to 64 launches
+ * between read-outs; the events are created on first use).  aero_kernel_timing_ms synchronises the
+ * stream, returns the summed duration and the number of launches since the last read-out (host
+ * pointers) and starts over.  Off by default; meant for benchmarks. */
+int aero_enable_kernel_timing(aero_ctx* ctx, int on);
+int aero_kernel_timing_ms(aero_ctx* ctx, float* total_ms, int* launches);
+
 /* Number of kernels the library has launched through this context since it was created
  * (copies and memsets are not counted).  Host-side counter, no synchronisation. */
 int64_t aero_launch_count(aero_ctx* ctx);

@@ -30,7 +30,7 @@ EXPORTS = [
     "aero_step_workspace_bytes", "aero_grpo_step_host", "aero_launch_count", "aero_group_stats_static",
     "aero_grpo_loss_reg_fwd", "aero_grpo_loss_reg_bwd", "aero_logprob_fwd",
     "aero_alloc_cfg_default", "aero_allocate_workspace_bytes", "aero_allocate_sim",
-    "aero_fwd_bwd_workspace_bytes", "aero_grpo_loss_fwd_bwd",
+    "aero_fwd_bwd_workspace_bytes", "aero_grpo_loss_fwd_bwd", "aero_enable_kernel_timing", "aero_kernel_timing_ms",
 ]
 
 
@@ -100,6 +100,8 @@ def load_library():
     lib.aero_fwd_bwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i64]
     lib.aero_grpo_loss_fwd_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 13 + [f32] +
                                            [vp, vp, C.c_int, vp, sz])
+    lib.aero_enable_kernel_timing.argtypes = [vp, C.c_int]
+    lib.aero_kernel_timing_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
     lib.aero_step_workspace_bytes.restype = sz
     lib.aero_step_workspace_bytes.argtypes = [i32, i32, i64, i32, i32, i64, i32]
     lib.aero_grpo_step_host.argtypes = ([vp, C.POINTER(AeroCfg), i32, i32, i64, i32, i32] + [vp] * 12 + [C.c_int] +
@@ -435,6 +437,15 @@ class Context:
                                         ws.data_ptr(), ws.numel())
         _check(rc, "aero_allocate_sim")
         return o
+
+    def enable_kernel_timing(self, on=True):
+        _check(self.lib.aero_enable_kernel_timing(self.h, 1 if on else 0), "aero_enable_kernel_timing")
+
+    def kernel_timing_ms(self):
+        """(summed ms, launches) of the lm_head launches of grpo_loss_fwd_bwd since the last read-out."""
+        ms, n = C.c_float(0), C.c_int(0)
+        _check(self.lib.aero_kernel_timing_ms(self.h, C.byref(ms), C.byref(n)), "aero_kernel_timing_ms")
+        return ms.value, n.value
 
     # ---- whole step from host buffers ---------------------------------------------------
     def launch_count(self) -> int:

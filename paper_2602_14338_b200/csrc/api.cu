@@ -69,6 +69,9 @@ int aero_create(aero_ctx** out, int device, void* cuda_stream) {
   ctx->d_status = nullptr;
   ctx->tmap_encode = nullptr;
   ctx->launches = 0;
+  ctx->timing = 0;
+  ctx->n_timed = 0;
+  for (int i = 0; i < 64; ++i) { ctx->ev0[i] = nullptr; ctx->ev1[i] = nullptr; }
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return AERO_ERR_CUDA; }
   ctx->sm_count = prop.multiProcessorCount;
@@ -84,7 +87,35 @@ int aero_destroy(aero_ctx* ctx) {
   if (!ctx) return AERO_ERR_INVALID;
   cudaSetDevice(ctx->device);
   cudaFree(ctx->d_status);
+  for (int i = 0; i < 64; ++i) {
+    if (ctx->ev0[i]) cudaEventDestroy(ctx->ev0[i]);
+    if (ctx->ev1[i]) cudaEventDestroy(ctx->ev1[i]);
+  }
   delete ctx;
+  return AERO_OK;
+}
+
+int aero_enable_kernel_timing(aero_ctx* ctx, int on) {
+  if (!ctx) return AERO_ERR_INVALID;
+  ctx->timing = on ? 1 : 0;
+  ctx->n_timed = 0;
+  return AERO_OK;
+}
+
+int aero_kernel_timing_ms(aero_ctx* ctx, float* total_ms, int* launches) {
+  if (!ctx || !total_ms || !launches) return AERO_ERR_INVALID;
+  int rc = check_ctx(ctx);
+  if (rc) return rc;
+  AERO_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+  float sum = 0.f;
+  for (int i = 0; i < ctx->n_timed; ++i) {
+    float ms = 0.f;
+    AERO_CUDA_TRY(cudaEventElapsedTime(&ms, ctx->ev0[i], ctx->ev1[i]));
+    sum += ms;
+  }
+  *total_ms = sum;
+  *launches = ctx->n_timed;
+  ctx->n_timed = 0;
   return AERO_OK;
 }
 

@@ -17,6 +17,11 @@ struct aero_ctx {
   int sm_count;
   void* tmap_encode;      // cuTensorMapEncodeTiled, resolved once through the runtime
   long long launches;     // kernels launched so far (host-side count)
+  // optional timing of the lm_head launches of aero_grpo_loss_fwd_bwd (off by default):
+  // pairs of events recorded around each launch, read back by aero_kernel_timing_ms
+  int timing;
+  int n_timed;
+  cudaEvent_t ev0[64], ev1[64];
 };
 
 #define AERO_CUDA_TRY(expr)                          \

@@ -316,6 +316,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
     bool ok = true;
     const int r_in_tile = warp * 32 + lane;
     uint8_t* stg_warp = stg_all + warp * 2 * STG_BUF_BYTES;
+    const uint64_t pol_store = tc::l2_policy_evict_first();
     for (int k = 0; ok && unit_first(k) < n_tiles; ++k) {
       const int tile = unit_first(k) + (int)rank;
       const bool have_tile = tile < n_tiles;
@@ -379,7 +380,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
             tc::fence_proxy_async();
             __syncwarp();
             if (lane == 0) {
-              tc::tma_store_4d(&tmDZ, stg, 0, warp * 32, (col0 - 32) / 64, tile - p.tile_begin);
+              // p~ is read back only by the rescaling pass, long after it has left L2: do not let it
+              // push the H and W tiles out on its way
+              if (STORE_P) tc::tma_store_4d_hint(&tmDZ, stg, 0, warp * 32, (col0 - 32) / 64, tile - p.tile_begin, pol_store);
+              else tc::tma_store_4d(&tmDZ, stg, 0, warp * 32, (col0 - 32) / 64, tile - p.tile_begin);
               tc::tma_store_commit();
             }
             ++nstore;

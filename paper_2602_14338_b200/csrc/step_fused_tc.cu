@@ -195,7 +195,19 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
       AERO_CUDA_TRY(cudaMemsetAsync(f.sync_ctr, 0, 256, ctx->stream));
       const long long pairs = (tpc + 1) / 2 * vs;
       const int grid = 2 * (int)(pairs < max_pairs ? pairs : max_pairs);
+      const bool timed = ctx->timing && ctx->n_timed < 64;
+      if (timed) {
+        if (!ctx->ev0[ctx->n_timed]) {
+          AERO_CUDA_TRY(cudaEventCreate(&ctx->ev0[ctx->n_timed]));
+          AERO_CUDA_TRY(cudaEventCreate(&ctx->ev1[ctx->n_timed]));
+        }
+        AERO_CUDA_TRY(cudaEventRecord(ctx->ev0[ctx->n_timed], ctx->stream));
+      }
       k_fwd<<<grid, lmhead::THREADS, lmhead::SMEM_BYTES, ctx->stream>>>(tmH_k, tmW_k, tmDZ_st, p);
+      if (timed) {
+        AERO_CUDA_TRY(cudaEventRecord(ctx->ev1[ctx->n_timed], ctx->stream));
+        ctx->n_timed += 1;
+      }
       ctx->launches += 1;
       if (vs > 1) {
         lmhead::merge_kernel<<<(int)(tpc < 8 * ctx->sm_count ? tpc : 8 * ctx->sm_count), lmhead::BM, 0, ctx->stream>>>(p, 0);
