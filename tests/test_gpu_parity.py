@@ -670,3 +670,29 @@ def test_full_size_workload_in_bench_configuration(ctx, config):
     assert torch.equal(dH2, dH)
     assert ((dW2 - dW).double().norm() / dW.double().norm()).item() < 1e-4
     assert ctx.last_status() == 0
+    del dH2, dW2, ws2, ws
+    torch.cuda.empty_cache()
+    # forward and backward in one call, as bench.py times the step: same forward up to rounding, gradients within the
+    # tolerance of the two-call path (the stored exponentials are rounded to bf16 before, not after, the scaling)
+    # and of the oracle on the sampled rows
+    ws3 = torch.empty(ctx.fwd_bwd_workspace_bytes(T, wl.d, wl.V, R, chunk), dtype=torch.uint8, device="cuda")
+    f3, dH3, dW3 = ctx.grpo_loss_fwd_bwd(cfg, H, W, y, oldd, cs, g["adv"], g["w"], g["keep"], workspace=ws3)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    # (the two forward modes add the exponentials of a row in a different order)
+    assert (f3["logp"][:T] - f["logp"][:T]).abs().max().item() < 2e-5
+    assert abs(f3["loss"].item() - f["loss"].item()) <= 1e-5 * abs(f["loss"].item())
+    assert np.abs(f3["logp"][:T].cpu().numpy()[sample] - lp_s).max() <= LOGP_ABS
+    dHs3 = dH3[torch.from_numpy(sample).cuda()].float().cpu().numpy()
+    assert TL.rel_l2(dHs3[live], rdH[live]) < GRAD_L2
+    assert not dH3[dropped].float().abs().sum().item()
+    num = den = 0.0
+    for a in range(0, T, 1 << 18):                       # row blocks bound the fp32 copies
+        b = min(T, a + (1 << 18))
+        x, x3 = dH[a:b].float(), dH3[a:b].float()
+        num += float((x3 - x).pow(2).sum())
+        den += float(x.pow(2).sum())
+        del x, x3
+    assert (num / den) ** 0.5 < GRAD_L2
+    assert ((dW3 - dW).double().norm() / dW.double().norm()).item() < GRAD_L2
+    assert TL.rel_l2(dW3[vr].cpu().numpy(), ref_rows.cpu().numpy()) < GRAD_L2
