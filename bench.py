@@ -31,7 +31,7 @@ METRIC = "rollout tokens/sec, fused GRPO logprob+loss fwd+bwd"
 # from the one-pass ncu captures summarised in profiles/lmhead_fwd_full_size_dram.md (per workload index).
 NCU_FWD_TRAFFIC = {1: {"bytes": 5.795e9, "tokens": 204780}, 2: {"bytes": 85.26e9, "tokens": 468700}}
 # the same for the launches of lmhead_kernel<MODE_FWD_P> of one step (they also write the chunk blocks)
-NCU_FWDP_TRAFFIC = {1: {"bytes": 76.8e9, "tokens": 204780}}
+NCU_FWDP_TRAFFIC = {1: {"bytes": 73.99e9, "tokens": 204780}, 2: {"bytes": 575e9, "tokens": 468700}}
 NCU_FWD_TRAFFIC_SOURCE = "ncu capture of the full-size launch (dram__bytes_read.sum + dram__bytes_write.sum)"
 UNIT = "tokens/s"
 
@@ -280,9 +280,12 @@ def run_ours(args):
     # dominant kernel of the timed step: lmhead_kernel<MODE_FWD_P> (one launch per chunk), timed with CUDA events
     # that the library records around its launches, over three more steps
     ctx.enable_kernel_timing(True)
+    fp_total_ms, fp_launches = 0.0, 0
     for _ in range(3):
         step()
-    fp_total_ms, fp_launches = ctx.kernel_timing_ms()
+        ms_i, n_i = ctx.kernel_timing_ms()          # read out per step: the library keeps at most 256 pairs of events
+        fp_total_ms += ms_i
+        fp_launches += n_i
     ctx.enable_kernel_timing(False)
     fwdp_ms_step = fp_total_ms / 3.0
     # the plain forward kernel (MODE_FWD, used by the separate forward call and the log-prob pass), timed over its call

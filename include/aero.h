@@ -419,7 +419,7 @@ int aero_allocate_sim(aero_ctx* ctx, const aero_cfg* cfg, const aero_alloc_cfg* 
                       void* workspace, size_t workspace_bytes);
 
 /* Optional timing of the dominant kernel.  With timing on, aero_grpo_loss_fwd_bwd records a pair of
- * CUDA events on the context's stream around each launch of its lm_head kernel (up to 64 launches
+ * CUDA events on the context's stream around each launch of its lm_head kernel (up to 256 launches
  * between read-outs; the events are created on first use).  aero_kernel_timing_ms synchronises the
  * stream, returns the summed duration and the number of launches since the last read-out (host
  * pointers) and starts over.  Off by default; meant for benchmarks. */

@@ -71,7 +71,7 @@ int aero_create(aero_ctx** out, int device, void* cuda_stream) {
   ctx->launches = 0;
   ctx->timing = 0;
   ctx->n_timed = 0;
-  for (int i = 0; i < 64; ++i) { ctx->ev0[i] = nullptr; ctx->ev1[i] = nullptr; }
+  for (int i = 0; i < 256; ++i) { ctx->ev0[i] = nullptr; ctx->ev1[i] = nullptr; }
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return AERO_ERR_CUDA; }
   ctx->sm_count = prop.multiProcessorCount;
@@ -87,7 +87,7 @@ int aero_destroy(aero_ctx* ctx) {
   if (!ctx) return AERO_ERR_INVALID;
   cudaSetDevice(ctx->device);
   cudaFree(ctx->d_status);
-  for (int i = 0; i < 64; ++i) {
+  for (int i = 0; i < 256; ++i) {
     if (ctx->ev0[i]) cudaEventDestroy(ctx->ev0[i]);
     if (ctx->ev1[i]) cudaEventDestroy(ctx->ev1[i]);
   }

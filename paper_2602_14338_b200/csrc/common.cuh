@@ -21,7 +21,7 @@ struct aero_ctx {
   // pairs of events recorded around each launch, read back by aero_kernel_timing_ms
   int timing;
   int n_timed;
-  cudaEvent_t ev0[64], ev1[64];
+  cudaEvent_t ev0[256], ev1[256];
 };
 
 #define AERO_CUDA_TRY(expr)                          \

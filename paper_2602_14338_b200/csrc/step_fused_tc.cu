@@ -195,7 +195,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
       AERO_CUDA_TRY(cudaMemsetAsync(f.sync_ctr, 0, 256, ctx->stream));
       const long long pairs = (tpc + 1) / 2 * vs;
       const int grid = 2 * (int)(pairs < max_pairs ? pairs : max_pairs);
-      const bool timed = ctx->timing && ctx->n_timed < 64;
+      const bool timed = ctx->timing && ctx->n_timed < 256;
       if (timed) {
         if (!ctx->ev0[ctx->n_timed]) {
           AERO_CUDA_TRY(cudaEventCreate(&ctx->ev0[ctx->n_timed]));
