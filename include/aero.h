@@ -201,11 +201,9 @@ int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
  * device memory, or a latency-bound loop that must not call the allocator because an
  * allocation can synchronise the whole device.  Instead of a caller workspace, the scratch
  * is a fixed array in device memory that belongs to the loaded library itself: about
- * 1.2 MB per GPU that loads the library, held until the process exits, sized for at most
- * AERO_STATIC_MAX_PROMPTS prompts in at most 16384 tiles (the stage works on tiles of up to
- * 256 consecutive prompts holding about 1800 rollouts, so the tile limit only binds when
- * P > 16384 and the mean group has more than about 450 rollouts; R itself is not limited).
- * A batch beyond either limit returns AERO_ERR_TOO_LARGE and launches nothing.  The call,
+ * 1.6 MB per GPU that loads the library, held until the process exits, sized for at most
+ * AERO_STATIC_MAX_PROMPTS prompts whatever their group sizes (R itself is not limited).
+ * A batch beyond that limit returns AERO_ERR_TOO_LARGE and launches nothing.  The call,
  * and everything it calls, performs no cudaMalloc/cudaFree and uses no allocating library
  * routine.
  *
@@ -214,9 +212,7 @@ int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
  * All calls on a device share the one array: two calls whose kernels may overlap on the
  * GPU (different streams, or different contexts of this library on one device) race on
  * it -- order them on one stream or with events.  The array keeps the previous call's
- * contents; each call clears the words that must start at zero (the scan records and the
- * tile counters at its head, with one asynchronous memset on the context's stream) and
- * writes every other word before reading it.  Arguments, outputs and status bits are
+ * contents; each call writes every word before reading it.  Arguments, outputs and status bits are
  * those of aero_group_stats.
  */
 #define AERO_STATIC_MAX_PROMPTS 65536

@@ -1,23 +1,25 @@
 // Stage (a): segmented per-prompt group statistics (Eq. 1; Sec. 3.2; Sec. 4.2
-// Strategies 2-3; Appendix C) in one pass over the rollout arrays.
+// Strategies 2-3; Appendix C) in four launches.
 //
-//   curate_kernel   one block per tile of consecutive prompts.  The tile's rollouts are
-//                   staged in shared memory with coalesced loads; per-prompt steps (counts,
-//                   category, posterior, curation rule, mean/std) run one thread per prompt,
-//                   per-rollout steps (rank among (key, index), keep, advantage, compaction)
-//                   one thread per rollout.  The positions of the kept rollouts in the
-//                   compacted outputs come from a chained scan across tiles (each tile
-//                   publishes its totals, then sums its predecessors' until it meets one
-//                   whose running total is known), so every input is read once and every
-//                   output written once.  The last block to finish reduces the tiles'
-//                   metrics records in a fixed order.
-//   weights_kernel  per-rollout weights, which need the batch totals, and the tails of the
-//                   compacted arrays.
+//   curate_kernel   one warp per share of up to 32 consecutive prompts, eight shares to a tile.
+//                   A warp stages its share's rollouts with coalesced loads (sort words with
+//                   the lengths in shared memory, presence and correctness as bit masks) and runs the per-prompt steps (counts, category, posterior, curation
+//                   rule, mean/std) one lane per prompt and the per-rollout steps (rank among
+//                   (key, index), keep, advantage) one lane per rollout.  Warps never wait for
+//                   one another; each leaves its totals of kept rollouts and tokens, each tile
+//                   its sums of them and its metrics record.
+//   run_prefix_kernel, totals_kernel
+//                   exclusive prefixes of the tiles' totals in two levels (runs of 1024 tiles,
+//                   then the runs), the batch totals, counters and metrics (fixed order).
+//   emit_kernel     the same shares again: compacted ids and token offsets of the kept rollouts
+//                   from the keep flags and the prefixes, per-rollout weights (which need the
+//                   batch totals), and the tails of the compacted arrays.
 //
-// Tiles are handed out through a ticket counter, so a tile only ever waits for tiles taken
-// earlier by blocks that are already running; every wait is bounded and ends with the
-// AERO_ST_TIMEOUT status bit.  A tile whose rollouts do not fit the shared-memory staging
-// area (one huge group) runs the same steps straight from global memory.
+// Splitting where the batch-wide prefix is needed costs a second read of the keep flags and the
+// token offsets (9 bytes per rollout) and saves every wait between blocks: no launch depends on
+// the order in which its blocks run.  A share whose rollouts do not fit the warp's staging area
+// (a huge group, or a rollout of 2^22 tokens or more) runs the first launch's steps straight from
+// global memory, one lane per prompt.
 #include "common.cuh"
 
 #include <mutex>
@@ -25,18 +27,28 @@
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kCap = 2304;             // rollouts a tile can stage in shared memory
-constexpr int kMaxPT = 256;            // prompts per tile: one thread each in the per-prompt steps
-constexpr int kTargetRollouts = 1792;  // mean rollouts per tile the host aims at
+constexpr int kWarps = kThreads / 32;
+constexpr int kBlocksPerSM = 5;
+constexpr int kWCap = 512;             // rollouts a warp can stage
+constexpr int kWChunks = kWCap / 32;
+constexpr int kLenBits = 22;           // staged rollouts are shorter than 2^22 tokens
+constexpr unsigned kLenMask = (1u << kLenBits) - 1u;
+constexpr int kMaxPW = 32;             // prompts per warp: one lane each in the per-prompt steps
+constexpr int kWTarget = 352;          // rollouts per warp the host aims at (mean group size rounded up)
+constexpr int kRunThreads = 256;
+constexpr int kRunTiles = kRunThreads * 4;   // tiles per run of the batch-wide prefix
 constexpr unsigned long long kNone = ~0ull;
-constexpr unsigned long long kFlagAgg = 1ull << 62, kFlagPrefix = 2ull << 62, kValueMask = (1ull << 62) - 1;
-constexpr unsigned long long kSpinLimitNs = 1000000000ull;
 
 struct TilePartial {
   long long present_tok;
   int present_roll, surv;
   int cat[5];
   float abs_adv;
+};
+
+struct RunPartial {
+  long long misc[8];      // present tokens, present rollouts, surviving prompts, 5 categories
+  double abs_adv;
 };
 
 struct Globals {
@@ -48,34 +60,48 @@ struct Globals {
 };
 
 struct Workspace {
-  int* nkept;                        // [P] kept rollouts per prompt (sequence-mean weights)
-  unsigned long long* desc_roll;     // [ntiles] flag | kept rollouts (tile total, then running total)
-  unsigned long long* desc_tok;      // [ntiles] flag | kept tokens
-  unsigned int* ctrl;                // [4] ticket, tiles done, abort
-  TilePartial* part;                 // [ntiles]
-  Globals* glob;                     // [1]
+  int* nkept;              // [P] kept rollouts per prompt (sequence-mean weights)
+  int* share_cnt;          // [ntiles * kWarps] kept rollouts per share
+  long long* share_tok;    // [ntiles * kWarps] kept tokens per share
+  int* tile_cnt;           // [ntiles] kept rollouts per tile, then of the earlier tiles of its run
+  long long* tile_tok;     // [ntiles] kept tokens per tile, then of the earlier tiles of its run
+  TilePartial* part;       // [ntiles]
+  int* run_cnt;            // [nruns] kept rollouts per run of kRunTiles tiles, then of all earlier runs
+  long long* run_tok;      // [nruns] likewise for kept tokens
+  RunPartial* run_part;    // [nruns]
+  Globals* glob;           // [1]
 };
 
-__host__ __device__ inline size_t up256(size_t x) { return (x + 255) / 256 * 256; }
+__host__ __device__ constexpr size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
-inline int prompts_per_tile(int32_t P, int32_t R) {
+inline int prompts_per_warp(int32_t P, int32_t R) {
   const long long avg = P > 0 ? ((long long)R + P - 1) / P : 1;
-  long long pt = kTargetRollouts / (avg > 0 ? avg : 1);
-  return (int)(pt < 1 ? 1 : (pt > kMaxPT ? kMaxPT : pt));
+  long long pw = kWTarget / (avg > 0 ? avg : 1);
+  return (int)(pw < 1 ? 1 : (pw > kMaxPW ? kMaxPW : pw));
 }
 
-inline size_t cleared_bytes(int ntiles) { return up256(sizeof(unsigned long long) * 2 * (size_t)ntiles + 16); }
+constexpr size_t runs_of(size_t ntiles) { return (ntiles + kRunTiles - 1) / kRunTiles; }
+
+constexpr size_t workspace_bytes(size_t P, size_t ntiles) {
+  return up256(sizeof(int) * P) + up256(sizeof(int) * ntiles * kWarps) + up256(sizeof(long long) * ntiles * kWarps) +
+         up256(sizeof(int) * ntiles) + up256(sizeof(long long) * ntiles) + up256(sizeof(TilePartial) * ntiles) +
+         up256(sizeof(int) * runs_of(ntiles)) + up256(sizeof(long long) * runs_of(ntiles)) +
+         up256(sizeof(RunPartial) * runs_of(ntiles)) + up256(sizeof(Globals));
+}
 
 inline Workspace carve(void* ws, int32_t P, int ntiles) {
   char* p = static_cast<char*>(ws);
   Workspace w;
-  // the scan records and the counters are contiguous: one memset clears them before each launch
-  w.desc_roll = reinterpret_cast<unsigned long long*>(p);
-  w.desc_tok = w.desc_roll + ntiles;
-  w.ctrl = reinterpret_cast<unsigned int*>(w.desc_tok + ntiles);
-  p += cleared_bytes(ntiles);
-  w.nkept = reinterpret_cast<int*>(p);            p += up256(sizeof(int) * (size_t)P);
-  w.part = reinterpret_cast<TilePartial*>(p);     p += up256(sizeof(TilePartial) * (size_t)ntiles);
+  w.nkept = reinterpret_cast<int*>(p);              p += up256(sizeof(int) * (size_t)P);
+  w.share_cnt = reinterpret_cast<int*>(p);          p += up256(sizeof(int) * (size_t)ntiles * kWarps);
+  w.share_tok = reinterpret_cast<long long*>(p);    p += up256(sizeof(long long) * (size_t)ntiles * kWarps);
+  w.tile_cnt = reinterpret_cast<int*>(p);           p += up256(sizeof(int) * (size_t)ntiles);
+  w.tile_tok = reinterpret_cast<long long*>(p);     p += up256(sizeof(long long) * (size_t)ntiles);
+  w.part = reinterpret_cast<TilePartial*>(p);       p += up256(sizeof(TilePartial) * (size_t)ntiles);
+  const size_t nruns = runs_of((size_t)ntiles);
+  w.run_cnt = reinterpret_cast<int*>(p);            p += up256(sizeof(int) * nruns);
+  w.run_tok = reinterpret_cast<long long*>(p);      p += up256(sizeof(long long) * nruns);
+  w.run_part = reinterpret_cast<RunPartial*>(p);    p += up256(sizeof(RunPartial) * nruns);
   w.glob = reinterpret_cast<Globals*>(p);
   return w;
 }
@@ -89,18 +115,10 @@ __device__ __forceinline__ uint32_t default_key(uint64_t seed, uint32_t i) {
   return (uint32_t)(z >> 32);
 }
 
-__device__ __forceinline__ unsigned long long ld_acquire(const unsigned long long* p) {
-  unsigned long long v;
-  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_release(unsigned long long* p, unsigned long long v) {
-  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-__device__ __forceinline__ unsigned long long timer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
+// Token count of rollout i as the stage uses it: negative lengths (bad offsets) count as 0 and
+// a length is capped at 2^31 - 1.
+__device__ __forceinline__ int clamped_len(long long len) {
+  return len > 0 ? (int)(len < 0x7fffffffLL ? len : 0x7fffffffLL) : 0;
 }
 
 struct Args {
@@ -127,120 +145,6 @@ struct Args {
   float* metrics;
   uint32_t* status;
 };
-
-// Per-prompt state of a tile (shared memory, one entry per prompt of the tile).
-struct PromptState {
-  int lo[kMaxPT + 1];        // rollout range of each prompt, relative to the tile's first rollout
-  unsigned nc[kMaxPT];       // present rollouts | correct ones << 16   (staged path)
-  unsigned kb[kMaxPT];       // kept rollouts | kept correct ones << 16 (staged path)
-  int quota[kMaxPT];
-  uint8_t mode[kMaxPT];      // 0 keep all present, 1 keep none, 2 select by rank
-  uint8_t reject[kMaxPT];    // 1: select among the incorrect only; 2: among the correct only; 0: among all
-  uint8_t uniform[kMaxPT];
-  float ut[kMaxPT];
-  float mu[kMaxPT];
-  float inv[kMaxPT];
-  int nk[kMaxPT];            // global path: kept rollouts, then their exclusive prefix inside the tile
-  long long ktok[kMaxPT];    // global path: kept tokens, then their exclusive prefix inside the tile
-};
-
-// Per-rollout staging of a tile.  `ck` orders the candidates of a selection:
-// correct << 63 | key << 16 | local index for a present rollout, all ones for an absent one, so
-// that in a group that selects among its incorrect rollouts no correct one ever compares
-// smaller.  After the selection the same words hold a kept rollout's token offset inside its
-// 32-rollout chunk, and `len` its position among the chunk's kept rollouts.
-constexpr int kChunks = kCap / 32;
-struct RolloutStage {
-  unsigned long long ck[kCap];
-  int len[kCap];
-  uint16_t pid[kCap];
-  uint8_t flag[kCap];        // bit 0 present, bit 1 correct, bit 2 kept
-  long long chunk_tok[kChunks];   // kept tokens per chunk, then their exclusive prefix inside the tile
-  int chunk_cnt[kChunks];
-};
-
-struct TileShared {
-  PromptState ps;
-  RolloutStage rs;
-  TilePartial red[kThreads / 32];
-  long long warp_tok[kThreads / 32];
-  int warp_cnt[kThreads / 32];
-  long long base_tok;
-  int base_roll;
-  int tile;
-  int failed;
-};
-
-__device__ __forceinline__ bool aborted(const Workspace& ws) {
-  return *reinterpret_cast<volatile unsigned int*>(ws.ctrl + 2) != 0;
-}
-
-// Running totals of the kept rollouts and kept tokens of all tiles before `tile` (warp 0).
-__device__ bool scan_predecessors(const Workspace& ws, int tile, int lane, int* excl_roll, long long* excl_tok) {
-  unsigned long long sum_r = 0, sum_t = 0;
-  bool done_r = false, done_t = false;
-  const unsigned long long t0 = timer_ns();
-  for (int base = tile - 1; base >= 0 && !(done_r && done_t); base -= 32) {
-    const int idx = base - lane;
-    unsigned long long vr = kFlagPrefix, vt = kFlagPrefix;      // tiles before the first: running total 0
-    unsigned spins = 0;
-    while (true) {
-      if (idx >= 0) { vr = ld_acquire(ws.desc_roll + idx); vt = ld_acquire(ws.desc_tok + idx); }
-      if (__all_sync(0xffffffffu, (vr >> 62) != 0 && (vt >> 62) != 0)) break;
-      if ((++spins & 63u) == 0) {
-        const bool give_up = aborted(ws) || timer_ns() - t0 > kSpinLimitNs;
-        if (__any_sync(0xffffffffu, give_up)) return false;
-      }
-      __nanosleep(200);
-    }
-    if (!done_r) {
-      const unsigned m = __ballot_sync(0xffffffffu, (vr >> 62) == 2);
-      const int first = m ? __ffs(m) - 1 : 31;
-      unsigned long long v = lane <= first ? (vr & kValueMask) : 0;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      sum_r += v;
-      done_r = m != 0;
-    }
-    if (!done_t) {
-      const unsigned m = __ballot_sync(0xffffffffu, (vt >> 62) == 2);
-      const int first = m ? __ffs(m) - 1 : 31;
-      unsigned long long v = lane <= first ? (vt & kValueMask) : 0;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-      sum_t += v;
-      done_t = m != 0;
-    }
-  }
-  *excl_roll = (int)sum_r;
-  *excl_tok = (long long)sum_t;
-  return true;
-}
-
-// Publish the tile's totals, sum the predecessors', publish the running totals (warp 0).
-// Leaves the totals of all earlier tiles in sh.base_roll / sh.base_tok.
-__device__ void chain_tile(const Workspace& ws, TileShared& sh, int tile, int tile_cnt, long long tile_tok, uint32_t& st) {
-  const int lane = threadIdx.x;
-  if (lane == 0 && tile > 0) {
-    st_release(ws.desc_roll + tile, kFlagAgg | (unsigned long long)tile_cnt);
-    st_release(ws.desc_tok + tile, kFlagAgg | (unsigned long long)tile_tok);
-  }
-  int excl_roll = 0;
-  long long excl_tok = 0;
-  const bool ok = scan_predecessors(ws, tile, lane, &excl_roll, &excl_tok);
-  if (lane == 0) {
-    if (ok) {
-      st_release(ws.desc_roll + tile, kFlagPrefix | (unsigned long long)(excl_roll + tile_cnt));
-      st_release(ws.desc_tok + tile, kFlagPrefix | (unsigned long long)(excl_tok + tile_tok));
-    } else {
-      atomicExch(ws.ctrl + 2, 1u);
-      st |= AERO_ST_TIMEOUT;
-    }
-    sh.failed = ok ? 0 : 1;
-    sh.base_roll = excl_roll;
-    sh.base_tok = excl_tok;
-  }
-}
 
 // Category, posterior and curation rule of one prompt from its counts (Appendix C; Sec. 4.2).
 struct Rule {
@@ -284,232 +188,272 @@ __device__ __forceinline__ Rule decide(const Args& a, int p, int n, int c) {
   return r;
 }
 
-// Metrics record of the tile: shuffle tree per warp, warps added in order by thread 0.
-__device__ __forceinline__ void reduce_partial(TileShared& sh, TilePartial mine) {
+// What the rollouts of one prompt need to know about it (shared memory, one entry per prompt of
+// a warp's share).
+struct PromptRule {
+  float mu, inv;
+  unsigned range;      // first rollout | one past the last << 16, relative to the share's first rollout
+  unsigned sel;        // mode (0 keep all present, 1 keep none, 2 select by rank) | reject << 2 | quota << 4
+};
+
+// Staging of one warp's share.  `ck` orders the candidates of a selection and carries the
+// rollout's length: correct << 63 | key << 31 | local index << 22 | length for a present rollout,
+// all ones for an absent one, so that in a group that selects among its incorrect rollouts no
+// correct one ever compares smaller.  One bit per rollout in `pmask` (present) and `cmask` (present and correct), one word
+// per chunk of 32 rollouts.
+struct WarpStage {
+  unsigned long long ck[kWCap];
+  PromptRule rule[kMaxPW];
+  unsigned pmask[kWChunks], cmask[kWChunks];
+  uint8_t pid[kWCap];        // which prompt of the share owns the rollout
+};
+
+struct BlockShared {
+  WarpStage stage[kWarps];
+  TilePartial red[kWarps];
+  long long share_tok[kWarps];
+  int share_cnt[kWarps];
+};
+
+// A warp's share of a tile: prompts [p0, p0 + np), their rollouts [r0, r0 + nroll); lane q holds
+// the rollout range [lo, hi) of prompt p0 + q, relative to r0 (empty for q >= np).
+struct Share {
+  int p0, np;
+  int r0, nroll;
+  int lo, hi;
+};
+
+// Reads the share's group offsets, clamping them into [0, R] and into non-decreasing order if
+// they are bad (which also raises AERO_ST_BAD_OFFSETS).
+__device__ __forceinline__ Share load_share(const Args& a, int share, int pw, uint32_t& st) {
+  const int lane = threadIdx.x & 31;
+  Share sh;
+  sh.p0 = share * pw;
+  sh.np = max(0, min(pw, a.P - sh.p0));
+  sh.r0 = sh.nroll = sh.lo = sh.hi = 0;
+  if (sh.np == 0) return sh;
+  const int v = lane < sh.np ? a.go[sh.p0 + lane] : 0;
+  const int end = a.go[sh.p0 + sh.np];
+  int prev = __shfl_up_sync(0xffffffffu, v, 1);
+  if (lane == 0) prev = sh.p0 > 0 ? a.go[sh.p0 - 1] : v;
+  bool bad = lane < sh.np && (v < 0 || v > a.R || v < prev);
+  if (lane == sh.np - 1) bad = bad || end < v || end > a.R || end < 0;
+  int lo = min(max(v, 0), a.R);
+  int last = min(max(end, 0), a.R);
+  if (__any_sync(0xffffffffu, bad)) {
+    st |= AERO_ST_BAD_OFFSETS;
+    if (lane >= sh.np) lo = 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, lo, o);
+      if (lane >= o) lo = max(lo, u);
+    }
+    last = max(last, __shfl_sync(0xffffffffu, lo, sh.np - 1));
+  }
+  int hi = __shfl_down_sync(0xffffffffu, lo, 1);
+  if (lane >= sh.np - 1) hi = last;
+  if (lane >= sh.np) lo = last;
+  sh.r0 = __shfl_sync(0xffffffffu, lo, 0);
+  sh.nroll = last - sh.r0;
+  sh.lo = lo - sh.r0;
+  sh.hi = hi - sh.r0;
+  return sh;
+}
+
+// Metrics record of a warp's share: integer fields by warp reduction, the float by a shuffle tree
+// (fixed order).
+__device__ __forceinline__ TilePartial warp_partial(TilePartial mine) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     mine.present_tok += __shfl_xor_sync(0xffffffffu, mine.present_tok, o);
-    mine.present_roll += __shfl_xor_sync(0xffffffffu, mine.present_roll, o);
-    mine.surv += __shfl_xor_sync(0xffffffffu, mine.surv, o);
-#pragma unroll
-    for (int k = 0; k < 5; ++k) mine.cat[k] += __shfl_xor_sync(0xffffffffu, mine.cat[k], o);
     mine.abs_adv += __shfl_xor_sync(0xffffffffu, mine.abs_adv, o);
   }
-  if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = mine;
-}
-__device__ __forceinline__ TilePartial sum_partials(const TileShared& sh) {
-  TilePartial tot = {};
-  for (int k = 0; k < kThreads / 32; ++k) {
-    tot.present_tok += sh.red[k].present_tok; tot.present_roll += sh.red[k].present_roll; tot.surv += sh.red[k].surv;
-    for (int c = 0; c < 5; ++c) tot.cat[c] += sh.red[k].cat[c];
-    tot.abs_adv += sh.red[k].abs_adv;
-  }
-  return tot;
+  mine.present_roll = __reduce_add_sync(0xffffffffu, mine.present_roll);
+  mine.surv = __reduce_add_sync(0xffffffffu, mine.surv);
+#pragma unroll
+  for (int k = 0; k < 5; ++k) mine.cat[k] = __reduce_add_sync(0xffffffffu, mine.cat[k]);
+  return mine;
 }
 
-// A tile whose rollouts fit the staging area.  Rewards enter as the bit r > 0.5 (they must be
-// exactly 0 or 1; anything else raises AERO_ST_BAD_REWARD), so per-prompt sums are counts,
-// gathered with shared-memory atomics, and mean and deviation are closed forms of the counts.
-__device__ void run_tile_staged(const Args& a, const Workspace& ws, TileShared& sh, int tile, int p0, int npt, int r0,
-                                int nroll, uint32_t& st) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  PromptState& ps = sh.ps;
-  RolloutStage& rs = sh.rs;
+// Set bits of a chunked bit mask inside the rollout range [lo, hi).
+__device__ __forceinline__ int range_popc(const unsigned* mask, int lo, int hi) {
+  int cnt = 0;
+  if (hi > lo) {
+    const int w0 = lo >> 5, w1 = (hi - 1) >> 5;
+    for (int w = w0; w <= w1; ++w) {
+      unsigned m = mask[w];
+      if (w == w0) m &= 0xffffffffu << (lo & 31);
+      if (w == w1) m &= 0xffffffffu >> (31 - ((hi - 1) & 31));
+      cnt += __popc(m);
+    }
+  }
+  return cnt;
+}
+
+// Mean and reciprocal deviation of a group's base set from its counts (Eq. 1 with binary
+// rewards; posterior mean and Bernoulli deviation for a uniform group).
+__device__ __forceinline__ void group_moments(const Args& a, const Rule& ru, int nb, int cb, float* mu_out, float* inv_out) {
+  float mu = 0.f, sd = 0.f;
+  if (ru.uniform) {
+    mu = ru.ut;
+    sd = sqrtf(mu * (1.f - mu));
+  } else if (nb > 0) {
+    mu = (float)cb / (float)nb;
+    const float d1 = 1.f - mu;
+    sd = sqrtf(((float)cb * d1 * d1 + (float)(nb - cb) * mu * mu) / (float)nb);
+  }
+  *mu_out = mu;
+  *inv_out = 1.f / (sd + a.cfg.eps_std);
+}
+
+// A share whose rollouts fit the warp's staging area and are shorter than 2^22 tokens each.
+// Rewards enter as the bit r > 0.5 (they must be exactly 0 or 1; anything else raises
+// AERO_ST_BAD_REWARD), so per-prompt sums are bit counts and mean and deviation are closed
+// forms of the counts; the number of rollouts a selection keeps is known from the rule alone,
+// so the per-prompt outputs are written before any rollout is ranked.  Returns false, with
+// nothing written, if a rollout is too long for the staging word; else the share's kept
+// rollouts and tokens.
+__device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws, WarpStage& S, const Share& sh,
+                                              TilePartial& mine, uint32_t& st, int* cnt_out, long long* tok_out) {
+  const int lane = threadIdx.x & 31;
+  const int r0 = sh.r0, nroll = sh.nroll;
 
   // ---- which prompt owns which rollout ----
-  if (tid < npt) {
-    for (int j = ps.lo[tid]; j < ps.lo[tid + 1]; ++j) rs.pid[j] = (uint16_t)tid;
-    ps.nc[tid] = 0;
-    ps.kb[tid] = 0;
-  }
-  __syncthreads();
+  if (lane < sh.np)
+    for (int j = sh.lo; j < sh.hi; ++j) S.pid[j] = (uint8_t)lane;
 
-  // ---- stage the rollouts (coalesced) and count per prompt ----
-  TilePartial mine = {};
-  for (int j = tid; j < nroll; j += kThreads) {
+  // ---- stage the rollouts (coalesced), one bit each for present and correct ----
+  uint32_t bits = 0;
+  long long ptok = 0;
+  bool too_long = false;
+  for (int c = 0; c * 32 < nroll; ++c) {
+    const int j = c * 32 + lane;
     const int i = r0 + j;
-    const bool pres = a.keep_in ? a.keep_in[i] != 0 : true;
-    const float r = a.reward[i];
-    const long long len = a.cs[i + 1] - a.cs[i];
-    const bool corr = r > 0.5f;
-    unsigned long long ck = kNone;
-    if (pres) {
-      if (r != 0.f && r != 1.f) st |= AERO_ST_BAD_REWARD;
-      if (len < 0) st |= AERO_ST_BAD_OFFSETS;
-      if (len == 0) st |= AERO_ST_EMPTY_ROLLOUT;
-      const uint32_t key = a.key ? a.key[i] : default_key(a.cfg.seed, (uint32_t)i);
-      ck = (corr ? 1ull << 63 : 0ull) | ((unsigned long long)key << 16) | (unsigned)j;
-      atomicAdd(&ps.nc[rs.pid[j]], corr ? 0x10001u : 1u);
-      mine.present_tok += len > 0 ? len : 0;
-      mine.present_roll += 1;
+    bool pres = false, corr = false;
+    if (j < nroll) {
+      const float r = a.reward[i];
+      const long long len = a.cs[i + 1] - a.cs[i];
+      pres = a.keep_in ? a.keep_in[i] != 0 : true;
+      corr = r > 0.5f;
+      unsigned long long ck = kNone;
+      if (pres) {
+        if (r != 0.f && r != 1.f) bits |= AERO_ST_BAD_REWARD;
+        if (len < 0) bits |= AERO_ST_BAD_OFFSETS;
+        if (len == 0) bits |= AERO_ST_EMPTY_ROLLOUT;
+        too_long = too_long || len >= (1ll << kLenBits);
+        const uint32_t key = a.key ? a.key[i] : default_key(a.cfg.seed, (uint32_t)i);
+        const unsigned l = (unsigned)clamped_len(len) & kLenMask;
+        ck = (corr ? 1ull << 63 : 0ull) | ((unsigned long long)key << 31) | ((unsigned long long)j << kLenBits) | l;
+        ptok += l;
+      }
+      S.ck[j] = ck;
     }
-    rs.ck[j] = ck;
-    rs.len[j] = len > 0 ? (int)(len < 0x7fffffffLL ? len : 0x7fffffffLL) : 0;
-    rs.flag[j] = (uint8_t)((pres ? 1 : 0) | (corr ? 2 : 0));
+    const unsigned pm = __ballot_sync(0xffffffffu, pres);
+    const unsigned cm = __ballot_sync(0xffffffffu, pres && corr);
+    if (lane == 0) { S.pmask[c] = pm; S.cmask[c] = cm; }
   }
-  __syncthreads();
+  if (__any_sync(0xffffffffu, too_long)) return false;
+  st |= bits;
+  mine.present_tok = ptok;
+  __syncwarp();
 
-  // ---- per prompt: category, posterior, curation rule ----
-  if (tid < npt) {
-    const int p = p0 + tid;
-    const int n = (int)(ps.nc[tid] & 0xffffu), c = (int)(ps.nc[tid] >> 16);
+  // ---- per prompt: counts, category, posterior, curation rule, moments of the base set ----
+  if (lane < sh.np) {
+    const int p = sh.p0 + lane;
+    const int n = a.keep_in ? range_popc(S.pmask, sh.lo, sh.hi) : sh.hi - sh.lo;
+    const int c = range_popc(S.cmask, sh.lo, sh.hi);
     const Rule ru = decide(a, p, n, c);
     a.cat[p] = (uint8_t)ru.category;
     a.u_tilde[p] = ru.ut;
     a.alpha_out[p] = ru.al;
     a.beta_out[p] = ru.be;
-    ps.mode[tid] = (uint8_t)ru.mode;
-    ps.reject[tid] = (uint8_t)ru.reject;
-    // every incorrect rollout orders before every correct one: when the correct ones are the
-    // candidates, the n - c incorrect ones are counted by each rank and the quota allows for them
-    ps.quota[tid] = (int)ru.quota + (ru.reject == 2 ? n - c : 0);
-    ps.uniform[tid] = ru.uniform ? 1 : 0;
-    ps.ut[tid] = ru.ut;
-    mine.cat[ru.category] = 1;
-  }
-  __syncthreads();
-
-  // ---- per rollout: keep decision (rank among the group's candidates) ----
-  for (int j = tid; j < nroll; j += kThreads) {
-    const int q = rs.pid[j];
-    const int mode = ps.mode[q];
-    const uint8_t f = rs.flag[j];
-    bool kp = (f & 1) && mode != 1;
-    const int rej = ps.reject[q];
-    if (kp && mode == 2 && !(rej == 1 && (f & 2)) && !(rej == 2 && !(f & 2))) {
-      const unsigned long long mykey = rs.ck[j];
-      const int lo = ps.lo[q], hi = ps.lo[q + 1];
-      int rank = 0;
-#pragma unroll 4
-      for (int k = lo; k < hi; ++k) rank += rs.ck[k] < mykey ? 1 : 0;
-      kp = rank < ps.quota[q];
+    // keys with the index appended are distinct, so a selection keeps exactly its quota
+    int nk = n, ck = c;
+    if (ru.mode == 1) { nk = 0; ck = 0; }
+    else if (ru.mode == 2) {
+      const int q = (int)ru.quota;
+      if (ru.reject == 0) { nk = q; ck = c > 0 ? q : 0; }
+      else if (ru.reject == 1) { nk = c + q; ck = c; }
+      else { nk = (n - c) + q; ck = q; }
     }
-    if (kp) {
-      rs.flag[j] = f | 4;
-      atomicAdd(&ps.kb[q], (f & 2) ? 0x10001u : 1u);
-    }
-  }
-  __syncthreads();
-
-  // ---- per prompt: mean and deviation of the base set; per chunk of 32 rollouts: kept counts and tokens ----
-  if (tid < npt) {
-    const int p = p0 + tid;
-    const int nk = (int)(ps.kb[tid] & 0xffffu), ck = (int)(ps.kb[tid] >> 16);
     const bool over_kept = a.cfg.stats_over == AERO_STATS_KEPT;
-    const int nb = over_kept ? nk : (int)(ps.nc[tid] & 0xffffu);
-    const int cb = over_kept ? ck : (int)(ps.nc[tid] >> 16);
-    float mu = 0.f, sd = 0.f;
-    if (ps.uniform[tid]) {
-      mu = ps.ut[tid];
-      sd = sqrtf(mu * (1.f - mu));
-    } else if (nb > 0) {
-      mu = (float)cb / (float)nb;
-      const float d1 = 1.f - mu;
-      sd = sqrtf(((float)cb * d1 * d1 + (float)(nb - cb) * mu * mu) / (float)nb);
-    }
-    const float inv = 1.f / (sd + a.cfg.eps_std);
-    ps.mu[tid] = mu;
-    ps.inv[tid] = inv;
+    float mu, inv;
+    group_moments(a, ru, over_kept ? nk : n, over_kept ? ck : c, &mu, &inv);
     a.gmask[p] = nk > 0 ? 1 : 0;
     if (a.cfg.agg != AERO_TOKEN_MEAN) ws.nkept[p] = nk;
+    PromptRule pr;
+    pr.mu = mu;
+    pr.inv = inv;
+    pr.range = (unsigned)sh.lo | ((unsigned)sh.hi << 16);
+    // every incorrect rollout orders before every correct one: when the correct ones are the
+    // candidates, the n - c incorrect ones are counted by each rank and the quota allows for them
+    pr.sel = (unsigned)ru.mode | ((unsigned)ru.reject << 2) | ((unsigned)((int)ru.quota + (ru.reject == 2 ? n - c : 0)) << 4);
+    S.rule[lane] = pr;
+    mine.present_roll = n;
+#pragma unroll
+    for (int k = 0; k < 5; ++k) mine.cat[k] = ru.category == k ? 1 : 0;
     mine.surv = nk > 0 ? 1 : 0;
     mine.abs_adv = ((float)ck * fabsf(1.f - mu) + (float)(nk - ck) * fabsf(mu)) * inv;
   }
-  for (int j0 = warp * 32; j0 < nroll; j0 += kThreads) {     // whole warps: the scan is warp-wide
-    const int j = j0 + lane;
-    const bool kp = j < nroll && (rs.flag[j] & 4);
-    const unsigned kept_mask = __ballot_sync(0xffffffffu, kp);
-    long long tok = kp ? rs.len[j] : 0;
-    if (__reduce_max_sync(0xffffffffu, (unsigned)tok) < (1u << 26)) {      // 32 lengths below 2^26: a 32-bit scan
-      unsigned t32 = (unsigned)tok;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned t2 = __shfl_up_sync(0xffffffffu, t32, o);
-        if (lane >= o) t32 += t2;
-      }
-      tok = t32;
-    } else {
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const long long t2 = __shfl_up_sync(0xffffffffu, tok, o);
-        if (lane >= o) tok += t2;
-      }
-    }
-    if (kp) {
-      rs.ck[j] = (unsigned long long)(tok - rs.len[j]);
-      rs.len[j] = __popc(kept_mask & ((1u << lane) - 1u));
-    }
-    if (lane == 31) { rs.chunk_cnt[j0 >> 5] = __popc(kept_mask); rs.chunk_tok[j0 >> 5] = tok; }
-  }
-  reduce_partial(sh, mine);
-  __syncthreads();
+  __syncwarp();
 
-  // ---- warp 0: exclusive prefixes over the chunks, then the chained scan across tiles; meanwhile
-  // the other warps write what does not depend on it: advantage and keep flag per rollout ----
-  if (tid >= 32) {
-    for (int j = tid - 32; j < nroll; j += kThreads - 32) {
-      const int q = rs.pid[j];
-      const uint8_t f = rs.flag[j];
-      const bool kp = (f & 4) != 0;
-      a.adv[r0 + j] = kp ? (((f & 2) ? 1.f : 0.f) - ps.mu[q]) * ps.inv[q] : 0.f;
+  // ---- per rollout: keep decision (rank among the group's candidates), advantage ----
+  int cnt = 0;
+  long long tok = 0;
+  for (int c = 0; c * 32 < nroll; ++c) {
+    const int j = c * 32 + lane;
+    const bool valid = j < nroll;
+    const PromptRule pr = S.rule[valid ? S.pid[j] : 0];
+    const unsigned long long mykey = S.ck[j & (kWCap - 1)];
+    const bool pres = (S.pmask[c] >> lane) & 1u;
+    const bool corr = (S.cmask[c] >> lane) & 1u;
+    const int mode = (int)(pr.sel & 3u), rej = (int)((pr.sel >> 2) & 3u);
+    bool kp = pres && mode != 1;
+    const bool ranked = kp && mode == 2 && !(rej == 1 && corr) && !(rej == 2 && !corr);
+    // the loop runs as long as the longest group among the chunk's ranked rollouts, the same for all lanes
+    const int lo = (int)(pr.range & 0xffffu);
+    const int span = ranked ? (int)(pr.range >> 16) - lo : 0;
+    const int longest = (int)__reduce_max_sync(0xffffffffu, (unsigned)span);
+    if (longest > 0) {
+      const unsigned long long* grp = S.ck + lo;
+      int rank = 0;
+#pragma unroll 4
+      for (int d = 0; d < longest; ++d)
+        if (d < span) rank += grp[d] < mykey ? 1 : 0;
+      if (ranked) kp = rank < (int)(pr.sel >> 4);
+    }
+    const unsigned km = __ballot_sync(0xffffffffu, kp);
+    if (valid) {
+      a.adv[r0 + j] = kp ? ((corr ? 1.f : 0.f) - pr.mu) * pr.inv : 0.f;
       a.keep[r0 + j] = kp ? 1 : 0;
     }
-  } else {
-    const int nchunks = (nroll + 31) >> 5;
-    int run_cnt = 0;
-    long long run_tok = 0;
-    for (int c0 = 0; c0 < nchunks; c0 += 32) {
-      const int c = c0 + lane;
-      int cnt = c < nchunks ? rs.chunk_cnt[c] : 0;
-      long long tok = c < nchunks ? rs.chunk_tok[c] : 0;
-      const int my_cnt = cnt;
-      const long long my_tok = tok;
+    cnt += __popc(km);
+    tok += kp ? (long long)((unsigned)mykey & kLenMask) : 0ll;
+  }
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int c2 = __shfl_up_sync(0xffffffffu, cnt, o);
-        const long long t2 = __shfl_up_sync(0xffffffffu, tok, o);
-        if (lane >= o) { cnt += c2; tok += t2; }
-      }
-      if (c < nchunks) { rs.chunk_cnt[c] = run_cnt + cnt - my_cnt; rs.chunk_tok[c] = run_tok + tok - my_tok; }
-      run_cnt += __shfl_sync(0xffffffffu, cnt, 31);
-      run_tok += __shfl_sync(0xffffffffu, tok, 31);
-    }
-    if (tid == 0) ws.part[tile] = sum_partials(sh);
-    chain_tile(ws, sh, tile, run_cnt, run_tok, st);
-  }
-  __syncthreads();
-  const bool failed = sh.failed != 0;
-  const int base_roll = sh.base_roll;
-  const long long base_tok = sh.base_tok;
-
-  // ---- per kept rollout: compacted id and token offset ----
-  if (!failed) {
-    for (int j = tid; j < nroll; j += kThreads) {
-      if (!(rs.flag[j] & 4)) continue;
-      const int pos = base_roll + rs.chunk_cnt[j >> 5] + rs.len[j];
-      a.kept_ids[pos] = r0 + j;
-      a.kept_tok_off[pos] = base_tok + rs.chunk_tok[j >> 5] + (long long)rs.ck[j];
-    }
-  }
+  for (int o = 16; o > 0; o >>= 1) tok += __shfl_xor_sync(0xffffffffu, tok, o);
+  *cnt_out = cnt;
+  *tok_out = tok;
+  return true;
 }
 
-// A tile whose rollouts exceed the staging area (a very large group): the same steps with
-// one thread per prompt walking the caller's arrays.
-__device__ void run_tile_global(const Args& a, const Workspace& ws, TileShared& sh, int tile, int p0, int npt, int r0,
-                                uint32_t& st) {
-  const int tid = threadIdx.x;
-  PromptState& ps = sh.ps;
+// A share whose rollouts exceed the staging area (a very large group): the same steps with one
+// lane per prompt walking the caller's arrays.
+__device__ void curate_global(const Args& a, const Workspace& ws, const Share& sh, TilePartial& mine, uint32_t& st,
+                              int* cnt_out, long long* tok_out) {
+  const int lane = threadIdx.x & 31;
+  const int r0 = sh.r0;
   auto present = [&](int j) { return a.keep_in ? a.keep_in[r0 + j] != 0 : true; };
-  auto length = [&](int j) { const long long l = a.cs[r0 + j + 1] - a.cs[r0 + j]; return l > 0 ? l : 0; };
   auto order_key = [&](int j) {
     if (!present(j)) return kNone;
     const uint32_t key = a.key ? a.key[r0 + j] : default_key(a.cfg.seed, (uint32_t)(r0 + j));
     return ((unsigned long long)key << 32) | (unsigned)j;
   };
-  TilePartial mine = {};
-  if (tid < npt) {
-    const int p = p0 + tid;
-    const int lo = ps.lo[tid], hi = ps.lo[tid + 1];
+  int nk = 0;
+  long long ktok = 0;
+  if (lane < sh.np) {
+    const int p = sh.p0 + lane;
+    const int lo = sh.lo, hi = sh.hi;
     int n = 0, c = 0;
     for (int j = lo; j < hi; ++j) {
       if (!present(j)) continue;
@@ -519,7 +463,7 @@ __device__ void run_tile_global(const Args& a, const Workspace& ws, TileShared& 
       if (len < 0) st |= AERO_ST_BAD_OFFSETS;
       if (len == 0) st |= AERO_ST_EMPTY_ROLLOUT;
       n += 1; c += r > 0.5f ? 1 : 0;
-      mine.present_tok += len > 0 ? len : 0;
+      mine.present_tok += clamped_len(len);
     }
     mine.present_roll = n;
     const Rule ru = decide(a, p, n, c);
@@ -527,10 +471,10 @@ __device__ void run_tile_global(const Args& a, const Workspace& ws, TileShared& 
     a.u_tilde[p] = ru.ut;
     a.alpha_out[p] = ru.al;
     a.beta_out[p] = ru.be;
-    mine.cat[ru.category] = 1;
+#pragma unroll
+    for (int k = 0; k < 5; ++k) mine.cat[k] = ru.category == k ? 1 : 0;
 
-    int nk = 0, ck = 0;
-    long long ktok = 0;
+    int ck = 0;
     for (int j = lo; j < hi; ++j) {
       const bool corr = a.reward[r0 + j] > 0.5f;
       bool kp = present(j) && ru.mode != 1;
@@ -538,112 +482,203 @@ __device__ void run_tile_global(const Args& a, const Workspace& ws, TileShared& 
         const unsigned long long mykey = order_key(j);
         long long rank = 0;
         for (int k = lo; k < hi; ++k) {
-          const bool ck = a.reward[r0 + k] > 0.5f;
-          if ((ru.reject == 1 && ck) || (ru.reject == 2 && !ck)) continue;
+          const bool other = a.reward[r0 + k] > 0.5f;
+          if ((ru.reject == 1 && other) || (ru.reject == 2 && !other)) continue;
           rank += order_key(k) < mykey ? 1 : 0;
         }
         kp = rank < ru.quota;
       }
       a.keep[r0 + j] = kp ? 1 : 0;
-      if (kp) { nk += 1; ck += corr ? 1 : 0; ktok += length(j); }
+      if (kp) { nk += 1; ck += corr ? 1 : 0; ktok += clamped_len(a.cs[r0 + j + 1] - a.cs[r0 + j]); }
     }
     const bool over_kept = a.cfg.stats_over == AERO_STATS_KEPT;
-    const int nb = over_kept ? nk : n, cb = over_kept ? ck : c;
-    float mu = 0.f, sd = 0.f;
-    if (ru.uniform) {
-      mu = ru.ut;
-      sd = sqrtf(mu * (1.f - mu));
-    } else if (nb > 0) {
-      mu = (float)cb / (float)nb;
-      const float d1 = 1.f - mu;
-      sd = sqrtf(((float)cb * d1 * d1 + (float)(nb - cb) * mu * mu) / (float)nb);
-    }
-    const float inv = 1.f / (sd + a.cfg.eps_std);
+    float mu, inv;
+    group_moments(a, ru, over_kept ? nk : n, over_kept ? ck : c, &mu, &inv);
     for (int j = lo; j < hi; ++j)
       a.adv[r0 + j] = a.keep[r0 + j] ? ((a.reward[r0 + j] > 0.5f ? 1.f : 0.f) - mu) * inv : 0.f;
-    ps.nk[tid] = nk;
-    ps.ktok[tid] = ktok;
     a.gmask[p] = nk > 0 ? 1 : 0;
     if (a.cfg.agg != AERO_TOKEN_MEAN) ws.nkept[p] = nk;
     mine.surv = nk > 0 ? 1 : 0;
     mine.abs_adv = ((float)ck * fabsf(1.f - mu) + (float)(nk - ck) * fabsf(mu)) * inv;
   }
-
-  // tile totals and exclusive prefixes over the tile's prompts (block scan, fixed order)
-  const int lane = tid & 31, warp = tid >> 5;
-  int cnt = tid < npt ? ps.nk[tid] : 0;
-  long long tok = tid < npt ? ps.ktok[tid] : 0;
-  const int my_cnt = cnt;
-  const long long my_tok = tok;
+  *cnt_out = __reduce_add_sync(0xffffffffu, nk);
 #pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int c2 = __shfl_up_sync(0xffffffffu, cnt, o);
-    const long long t2 = __shfl_up_sync(0xffffffffu, tok, o);
-    if (lane >= o) { cnt += c2; tok += t2; }
+  for (int o = 16; o > 0; o >>= 1) ktok += __shfl_xor_sync(0xffffffffu, ktok, o);
+  *tok_out = ktok;
+}
+
+__global__ void __launch_bounds__(kThreads, kBlocksPerSM) curate_kernel(Args a, Workspace ws, int pw) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  BlockShared& bs = *reinterpret_cast<BlockShared*>(smem_raw);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int tile = blockIdx.x;
+  uint32_t st = 0;
+  const Share sh = load_share(a, tile * kWarps + warp, pw, st);
+  TilePartial mine = {};
+  int cnt = 0;
+  long long tok = 0;
+  if (sh.np > 0) {
+    const bool done = sh.nroll <= kWCap && curate_staged(a, ws, bs.stage[warp], sh, mine, st, &cnt, &tok);
+    if (!done) curate_global(a, ws, sh, mine, st, &cnt, &tok);
   }
-  if (lane == 31) { sh.warp_cnt[warp] = cnt; sh.warp_tok[warp] = tok; }
-  reduce_partial(sh, mine);
-  __syncthreads();
-  int wbase_cnt = 0;
-  long long wbase_tok = 0;
-  for (int k = 0; k < warp; ++k) { wbase_cnt += sh.warp_cnt[k]; wbase_tok += sh.warp_tok[k]; }
-  const int excl_cnt = wbase_cnt + cnt - my_cnt;
-  const long long excl_tok = wbase_tok + tok - my_tok;
-  if (tid < 32) {
-    int tile_cnt = 0;
-    long long tile_tok = 0;
-    for (int k = 0; k < kThreads / 32; ++k) { tile_cnt += sh.warp_cnt[k]; tile_tok += sh.warp_tok[k]; }
-    if (tid == 0) ws.part[tile] = sum_partials(sh);
-    chain_tile(ws, sh, tile, tile_cnt, tile_tok, st);
+  mine = warp_partial(mine);
+  if (lane == 0) {
+    bs.red[warp] = mine;
+    bs.share_cnt[warp] = cnt;
+    bs.share_tok[warp] = tok;
+    ws.share_cnt[tile * kWarps + warp] = cnt;
+    ws.share_tok[tile * kWarps + warp] = tok;
   }
+  st = __reduce_or_sync(0xffffffffu, st);
+  if (lane == 0) aero_raise(a.status, st);
   __syncthreads();
-  if (tid < npt && !sh.failed) {
-    int pos = sh.base_roll + excl_cnt;
-    long long toff = sh.base_tok + excl_tok;
-    for (int j = ps.lo[tid]; j < ps.lo[tid + 1]; ++j) {
-      if (!a.keep[r0 + j]) continue;
-      a.kept_ids[pos] = r0 + j;
-      a.kept_tok_off[pos] = toff;
-      pos += 1;
-      toff += length(j);
+  // the tile's record: its warps added in order
+  if (threadIdx.x == 0) {
+    TilePartial tot = {};
+    int tcnt = 0;
+    long long ttok = 0;
+    for (int k = 0; k < kWarps; ++k) {
+      tot.present_tok += bs.red[k].present_tok; tot.present_roll += bs.red[k].present_roll; tot.surv += bs.red[k].surv;
+      for (int c = 0; c < 5; ++c) tot.cat[c] += bs.red[k].cat[c];
+      tot.abs_adv += bs.red[k].abs_adv;
+      tcnt += bs.share_cnt[k];
+      ttok += bs.share_tok[k];
     }
+    ws.part[tile] = tot;
+    ws.tile_cnt[tile] = tcnt;
+    ws.tile_tok[tile] = ttok;
   }
 }
 
-// Fixed-order reduction of the tiles' metrics records and the batch totals (one block).
-__device__ void finish_batch(const Args& a, const Workspace& ws, int ntiles) {
-  __shared__ long long s_misc[kThreads / 32][8];
-  __shared__ double s_abs[kThreads / 32];
-  const int tid = threadIdx.x;
-  long long misc[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // present tokens, present rollouts, surviving prompts, 5 categories
-  double aabs = 0.0;
-  for (int t = tid; t < ntiles; t += kThreads) {
-    const TilePartial q = ws.part[t];
-    misc[0] += q.present_tok; misc[1] += q.present_roll; misc[2] += q.surv;
-    for (int k = 0; k < 5; ++k) misc[3 + k] += q.cat[k];
-    aabs += (double)q.abs_adv;
+// Level 1 of the batch-wide prefix: one block per run of kRunTiles consecutive tiles (each
+// thread owns four of them) turns the run's tile totals into exclusive prefixes inside the run
+// and leaves the run's totals and the sum of its metrics records, all sums in a fixed order.
+__global__ void __launch_bounds__(kRunThreads) run_prefix_kernel(Workspace ws, int ntiles) {
+  __shared__ long long s_tok[kRunThreads / 32];
+  __shared__ int s_cnt[kRunThreads / 32];
+  __shared__ RunPartial s_part[kRunThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int t0 = min(blockIdx.x * kRunTiles + tid * 4, ntiles), t1 = min(t0 + 4, ntiles);
+  int c[4];
+  long long k[4];
+  int cnt = 0;
+  long long tok = 0;
+  RunPartial mine = {};
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    c[e] = 0; k[e] = 0;
+    if (t0 + e < t1) {
+      c[e] = ws.tile_cnt[t0 + e];
+      k[e] = ws.tile_tok[t0 + e];
+      const TilePartial q = ws.part[t0 + e];
+      mine.misc[0] += q.present_tok; mine.misc[1] += q.present_roll; mine.misc[2] += q.surv;
+#pragma unroll
+      for (int m = 0; m < 5; ++m) mine.misc[3 + m] += q.cat[m];
+      mine.abs_adv += (double)q.abs_adv;
+    }
+    cnt += c[e];
+    tok += k[e];
+  }
+  int icnt = cnt;
+  long long itok = tok;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int c2 = __shfl_up_sync(0xffffffffu, icnt, o);
+    const long long t2 = __shfl_up_sync(0xffffffffu, itok, o);
+    if (lane >= o) { icnt += c2; itok += t2; }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
-    aabs += __shfl_xor_sync(0xffffffffu, aabs, o);
+    mine.abs_adv += __shfl_xor_sync(0xffffffffu, mine.abs_adv, o);
 #pragma unroll
-    for (int k = 0; k < 8; ++k) misc[k] += __shfl_xor_sync(0xffffffffu, misc[k], o);
+    for (int m = 0; m < 8; ++m) mine.misc[m] += __shfl_xor_sync(0xffffffffu, mine.misc[m], o);
   }
-  if ((tid & 31) == 0) {
-    s_abs[tid >> 5] = aabs;
-    for (int k = 0; k < 8; ++k) s_misc[tid >> 5][k] = misc[k];
-  }
+  if (lane == 31) { s_cnt[warp] = icnt; s_tok[warp] = itok; }
+  if (lane == 0) s_part[warp] = mine;
   __syncthreads();
+  int run_cnt = icnt - cnt;
+  long long run_tok = itok - tok;
+  for (int w = 0; w < warp; ++w) { run_cnt += s_cnt[w]; run_tok += s_tok[w]; }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    if (t0 + e < t1) {
+      ws.tile_cnt[t0 + e] = run_cnt;
+      ws.tile_tok[t0 + e] = run_tok;
+    }
+    run_cnt += c[e];
+    run_tok += k[e];
+  }
+  if (tid == 0) {
+    RunPartial tot = {};
+    int rc = 0;
+    long long rt = 0;
+    for (int w = 0; w < kRunThreads / 32; ++w) {
+      tot.abs_adv += s_part[w].abs_adv;
+      for (int m = 0; m < 8; ++m) tot.misc[m] += s_part[w].misc[m];
+      rc += s_cnt[w];
+      rt += s_tok[w];
+    }
+    ws.run_part[blockIdx.x] = tot;
+    ws.run_cnt[blockIdx.x] = rc;
+    ws.run_tok[blockIdx.x] = rt;
+  }
+}
+
+// Level 2, one block: exclusive prefixes of the runs' totals (each thread owns consecutive
+// runs), then the batch totals, counters and metrics, all sums in a fixed order.
+__global__ void __launch_bounds__(kRunThreads) totals_kernel(Args a, Workspace ws, int nruns) {
+  __shared__ long long s_tok[kRunThreads / 32];
+  __shared__ long long s_cnt[kRunThreads / 32];
+  __shared__ RunPartial s_part[kRunThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per = (nruns + kRunThreads - 1) / kRunThreads;
+  const int t0 = min(tid * per, nruns), t1 = min(t0 + per, nruns);
+  long long cnt = 0, tok = 0;
+  RunPartial mine = {};
+  for (int t = t0; t < t1; ++t) {
+    cnt += ws.run_cnt[t];
+    tok += ws.run_tok[t];
+    const RunPartial q = ws.run_part[t];
+    mine.abs_adv += q.abs_adv;
+#pragma unroll
+    for (int m = 0; m < 8; ++m) mine.misc[m] += q.misc[m];
+  }
+  long long icnt = cnt, itok = tok;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long c2 = __shfl_up_sync(0xffffffffu, icnt, o);
+    const long long t2 = __shfl_up_sync(0xffffffffu, itok, o);
+    if (lane >= o) { icnt += c2; itok += t2; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mine.abs_adv += __shfl_xor_sync(0xffffffffu, mine.abs_adv, o);
+#pragma unroll
+    for (int m = 0; m < 8; ++m) mine.misc[m] += __shfl_xor_sync(0xffffffffu, mine.misc[m], o);
+  }
+  if (lane == 31) { s_cnt[warp] = icnt; s_tok[warp] = itok; }
+  if (lane == 0) s_part[warp] = mine;
+  __syncthreads();
+  long long run_cnt = icnt - cnt, run_tok = itok - tok;
+  for (int w = 0; w < warp; ++w) { run_cnt += s_cnt[w]; run_tok += s_tok[w]; }
+  for (int t = t0; t < t1; ++t) {
+    const int c = ws.run_cnt[t];
+    const long long k = ws.run_tok[t];
+    ws.run_cnt[t] = (int)run_cnt;
+    ws.run_tok[t] = run_tok;
+    run_cnt += c;
+    run_tok += k;
+  }
   if (tid == 0) {
     long long tot[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     double sabs = 0.0;
-    for (int t = 0; t < kThreads / 32; ++t) {
-      sabs += s_abs[t];
-      for (int k = 0; k < 8; ++k) tot[k] += s_misc[t][k];
+    long long R_kept = 0, T_kept = 0;
+    for (int w = 0; w < kRunThreads / 32; ++w) {
+      sabs += s_part[w].abs_adv;
+      for (int m = 0; m < 8; ++m) tot[m] += s_part[w].misc[m];
+      R_kept += s_cnt[w];
+      T_kept += s_tok[w];
     }
-    const bool failed = aborted(ws);
-    const long long R_kept = failed ? 0 : (long long)(ld_acquire(ws.desc_roll + ntiles - 1) & kValueMask);
-    const long long T_kept = failed ? 0 : (long long)(ld_acquire(ws.desc_tok + ntiles - 1) & kValueMask);
     const long long T_present = tot[0], R_present = tot[1], P_surv = tot[2];
     const long long* ccat = tot + 3;
     Globals g;
@@ -670,81 +705,79 @@ __device__ void finish_batch(const Args& a, const Workspace& ws, int ntiles) {
   }
 }
 
-__global__ void __launch_bounds__(kThreads, 4) curate_kernel(Args a, Workspace ws, int pt, int ntiles) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  TileShared& sh = *reinterpret_cast<TileShared*>(smem_raw);
-  const int tid = threadIdx.x;
-  if (tid == 0) sh.tile = (int)atomicAdd(ws.ctrl + 0, 1u);
-  __syncthreads();
-  const int tile = sh.tile;             // tiles are taken in order: every earlier tile is already running
-  uint32_t st = 0;
-  if (tile < ntiles) {
-    const int p0 = tile * pt;
-    const int npt = min(pt, a.P - p0);
-    // rollout range of the tile and of each of its prompts (clamped if the offsets are bad), later made
-    // relative to the tile's first rollout
-    for (int q = tid; q <= npt; q += kThreads) {
-      int v = a.go[p0 + q];
-      const int prev = q > 0 ? a.go[p0 + q - 1] : v;
-      if (v < 0 || v > a.R || v < prev) st |= AERO_ST_BAD_OFFSETS;
-      sh.ps.lo[q] = min(max(v, 0), a.R);
-    }
-    // bad offsets only: make the ranges non-decreasing (serial, so kept off the normal path)
-    if (__syncthreads_or((st & AERO_ST_BAD_OFFSETS) != 0)) {
-      if (tid == 0) {
-        int run = sh.ps.lo[0];
-        for (int q = 1; q <= npt; ++q) { run = max(run, sh.ps.lo[q]); sh.ps.lo[q] = run; }
-      }
-      __syncthreads();
-    }
-    const int r0 = sh.ps.lo[0];
-    const int nroll = sh.ps.lo[npt] - r0;
-    __syncthreads();
-    for (int q = tid; q <= npt; q += kThreads) sh.ps.lo[q] -= r0;
-    __syncthreads();
-    if (nroll <= kCap) run_tile_staged(a, ws, sh, tile, p0, npt, r0, nroll, st);
-    else run_tile_global(a, ws, sh, tile, p0, npt, r0, st);
-  }
-  st = __reduce_or_sync(0xffffffffu, st);
-  if ((tid & 31) == 0) aero_raise(a.status, st);
-
-  // the last block to finish reduces the metrics records
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) sh.failed = atomicAdd(ws.ctrl + 1, 1u) == (unsigned)(ntiles - 1) ? 1 : 0;
-  __syncthreads();
-  if (sh.failed) {
-    __threadfence();
-    finish_batch(a, ws, ntiles);
-  }
-}
-
-// Per-rollout weights (Eq. 2 normalisers) and the tails of the compacted arrays.
-__global__ void __launch_bounds__(kThreads) weights_kernel(Args a, Workspace ws, int pt, int ntiles) {
-  __shared__ int s_lo[kMaxPT + 1];
+// Compacted ids and token offsets of the kept rollouts, per-rollout weights (Eq. 2 normalisers)
+// and the tails of the compacted arrays; one warp per share, one lane per rollout.
+__global__ void __launch_bounds__(kThreads) emit_kernel(Args a, Workspace ws, int pw) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int tile = blockIdx.x;
+  uint32_t st = 0;      // bad offsets were reported by the first launch
+  const Share sh = load_share(a, tile * kWarps + warp, pw, st);
+  if (sh.np == 0) return;
   const Globals g = *ws.glob;
-  const int tid = threadIdx.x;
-  for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-    const int p0 = tile * pt;
-    const int npt = min(pt, a.P - p0);
-    __syncthreads();
-    for (int q = tid; q <= npt; q += kThreads) s_lo[q] = min(max(a.go[p0 + q], 0), a.R);
-    __syncthreads();
-    const int r0 = s_lo[0];
-    const int r1 = max(s_lo[npt], r0);
-    for (int i = r0 + tid; i < r1; i += kThreads) {
+  // kept rollouts and tokens before this share: earlier tiles, then earlier warps of this tile
+  int pos0 = lane < warp ? ws.share_cnt[tile * kWarps + lane] : 0;
+  long long tok0 = lane < warp ? ws.share_tok[tile * kWarps + lane] : 0;
+  pos0 = __reduce_add_sync(0xffffffffu, pos0);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tok0 += __shfl_xor_sync(0xffffffffu, tok0, o);
+  pos0 += ws.run_cnt[tile / kRunTiles] + ws.tile_cnt[tile];
+  tok0 += ws.run_tok[tile / kRunTiles] + ws.tile_tok[tile];
+  const bool seq_mean = a.cfg.agg != AERO_TOKEN_MEAN;
+  const unsigned below = (1u << lane) - 1u;
+  for (int c0 = 0; c0 < sh.nroll; c0 += 32) {
+    const int j = c0 + lane;
+    const bool valid = j < sh.nroll;
+    const int i = sh.r0 + j;
+    bool kp = false;
+    int len = 0;
+    if (valid) {
+      kp = a.keep[i] != 0;
+      len = clamped_len(a.cs[i + 1] - a.cs[i]);
+    }
+    const unsigned km = __ballot_sync(0xffffffffu, kp);
+    if (km) {
+      long long incl;
+      if (__reduce_max_sync(0xffffffffu, kp ? (unsigned)len : 0u) < (1u << 26)) {   // the chunk's sum fits 32 bits
+        unsigned t32 = kp ? (unsigned)len : 0u;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned t2 = __shfl_up_sync(0xffffffffu, t32, o);
+          if (lane >= o) t32 += t2;
+        }
+        incl = t32;
+      } else {
+        incl = kp ? len : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const long long t2 = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += t2;
+        }
+      }
+      if (kp) {
+        const int pos = pos0 + __popc(km & below);
+        a.kept_ids[pos] = i;
+        a.kept_tok_off[pos] = tok0 + incl - len;
+      }
+      pos0 += __popc(km);
+      tok0 += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    // sequence mean: the rollout's prompt is the last one of the share that starts at or before it
+    int q = 0;
+    if (seq_mean) {
+#pragma unroll
+      for (int s = 16; s > 0; s >>= 1) {
+        const int cand = q + s;
+        const int start = __shfl_sync(0xffffffffu, sh.lo, cand & 31);
+        if (cand < sh.np && start <= j) q = cand;
+      }
+    }
+    if (valid) {
       float w = 0.f;
-      if (a.keep[i]) {
-        if (a.cfg.agg == AERO_TOKEN_MEAN) {
+      if (kp) {
+        if (!seq_mean) {
           w = g.inv_tok_den;
         } else {
-          int lo = 0, hi = npt;             // prompt of rollout i
-          while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (s_lo[mid] <= i) lo = mid; else hi = mid;
-          }
-          const int nk = ws.nkept[p0 + lo];
-          const long long len = a.cs[i + 1] - a.cs[i];
+          const int nk = ws.nkept[sh.p0 + q];
           w = (nk > 0 && len > 0) ? g.inv_prompt_den / (float)nk / (float)len : 0.f;
         }
       }
@@ -760,10 +793,9 @@ __global__ void __launch_bounds__(kThreads) weights_kernel(Args a, Workspace ws,
 
 size_t aero_group_ws_bytes_impl(int32_t P, int32_t R) {
   if (P < 0) P = 0;
-  const int pt = prompts_per_tile(P, R);
-  const int ntiles = (P + pt - 1) / pt + 1;
-  return cleared_bytes(ntiles) + up256(sizeof(int) * (size_t)P) + up256(sizeof(TilePartial) * (size_t)ntiles) +
-         up256(sizeof(Globals));
+  const int pt = prompts_per_warp(P, R) * kWarps;
+  const int ntiles = (P + pt - 1) / pt;
+  return workspace_bytes((size_t)P, (size_t)ntiles);
 }
 
 int aero_group_stats_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
@@ -787,16 +819,17 @@ int aero_group_stats_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32
     if (metrics) AERO_CUDA_TRY(cudaMemsetAsync(metrics, 0, 4 * sizeof(float), ctx->stream));
     if (P == 0) return AERO_OK;
   }
-  const int pt = prompts_per_tile(P, R);
+  const int pw = prompts_per_warp(P, R);
+  const int pt = pw * kWarps;
   const int ntiles = (P + pt - 1) / pt;
-  Workspace ws = carve(wsp, P, ntiles + 1);
-  // scan records, ticket and counters start at zero on every call
-  AERO_CUDA_TRY(cudaMemsetAsync(wsp, 0, cleared_bytes(ntiles + 1), ctx->stream));
-  AERO_CUDA_TRY(cudaFuncSetAttribute(curate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TileShared)));
-  curate_kernel<<<ntiles, kThreads, sizeof(TileShared), ctx->stream>>>(a, ws, pt, ntiles);
-  const int wblocks = ntiles < 8 * ctx->sm_count ? ntiles : 8 * ctx->sm_count;
-  weights_kernel<<<wblocks, kThreads, 0, ctx->stream>>>(a, ws, pt, ntiles);
-  ctx->launches += 2;
+  Workspace ws = carve(wsp, P, ntiles);
+  AERO_CUDA_TRY(cudaFuncSetAttribute(curate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(BlockShared)));
+  curate_kernel<<<ntiles, kThreads, sizeof(BlockShared), ctx->stream>>>(a, ws, pw);
+  const int nruns = (int)runs_of((size_t)ntiles);
+  run_prefix_kernel<<<nruns, kRunThreads, 0, ctx->stream>>>(ws, ntiles);
+  totals_kernel<<<1, kRunThreads, 0, ctx->stream>>>(a, ws, nruns);
+  emit_kernel<<<ntiles, kThreads, 0, ctx->stream>>>(a, ws, pw);
+  ctx->launches += 4;
   AERO_CUDA_TRY(cudaGetLastError());
   return AERO_OK;
 }
@@ -808,12 +841,8 @@ int aero_group_stats_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32
 namespace {
 
 constexpr int32_t kStaticMaxP = AERO_STATIC_MAX_PROMPTS;
-constexpr size_t cup256(size_t x) { return (x + 255) / 256 * 256; }
-// room for the per-prompt words of kStaticMaxP prompts and the records of kStaticMaxTiles tiles
-constexpr size_t kStaticMaxTiles = 16384;
-constexpr size_t kStaticBytes = cup256(sizeof(unsigned long long) * 2 * (kStaticMaxTiles + 1) + 16) +
-                                cup256(sizeof(int) * (size_t)kStaticMaxP) +
-                                cup256(sizeof(TilePartial) * (kStaticMaxTiles + 1)) + cup256(sizeof(Globals));
+// room for kStaticMaxP prompts in the smallest tiles there are (one prompt per warp)
+constexpr size_t kStaticBytes = workspace_bytes((size_t)kStaticMaxP, ((size_t)kStaticMaxP + kWarps - 1) / kWarps);
 
 static __device__ __align__(256) unsigned char g_group_scratch[kStaticBytes];
 
@@ -858,9 +887,9 @@ extern "C" int aero_group_stats_static(aero_ctx* ctx, const aero_cfg* cfg, int32
   void* scratch = nullptr;
   const int rc = static_scratch(ctx->device, &scratch);
   if (rc) return rc;
-  // the launch clears the scan records and counters at the head of the scratch; every other
-  // scratch word the kernels read is written earlier in the same call
+  // every scratch word the kernels read is written earlier in the same call
   return aero_group_stats_launch(ctx, cfg, P, R, go, reward, cs, key, keep_in, alpha_in, beta_in,
                                  adv, w, keep, gmask, cat, u_tilde, alpha_out, beta_out,
                                  kept_ids, kept_tok_off, counters, metrics, scratch);
 }
+
