@@ -191,9 +191,9 @@ __device__ __forceinline__ Rule decide(const Args& a, int p, int n, int c) {
 // What the rollouts of one prompt need to know about it (shared memory, one entry per prompt of
 // a warp's share).
 struct PromptRule {
-  float mu, inv;
+  float adv_correct, adv_incorrect;   // advantage of a kept rollout by its reward bit
   unsigned range;      // first rollout | one past the last << 16, relative to the share's first rollout
-  unsigned sel;        // mode (0 keep all present, 1 keep none, 2 select by rank) | reject << 2 | quota << 4
+  unsigned sel;        // bit 0: keep none; bit 1: the incorrect rollouts are ranked; bit 2: the correct ones are; quota << 4
 };
 
 // Staging of one warp's share.  `ck` orders the candidates of a selection and carries the
@@ -201,19 +201,29 @@ struct PromptRule {
 // all ones for an absent one, so that in a group that selects among its incorrect rollouts no
 // correct one ever compares smaller.  One bit per rollout in `pmask` (present) and `cmask` (present and correct), one word
 // per chunk of 32 rollouts.
-struct WarpStage {
-  unsigned long long ck[kWCap];
-  PromptRule rule[kMaxPW];
-  unsigned pmask[kWChunks], cmask[kWChunks];
-  uint8_t pid[kWCap];        // which prompt of the share owns the rollout
+struct WarpStage {          // a warp's view of the block's staging arrays
+  unsigned long long* ck;   // [kWCap]
+  PromptRule* rule;         // [kMaxPW]
+  unsigned* pmask;          // [kWChunks]
+  unsigned* cmask;          // [kWChunks]
+  uint8_t* pid;             // [kWCap] which prompt of the share owns the rollout
 };
 
+// The sort words of all warps come first and the other arrays (more than kWCap words together)
+// after them, so that a read up to kWCap entries past the end of any warp's sort words stays
+// inside the block's shared memory: the rank loop reads past a short group without clamping
+// and discards what it read.
 struct BlockShared {
-  WarpStage stage[kWarps];
+  unsigned long long ck[kWarps][kWCap];
+  PromptRule rule[kWarps][kMaxPW];
+  uint8_t pid[kWarps][kWCap];
+  unsigned pmask[kWarps][kWChunks], cmask[kWarps][kWChunks];
   TilePartial red[kWarps];
   long long share_tok[kWarps];
   int share_cnt[kWarps];
 };
+static_assert(sizeof(BlockShared) - sizeof(unsigned long long) * kWarps * kWCap >= sizeof(unsigned long long) * kWCap,
+              "the arrays after the sort words must cover the longest read past them");
 
 // A warp's share of a tile: prompts [p0, p0 + np), their rollouts [r0, r0 + nroll); lane q holds
 // the rollout range [lo, hi) of prompt p0 + q, relative to r0 (empty for q >= np).
@@ -306,14 +316,13 @@ __device__ __forceinline__ void group_moments(const Args& a, const Rule& ru, int
   *inv_out = 1.f / (sd + a.cfg.eps_std);
 }
 
-// A share whose rollouts fit the warp's staging area and are shorter than 2^22 tokens each.
-// Rewards enter as the bit r > 0.5 (they must be exactly 0 or 1; anything else raises
-// AERO_ST_BAD_REWARD), so per-prompt sums are bit counts and mean and deviation are closed
+// A share whose rollouts fit the warp's staging area, have between 1 and 2^22 - 1 tokens each
+// and rewards of exactly 0 or 1.  Rewards enter as the bit r > 0.5, so per-prompt sums are bit counts and mean and deviation are closed
 // forms of the counts; the number of rollouts a selection keeps is known from the rule alone,
 // so the per-prompt outputs are written before any rollout is ranked.  Returns false, with
-// nothing written, if a rollout is too long for the staging word; else the share's kept
-// rollouts and tokens.
-__device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws, WarpStage& S, const Share& sh,
+// nothing written, if a rollout does not qualify; else the share's kept rollouts and tokens.
+template <bool HAS_KEEP_IN, bool HAS_KEY>
+__device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws, const WarpStage& S, const Share& sh,
                                               TilePartial& mine, uint32_t& st, int* cnt_out, long long* tok_out) {
   const int lane = threadIdx.x & 31;
   const int r0 = sh.r0, nroll = sh.nroll;
@@ -323,44 +332,39 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
     for (int j = sh.lo; j < sh.hi; ++j) S.pid[j] = (uint8_t)lane;
 
   // ---- stage the rollouts (coalesced), one bit each for present and correct ----
-  uint32_t bits = 0;
-  long long ptok = 0;
-  bool too_long = false;
+  // (lanes past the share's end read its last rollout again and count as absent)
+  // A reward other than 0 or 1, or a length outside [1, 2^22), sends the whole share to the
+  // path that walks global memory, which also raises the status bits.
+  bool irregular = false;
+  unsigned ptok = 0;       // at most kWChunks lengths below 2^22 per lane
+#pragma unroll 2
   for (int c = 0; c * 32 < nroll; ++c) {
     const int j = c * 32 + lane;
-    const int i = r0 + j;
-    bool pres = false, corr = false;
-    if (j < nroll) {
-      const float r = a.reward[i];
-      const long long len = a.cs[i + 1] - a.cs[i];
-      pres = a.keep_in ? a.keep_in[i] != 0 : true;
-      corr = r > 0.5f;
-      unsigned long long ck = kNone;
-      if (pres) {
-        if (r != 0.f && r != 1.f) bits |= AERO_ST_BAD_REWARD;
-        if (len < 0) bits |= AERO_ST_BAD_OFFSETS;
-        if (len == 0) bits |= AERO_ST_EMPTY_ROLLOUT;
-        too_long = too_long || len >= (1ll << kLenBits);
-        const uint32_t key = a.key ? a.key[i] : default_key(a.cfg.seed, (uint32_t)i);
-        const unsigned l = (unsigned)clamped_len(len) & kLenMask;
-        ck = (corr ? 1ull << 63 : 0ull) | ((unsigned long long)key << 31) | ((unsigned long long)j << kLenBits) | l;
-        ptok += l;
-      }
-      S.ck[j] = ck;
-    }
+    const int i = r0 + min(j, nroll - 1);
+    const float r = a.reward[i];
+    const long long len = a.cs[i + 1] - a.cs[i];
+    bool pres = j < nroll;
+    if (HAS_KEEP_IN) pres = pres && a.keep_in[i] != 0;
+    const bool corr = r > 0.5f;
+    const uint32_t key = HAS_KEY ? a.key[i] : default_key(a.cfg.seed, (uint32_t)i);
+    irregular |= pres && ((r != 0.f && r != 1.f) || (unsigned long long)(len - 1) >= (unsigned long long)kLenMask);
+    const unsigned l = (unsigned)len & kLenMask;
+    const unsigned long long ck =
+        (corr ? 1ull << 63 : 0ull) | ((unsigned long long)key << 31) | ((unsigned long long)(unsigned)j << kLenBits) | l;
+    S.ck[j & (kWCap - 1)] = pres ? ck : kNone;
+    ptok += pres ? l : 0u;
     const unsigned pm = __ballot_sync(0xffffffffu, pres);
     const unsigned cm = __ballot_sync(0xffffffffu, pres && corr);
     if (lane == 0) { S.pmask[c] = pm; S.cmask[c] = cm; }
   }
-  if (__any_sync(0xffffffffu, too_long)) return false;
-  st |= bits;
+  if (__any_sync(0xffffffffu, irregular)) return false;
   mine.present_tok = ptok;
   __syncwarp();
 
   // ---- per prompt: counts, category, posterior, curation rule, moments of the base set ----
   if (lane < sh.np) {
     const int p = sh.p0 + lane;
-    const int n = a.keep_in ? range_popc(S.pmask, sh.lo, sh.hi) : sh.hi - sh.lo;
+    const int n = HAS_KEEP_IN ? range_popc(S.pmask, sh.lo, sh.hi) : sh.hi - sh.lo;
     const int c = range_popc(S.cmask, sh.lo, sh.hi);
     const Rule ru = decide(a, p, n, c);
     a.cat[p] = (uint8_t)ru.category;
@@ -382,12 +386,14 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
     a.gmask[p] = nk > 0 ? 1 : 0;
     if (a.cfg.agg != AERO_TOKEN_MEAN) ws.nkept[p] = nk;
     PromptRule pr;
-    pr.mu = mu;
-    pr.inv = inv;
+    pr.adv_correct = (1.f - mu) * inv;
+    pr.adv_incorrect = (0.f - mu) * inv;
     pr.range = (unsigned)sh.lo | ((unsigned)sh.hi << 16);
     // every incorrect rollout orders before every correct one: when the correct ones are the
     // candidates, the n - c incorrect ones are counted by each rank and the quota allows for them
-    pr.sel = (unsigned)ru.mode | ((unsigned)ru.reject << 2) | ((unsigned)((int)ru.quota + (ru.reject == 2 ? n - c : 0)) << 4);
+    const bool sel = ru.mode == 2;
+    pr.sel = (ru.mode == 1 ? 1u : 0u) | (sel && ru.reject != 2 ? 2u : 0u) | (sel && ru.reject != 1 ? 4u : 0u) |
+             ((unsigned)((int)ru.quota + (ru.reject == 2 ? n - c : 0)) << 4);
     S.rule[lane] = pr;
     mine.present_roll = n;
 #pragma unroll
@@ -399,7 +405,7 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
 
   // ---- per rollout: keep decision (rank among the group's candidates), advantage ----
   int cnt = 0;
-  long long tok = 0;
+  unsigned ktok = 0;       // at most kWChunks lengths below 2^22 per lane
   for (int c = 0; c * 32 < nroll; ++c) {
     const int j = c * 32 + lane;
     const bool valid = j < nroll;
@@ -407,29 +413,32 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
     const unsigned long long mykey = S.ck[j & (kWCap - 1)];
     const bool pres = (S.pmask[c] >> lane) & 1u;
     const bool corr = (S.cmask[c] >> lane) & 1u;
-    const int mode = (int)(pr.sel & 3u), rej = (int)((pr.sel >> 2) & 3u);
-    bool kp = pres && mode != 1;
-    const bool ranked = kp && mode == 2 && !(rej == 1 && corr) && !(rej == 2 && !corr);
+    bool kp = pres && !(pr.sel & 1u);
+    const bool ranked = pres && (pr.sel & (corr ? 4u : 2u));
     // the loop runs as long as the longest group among the chunk's ranked rollouts, the same for all lanes
     const int lo = (int)(pr.range & 0xffffu);
     const int span = ranked ? (int)(pr.range >> 16) - lo : 0;
     const int longest = (int)__reduce_max_sync(0xffffffffu, (unsigned)span);
     if (longest > 0) {
+      // (reads past the lane's own group stay inside the block's shared memory and are not counted)
       const unsigned long long* grp = S.ck + lo;
       int rank = 0;
 #pragma unroll 4
-      for (int d = 0; d < longest; ++d)
-        if (d < span) rank += grp[d] < mykey ? 1 : 0;
+      for (int d = 0; d < longest; ++d) {
+        const unsigned long long other = grp[d];
+        rank += (d < span && other < mykey) ? 1 : 0;
+      }
       if (ranked) kp = rank < (int)(pr.sel >> 4);
     }
     const unsigned km = __ballot_sync(0xffffffffu, kp);
     if (valid) {
-      a.adv[r0 + j] = kp ? ((corr ? 1.f : 0.f) - pr.mu) * pr.inv : 0.f;
+      a.adv[r0 + j] = kp ? (corr ? pr.adv_correct : pr.adv_incorrect) : 0.f;
       a.keep[r0 + j] = kp ? 1 : 0;
     }
     cnt += __popc(km);
-    tok += kp ? (long long)((unsigned)mykey & kLenMask) : 0ll;
+    ktok += kp ? (unsigned)mykey & kLenMask : 0u;
   }
+  long long tok = ktok;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) tok += __shfl_xor_sync(0xffffffffu, tok, o);
   *cnt_out = cnt;
@@ -507,6 +516,7 @@ __device__ void curate_global(const Args& a, const Workspace& ws, const Share& s
   *tok_out = ktok;
 }
 
+template <bool HAS_KEEP_IN, bool HAS_KEY>
 __global__ void __launch_bounds__(kThreads, kBlocksPerSM) curate_kernel(Args a, Workspace ws, int pw) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   BlockShared& bs = *reinterpret_cast<BlockShared*>(smem_raw);
@@ -518,7 +528,8 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSM) curate_kernel(Args a, 
   int cnt = 0;
   long long tok = 0;
   if (sh.np > 0) {
-    const bool done = sh.nroll <= kWCap && curate_staged(a, ws, bs.stage[warp], sh, mine, st, &cnt, &tok);
+    const WarpStage S = {bs.ck[warp], bs.rule[warp], bs.pmask[warp], bs.cmask[warp], bs.pid[warp]};
+    const bool done = sh.nroll <= kWCap && curate_staged<HAS_KEEP_IN, HAS_KEY>(a, ws, S, sh, mine, st, &cnt, &tok);
     if (!done) curate_global(a, ws, sh, mine, st, &cnt, &tok);
   }
   mine = warp_partial(mine);
@@ -707,14 +718,15 @@ __global__ void __launch_bounds__(kRunThreads) totals_kernel(Args a, Workspace w
 
 // Compacted ids and token offsets of the kept rollouts, per-rollout weights (Eq. 2 normalisers)
 // and the tails of the compacted arrays; one warp per share, one lane per rollout.
+template <bool SEQ_MEAN>
 __global__ void __launch_bounds__(kThreads) emit_kernel(Args a, Workspace ws, int pw) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int tile = blockIdx.x;
   uint32_t st = 0;      // bad offsets were reported by the first launch
   const Share sh = load_share(a, tile * kWarps + warp, pw, st);
-  if (sh.np == 0) return;
+  if (sh.np == 0 || sh.nroll == 0) return;
   const Globals g = *ws.glob;
-  // kept rollouts and tokens before this share: earlier tiles, then earlier warps of this tile
+  // kept rollouts and tokens before this share: earlier runs, earlier tiles of the run, earlier warps of the tile
   int pos0 = lane < warp ? ws.share_cnt[tile * kWarps + lane] : 0;
   long long tok0 = lane < warp ? ws.share_tok[tile * kWarps + lane] : 0;
   pos0 = __reduce_add_sync(0xffffffffu, pos0);
@@ -722,18 +734,9 @@ __global__ void __launch_bounds__(kThreads) emit_kernel(Args a, Workspace ws, in
   for (int o = 16; o > 0; o >>= 1) tok0 += __shfl_xor_sync(0xffffffffu, tok0, o);
   pos0 += ws.run_cnt[tile / kRunTiles] + ws.tile_cnt[tile];
   tok0 += ws.run_tok[tile / kRunTiles] + ws.tile_tok[tile];
-  const bool seq_mean = a.cfg.agg != AERO_TOKEN_MEAN;
   const unsigned below = (1u << lane) - 1u;
-  for (int c0 = 0; c0 < sh.nroll; c0 += 32) {
-    const int j = c0 + lane;
-    const bool valid = j < sh.nroll;
-    const int i = sh.r0 + j;
-    bool kp = false;
-    int len = 0;
-    if (valid) {
-      kp = a.keep[i] != 0;
-      len = clamped_len(a.cs[i + 1] - a.cs[i]);
-    }
+  // one chunk of 32 rollouts, its keep flags and lengths already loaded
+  auto emit_chunk = [&](int c0, int i, bool valid, bool kp, int len) {
     const unsigned km = __ballot_sync(0xffffffffu, kp);
     if (km) {
       long long incl;
@@ -761,31 +764,38 @@ __global__ void __launch_bounds__(kThreads) emit_kernel(Args a, Workspace ws, in
       pos0 += __popc(km);
       tok0 += __shfl_sync(0xffffffffu, incl, 31);
     }
-    // sequence mean: the rollout's prompt is the last one of the share that starts at or before it
-    int q = 0;
-    if (seq_mean) {
+    float w = kp ? g.inv_tok_den : 0.f;
+    if (SEQ_MEAN) {
+      // the rollout's prompt is the last one of the share that starts at or before it
+      const int j = c0 + lane;
+      int q = 0;
 #pragma unroll
       for (int s = 16; s > 0; s >>= 1) {
         const int cand = q + s;
         const int start = __shfl_sync(0xffffffffu, sh.lo, cand & 31);
         if (cand < sh.np && start <= j) q = cand;
       }
+      const int nk = kp ? ws.nkept[sh.p0 + q] : 0;
+      w = (nk > 0 && len > 0) ? g.inv_prompt_den / (float)nk / (float)len : 0.f;
     }
-    if (valid) {
-      float w = 0.f;
-      if (kp) {
-        if (!seq_mean) {
-          w = g.inv_tok_den;
-        } else {
-          const int nk = ws.nkept[sh.p0 + q];
-          w = (nk > 0 && len > 0) ? g.inv_prompt_den / (float)nk / (float)len : 0.f;
-        }
-      }
-      a.w[i] = w;
+    if (valid) a.w[i] = w;
+    // tails of the compacted arrays, only where the chunk reaches them
+    if ((long long)sh.r0 + c0 + 32 >= g.R_kept && valid) {
       if ((long long)i >= g.R_kept) a.kept_ids[i] = -1;
       if ((long long)i + 1 >= g.R_kept) a.kept_tok_off[i + 1] = g.T_kept;
       if (i == 0 && g.R_kept == 0) a.kept_tok_off[0] = 0;
     }
+  };
+  // two chunks per turn, the loads of both issued before either is processed; lanes past the
+  // share's end read its last rollout again and count as not kept
+  for (int c0 = 0; c0 < sh.nroll; c0 += 64) {
+    const int j0 = c0 + lane, j1 = j0 + 32;
+    const bool v0 = j0 < sh.nroll, v1 = j1 < sh.nroll;
+    const int i0 = sh.r0 + min(j0, sh.nroll - 1), i1 = sh.r0 + min(j1, sh.nroll - 1);
+    const uint8_t k0 = a.keep[i0], k1 = a.keep[i1];
+    const long long b0 = a.cs[i0], e0 = a.cs[i0 + 1], b1 = a.cs[i1], e1 = a.cs[i1 + 1];
+    emit_chunk(c0, i0, v0, v0 && k0 != 0, clamped_len(e0 - b0));
+    if (c0 + 32 < sh.nroll) emit_chunk(c0 + 32, i1, v1, v1 && k1 != 0, clamped_len(e1 - b1));
   }
 }
 
@@ -823,12 +833,15 @@ int aero_group_stats_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32
   const int pt = pw * kWarps;
   const int ntiles = (P + pt - 1) / pt;
   Workspace ws = carve(wsp, P, ntiles);
-  AERO_CUDA_TRY(cudaFuncSetAttribute(curate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(BlockShared)));
-  curate_kernel<<<ntiles, kThreads, sizeof(BlockShared), ctx->stream>>>(a, ws, pw);
+  auto curate = keep_in ? (key ? curate_kernel<true, true> : curate_kernel<true, false>)
+                        : (key ? curate_kernel<false, true> : curate_kernel<false, false>);
+  AERO_CUDA_TRY(cudaFuncSetAttribute(curate, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(BlockShared)));
+  curate<<<ntiles, kThreads, sizeof(BlockShared), ctx->stream>>>(a, ws, pw);
   const int nruns = (int)runs_of((size_t)ntiles);
   run_prefix_kernel<<<nruns, kRunThreads, 0, ctx->stream>>>(ws, ntiles);
   totals_kernel<<<1, kRunThreads, 0, ctx->stream>>>(a, ws, nruns);
-  emit_kernel<<<ntiles, kThreads, 0, ctx->stream>>>(a, ws, pw);
+  if (cfg->agg != AERO_TOKEN_MEAN) emit_kernel<true><<<ntiles, kThreads, 0, ctx->stream>>>(a, ws, pw);
+  else emit_kernel<false><<<ntiles, kThreads, 0, ctx->stream>>>(a, ws, pw);
   ctx->launches += 4;
   AERO_CUDA_TRY(cudaGetLastError());
   return AERO_OK;
