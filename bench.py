@@ -420,7 +420,7 @@ def variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, g, dH, dW, ws_b, T_kept,
 
 def group_stage_leg(ctx, pk, dev):
     """Stage (a) alone on an input large enough to be bandwidth-bound (2^22 prompts of 2..16 rollouts):
-    algorithmic bytes (37 per rollout + 26 per prompt) over the duration of the three launches."""
+    algorithmic bytes (37 per rollout + 26 per prompt) over the duration of the stage's four launches."""
     import torch
     from paper_2602_14338_b200 import binding as B
     from paper_2602_14338_b200 import synth

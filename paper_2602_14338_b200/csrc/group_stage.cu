@@ -28,13 +28,13 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kBlocksPerSM = 5;
-constexpr int kWCap = 512;             // rollouts a warp can stage
+constexpr int kBlocksPerSM = 6;
+constexpr int kWCap = 416;             // rollouts a warp can stage
 constexpr int kWChunks = kWCap / 32;
 constexpr int kLenBits = 22;           // staged rollouts are shorter than 2^22 tokens
 constexpr unsigned kLenMask = (1u << kLenBits) - 1u;
 constexpr int kMaxPW = 32;             // prompts per warp: one lane each in the per-prompt steps
-constexpr int kWTarget = 352;          // rollouts per warp the host aims at (mean group size rounded up)
+constexpr int kWTarget = 300;          // mean rollouts per warp the host aims at
 constexpr int kRunThreads = 256;
 constexpr int kRunTiles = kRunThreads * 4;   // tiles per run of the batch-wide prefix
 constexpr unsigned long long kNone = ~0ull;
@@ -74,9 +74,12 @@ struct Workspace {
 
 __host__ __device__ constexpr size_t up256(size_t x) { return (x + 255) / 256 * 256; }
 
+// Prompts per warp: as many as keep the mean share near kWTarget rollouts, which leaves the
+// staging area a margin of more than three standard deviations for group sizes spread
+// uniformly around their mean.
 inline int prompts_per_warp(int32_t P, int32_t R) {
-  const long long avg = P > 0 ? ((long long)R + P - 1) / P : 1;
-  long long pw = kWTarget / (avg > 0 ? avg : 1);
+  if (P <= 0 || R <= 0) return kMaxPW;
+  const long long pw = (long long)kWTarget * P / R;
   return (int)(pw < 1 ? 1 : (pw > kMaxPW ? kMaxPW : pw));
 }
 
@@ -351,7 +354,7 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
     const unsigned l = (unsigned)len & kLenMask;
     const unsigned long long ck =
         (corr ? 1ull << 63 : 0ull) | ((unsigned long long)key << 31) | ((unsigned long long)(unsigned)j << kLenBits) | l;
-    S.ck[j & (kWCap - 1)] = pres ? ck : kNone;
+    S.ck[min(j, kWCap - 1)] = pres ? ck : kNone;
     ptok += pres ? l : 0u;
     const unsigned pm = __ballot_sync(0xffffffffu, pres);
     const unsigned cm = __ballot_sync(0xffffffffu, pres && corr);
@@ -410,7 +413,7 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
     const int j = c * 32 + lane;
     const bool valid = j < nroll;
     const PromptRule pr = S.rule[valid ? S.pid[j] : 0];
-    const unsigned long long mykey = S.ck[j & (kWCap - 1)];
+    const unsigned long long mykey = S.ck[min(j, kWCap - 1)];
     const bool pres = (S.pmask[c] >> lane) & 1u;
     const bool corr = (S.cmask[c] >> lane) & 1u;
     bool kp = pres && !(pr.sel & 1u);
