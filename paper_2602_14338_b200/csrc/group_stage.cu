@@ -759,8 +759,10 @@ __global__ void __launch_bounds__(kThreads) emit_kernel(Args a, Workspace ws, in
           if (lane >= o) incl += t2;
         }
       }
-      if (kp) {
-        const int pos = pos0 + __popc(km & below);
+      // (with offsets that are not a partition of the rollouts the shares may overlap and the
+      // counts exceed R: such entries are dropped, the status bit has been raised)
+      const int pos = pos0 + __popc(km & below);
+      if (kp && pos < a.R) {
         a.kept_ids[pos] = i;
         a.kept_tok_off[pos] = tok0 + incl - len;
       }

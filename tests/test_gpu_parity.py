@@ -94,6 +94,59 @@ def test_group_stats_groups_larger_than_a_tile(ctx, high):
     assert ctx.last_status() == 0
 
 
+def test_group_stats_very_long_rollouts(ctx):
+    """Rollouts of 2^22 tokens and more leave the staged path (its staging word holds 22 bits of length),
+    and a chunk with one of 2^26 or more takes the 64-bit scan of the second pass; token totals pass 2^32."""
+    rng = np.random.default_rng(17)
+    sizes = rng.integers(1, 17, 400)
+    P, R = len(sizes), int(sizes.sum())
+    go = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int32)
+    reward = (rng.random(R) < 0.4).astype(np.float32)
+    lens = rng.integers(1, 3000, R).astype(np.int64)
+    lens[rng.integers(0, R, 25)] = rng.integers(1 << 22, 1 << 23, 25)
+    lens[rng.integers(0, R, 10)] = rng.integers(1 << 26, 1 << 30, 10)
+    lens[[0, R - 1]] = [(1 << 31) - 1, 1 << 22]
+    cs = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    assert cs[-1] > 1 << 32
+    key = rng.integers(0, 1 << 32, R, dtype=np.uint64).astype(np.uint32)
+    st = synth.Structure(go, cs, reward, key, None, None, None, None)
+    for over in (dict(), dict(agg=O.AGG_SEQ_MEAN, denom=O.DENOM_ALL)):
+        ocfg = O.Cfg(uniform_policy=O.UNIFORM_BAYES, rejection=1, **over)
+        ref = O.group_stats(ocfg, go, reward, cs, key=key)
+        _, out = TL.run_group_gpu(ctx, TL.lib_cfg(ocfg, "bf16"), st)
+        TL.check_group(out, ref, R, P)
+    assert ctx.last_status() == 0
+
+
+def test_group_stats_offsets_that_are_no_partition(ctx):
+    """Group offsets that go backwards or past R raise AERO_ST_BAD_OFFSETS; every index the kernels use is
+    clamped into the arrays (ranges into [0, R], compacted positions below R), so the call completes and
+    the next one on good inputs is exact again."""
+    rng = np.random.default_rng(23)
+    P, R = 700, 5000
+    go = np.sort(rng.integers(0, R + 1, P + 1)).astype(np.int32)
+    go[0], go[-1] = 0, R
+    bad = go.copy()
+    bad[100] = R + 50            # past the end
+    bad[300] = -7                # negative
+    bad[500:520] = bad[500:520][::-1].copy()      # backwards
+    bad[640] = 0                 # a share that starts over: overlaps everything before it
+    reward = (rng.random(R) < 0.5).astype(np.float32)
+    lens = rng.integers(1, 40, R)
+    cs = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    key = rng.integers(0, 1 << 32, R, dtype=np.uint64).astype(np.uint32)
+    cfg = B.cfg_default(uniform_policy=B.AERO_UNIFORM_BAYES, rejection=1)
+    ctx.group_stats(cfg, TL.dev(bad), TL.dev(reward), TL.dev(cs), key=TL.dev(key.view(np.int32)))
+    torch.cuda.synchronize()
+    assert ctx.last_status() & B.AERO_ST_BAD_OFFSETS
+    assert ctx.last_status() == 0
+    st = synth.Structure(go, cs, reward, key, None, None, None, None)
+    ocfg = O.Cfg(uniform_policy=O.UNIFORM_BAYES, rejection=1)
+    ref = O.group_stats(ocfg, go, reward, cs, key=key)
+    _, out = TL.run_group_gpu(ctx, TL.lib_cfg(ocfg, "bf16"), st)
+    TL.check_group(out, ref, R, P)
+
+
 def test_group_stats_empty_inputs_and_status_bits(ctx):
     cfg = B.cfg_default()
     go = torch.zeros(1, dtype=torch.int32, device="cuda")
