@@ -45,6 +45,8 @@ struct Params {
   __nv_bfloat16* dH;
   float* dW;
   uint32_t* status;
+  const float* row_scale;       // dH: factor of each token row, applied to the finished tile (NULL: none)
+  int h_local;                  // dW: operand B holds the chunk's rows tile after tile, not all T rows
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -110,7 +112,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
               const int nxt = kb / (BM / BK) + 1;
               row_next = nxt < chunk_tiles ? __ldg(p.tile_row + p.tile_begin + nxt) : 0;
             }
-            const int hrow = row_cur + (kb % (BM / BK)) * BK;
+            const int hrow = p.h_local ? kb * BK : row_cur + (kb % (BM / BK)) * BK;
             tc::tma_load_4d(a_s, &tmA, 0, (kb % (BM / BK)) * BK, mt * (BM / 64), kb / (BM / BK), &ctl->full[s]);
             tc::tma_load_3d(b_s, &tmB, 0, hrow, nt * (BN / 64), &ctl->full[s]);
           }
@@ -181,6 +183,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
           // rows outside the tile's run, past T or past V: nothing to write
         } else if (KIND == KIND_DH) {
           uint4* dst = reinterpret_cast<uint4*>(p.dH + out_row * p.d + col0);
+          if (p.row_scale) {
+            const float sc = p.row_scale[out_row];
+#pragma unroll
+            for (int q = 0; q < 32; ++q) r[q] = __float_as_uint(sc * __uint_as_float(r[q]));
+          }
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             dst[q] = make_uint4(pack_bf16(__uint_as_float(r[8 * q]), __uint_as_float(r[8 * q + 1])),

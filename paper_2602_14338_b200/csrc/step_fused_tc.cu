@@ -5,6 +5,12 @@
 //   merge_kernel               (large d only) merges the running states of the vocabulary splits
 //   scale_dz_kernel            dz = gs (g_t 1[v = y_t] - g_t exp(c_t - lse_t) p~), in place
 //   gemm_kernel<DH>, <DW>      dH rows of the chunk, dW += dz^T H
+// With one vocabulary split every row has one factor s_t = -gs g_t exp(c_t - lse_t), and the
+// rewriting pass is replaced by
+//   row_factors_kernel         p~[t, y_t] -= exp(lse_t - c_t) (so that dz = s_t p~), s_t, and the
+//                              chunk's rows of H times s_t
+//   gemm_kernel<DH>, <DW>      dH = s_t (p~ W) with the factor applied to the finished tile,
+//                              dW += p~^T (s H)
 // and once at the end the fixed-order reduction of the loss partials.
 #include "gemm_bwd_kernel.cuh"
 #include "lmhead_kernel.cuh"
@@ -13,6 +19,10 @@
 namespace {
 
 inline long long ldz_of(int32_t V) { return ((long long)V + 63) / 64 * 64; }
+// bytes of one token tile in the chunk's blocks: 128 rows of p~ / dz, and of the scaled H rows if used
+inline size_t chunk_tile_bytes(int32_t d, int32_t V) {
+  return (size_t)128 * ((size_t)ldz_of(V) * 2 + (aero_rowscale(d) ? (size_t)d * 2 : 0));
+}
 
 struct ScaleArgs {
   __nv_bfloat16* dz;        // tiled: [tile - tile_begin][ldz / 64][128][64]
@@ -74,6 +84,72 @@ __global__ void __launch_bounds__(256) scale_dz_kernel(ScaleArgs a) {
   }
 }
 
+struct RowArgs {
+  __nv_bfloat16* dz;        // tiled as above
+  int nblk;
+  const int32_t* tile_row;
+  const int32_t* tile_valid;
+  const int32_t* n_tiles;
+  int tile_begin, tile_end;
+  long long T;
+  int d;
+  const int32_t* y;
+  const float* lse;
+  const float* g;
+  const float* shift;       // [T], log2 domain
+  float grad_scale;
+  const __nv_bfloat16* H;   // [T, d]
+  __nv_bfloat16* Hs;        // [tile - tile_begin][128][d]: s_t H[t, :], zero rows where there is no token
+  float* row_scale;         // [T]: s_t
+};
+
+// One warp per row of the chunk's token tiles.  dz_tv = gs g_t (1[v = y_t] - p_tv) with
+// p_tv = p~_tv exp(c_t - lse_t), so with s_t = -gs g_t exp(c_t - lse_t) and the target's entry
+// lowered by exp(lse_t - c_t) (the sum of the row's p~), dz = s_t p~ everywhere.
+__global__ void __launch_bounds__(256) row_factors_kernel(RowArgs a) {
+  const int n_tiles = min(*a.n_tiles, a.tile_end);
+  const int lt = blockIdx.x / 16;                       // 16 blocks of 8 rows per tile
+  const int tile = a.tile_begin + lt;
+  const int r = (blockIdx.x % 16) * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  constexpr float kLog2e = 1.4426950408889634f;
+  uint4* dst = reinterpret_cast<uint4*>(a.Hs + ((size_t)lt * 128 + r) * a.d);
+  float sc = 0.f;
+  long long row = -1;
+  if (tile < n_tiles && r < a.tile_valid[tile]) {
+    row = (long long)a.tile_row[tile] + r;
+    if (row >= a.T) row = -1;
+  }
+  if (row >= 0) {
+    const float coef = a.g[row] * a.grad_scale;
+    if (coef != 0.f) {
+      const float e = a.shift[row] - a.lse[row] * kLog2e;
+      sc = -coef * exp2f(e);
+      if (lane == 0) {
+        const int yt = a.y[row];
+        __nv_bfloat16* pt = a.dz + (((size_t)lt * a.nblk + yt / 64) * 128 + r) * 64 + yt % 64;
+        *pt = __float2bfloat16_rn(__bfloat162float(*pt) - exp2f(-e));
+      }
+    }
+    if (lane == 0) a.row_scale[row] = sc;
+  }
+  if (sc == 0.f) {
+    for (int k = lane; k < a.d / 8; k += 32) dst[k] = make_uint4(0, 0, 0, 0);
+  } else {
+    const uint4* src = reinterpret_cast<const uint4*>(a.H + row * a.d);
+    for (int k = lane; k < a.d / 8; k += 32) {
+      uint4 v = src[k];
+      __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float2 f = __bfloat1622float2(h[q]);
+        h[q] = __floats2bfloat162_rn(sc * f.x, sc * f.y);
+      }
+      dst[k] = v;
+    }
+  }
+}
+
 // dH rows of dropped rollouts are defined to be zero; one warp per row.
 __global__ void __launch_bounds__(256) zero_dropped_rows_fused(long long T, int d, int R, const int64_t* __restrict__ cs,
                                                                const uint8_t* __restrict__ keep,
@@ -96,6 +172,7 @@ struct FusedWs {
   unsigned int* sync_ctr;
   float4* xstate;
   float* shift;
+  float* row_scale;
   __nv_bfloat16* dz;
   size_t head_bytes;
 };
@@ -117,6 +194,7 @@ FusedWs carve(void* ws, int64_t T, int32_t d, int32_t R) {
   f.sync_ctr = reinterpret_cast<unsigned int*>(p + off);       off += 256;
   f.xstate = reinterpret_cast<float4*>(p + off);               off += vs > 1 ? aero_align_up(vs * Tn * sizeof(float4), 256) : 0;
   f.shift = reinterpret_cast<float*>(p + off);                 off += aero_align_up(vs * Tn * sizeof(float), 256);
+  f.row_scale = reinterpret_cast<float*>(p + off);             off += aero_rowscale(d) ? aero_align_up(Tn * sizeof(float), 256) : 0;
   f.dz = reinterpret_cast<__nv_bfloat16*>(p + off);
   f.head_bytes = off;
   return f;
@@ -126,8 +204,8 @@ FusedWs carve(void* ws, int64_t T, int32_t d, int32_t R) {
 
 size_t aero_fwd_bwd_ws_bytes_tc(int64_t T, int32_t d, int32_t V, int32_t R, int64_t chunk_tokens) {
   if (chunk_tokens < 128) chunk_tokens = 128;
-  const size_t rows = (size_t)((chunk_tokens + 127) / 128 * 128);
-  return carve(nullptr, T, d, R).head_bytes + aero_align_up(rows * (size_t)ldz_of(V) * 2, 256);
+  const size_t tiles = (size_t)((chunk_tokens + 127) / 128);
+  return carve(nullptr, T, d, R).head_bytes + aero_align_up(tiles * chunk_tile_bytes(d, V), 256);
 }
 
 int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
@@ -147,7 +225,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
   if (rc) return rc;
   if (T > 0 && R > 0) {
     const long long ldz = ldz_of(V);
-    long long tpc = (long long)((ws_bytes - f.head_bytes) / ((size_t)lmhead::BM * (size_t)ldz * 2));
+    long long tpc = (long long)((ws_bytes - f.head_bytes) / chunk_tile_bytes(d, V));
     if (tpc < 1) return AERO_ERR_WORKSPACE;
     if (tpc > f.tiles.max_tiles) tpc = f.tiles.max_tiles;
     if (tpc > 32768) tpc = 32768;                                          // grid.y of the rescaling kernel
@@ -168,6 +246,10 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
     if ((rc = aero_make_tmap_dz(ctx, &tmDZ_mn, f.dz, (uint64_t)tpc, nblk, 64, gemmbwd::BM / 64))) return rc;
     if ((rc = aero_make_tmap_blocked(ctx, &tmW_mn, W, V, d, d, 64, gemmbwd::BN / 64))) return rc;
     if ((rc = aero_make_tmap_blocked(ctx, &tmH_mn, H, T, d, d, 64, gemmbwd::BN / 64))) return rc;
+    const bool rowscale = aero_rowscale(d);
+    __nv_bfloat16* Hs = f.dz + (size_t)tpc * lmhead::BM * (size_t)ldz;      // after the chunk's p~ block
+    CUtensorMap tmHs_mn;
+    if (rowscale && (rc = aero_make_tmap_blocked(ctx, &tmHs_mn, Hs, tpc * lmhead::BM, d, d, 64, gemmbwd::BN / 64))) return rc;
 
     auto k_fwd = lmhead::lmhead_kernel<lmhead::MODE_FWD_P>;
     auto k_dh = gemmbwd::gemm_kernel<gemmbwd::KIND_DH>;
@@ -213,23 +295,35 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
         lmhead::merge_kernel<<<(int)(tpc < 8 * ctx->sm_count ? tpc : 8 * ctx->sm_count), lmhead::BM, 0, ctx->stream>>>(p, 0);
         ctx->launches += 1;
       }
-      ScaleArgs sa;
-      sa.dz = f.dz; sa.nblk = (int)nblk; sa.tile_row = f.tiles.tile_row; sa.tile_valid = f.tiles.tile_valid;
-      sa.n_tiles = f.tiles.n_tiles; sa.tile_begin = (int)begin; sa.tile_end = (int)(begin + tpc);
-      sa.T = T; sa.V = V; sa.vsplit = vs; sa.nvt = nvt; sa.y = y; sa.lse = lse; sa.g = g; sa.shift = f.shift;
-      sa.grad_scale = grad_scale;
-      scale_dz_kernel<<<dim3((unsigned)((nblk + kBlocksPerCta - 1) / kBlocksPerCta), (unsigned)tpc), 256, 0, ctx->stream>>>(sa);
+      if (rowscale) {
+        RowArgs ra;
+        ra.dz = f.dz; ra.nblk = (int)nblk; ra.tile_row = f.tiles.tile_row; ra.tile_valid = f.tiles.tile_valid;
+        ra.n_tiles = f.tiles.n_tiles; ra.tile_begin = (int)begin; ra.tile_end = (int)(begin + tpc);
+        ra.T = T; ra.d = d; ra.y = y; ra.lse = lse; ra.g = g; ra.shift = f.shift; ra.grad_scale = grad_scale;
+        ra.H = static_cast<const __nv_bfloat16*>(H); ra.Hs = Hs; ra.row_scale = f.row_scale;
+        row_factors_kernel<<<(unsigned)(tpc * 16), 256, 0, ctx->stream>>>(ra);
+      } else {
+        ScaleArgs sa;
+        sa.dz = f.dz; sa.nblk = (int)nblk; sa.tile_row = f.tiles.tile_row; sa.tile_valid = f.tiles.tile_valid;
+        sa.n_tiles = f.tiles.n_tiles; sa.tile_begin = (int)begin; sa.tile_end = (int)(begin + tpc);
+        sa.T = T; sa.V = V; sa.vsplit = vs; sa.nvt = nvt; sa.y = y; sa.lse = lse; sa.g = g; sa.shift = f.shift;
+        sa.grad_scale = grad_scale;
+        scale_dz_kernel<<<dim3((unsigned)((nblk + kBlocksPerCta - 1) / kBlocksPerCta), (unsigned)tpc), 256, 0, ctx->stream>>>(sa);
+
+      }
 
       gemmbwd::Params gp = {};
       gp.T = T; gp.d = d; gp.V = V; gp.ldz = ldz;
       gp.tile_row = f.tiles.tile_row; gp.tile_valid = f.tiles.tile_valid; gp.n_tiles = f.tiles.n_tiles;
       gp.tile_begin = (int)begin; gp.tpc = (int)tpc;
       gp.dH = static_cast<__nv_bfloat16*>(dH); gp.dW = dW; gp.status = ctx->d_status;
+      gp.row_scale = rowscale ? f.row_scale : nullptr;
+      gp.h_local = rowscale ? 1 : 0;
       const long long dh_units = tpc * n_nt;
       k_dh<<<(int)(dh_units < ctx->sm_count ? dh_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
              ctx->stream>>>(tmDZ_k, tmW_mn, gp);
       k_dw<<<(int)(dw_units < ctx->sm_count ? dw_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
-             ctx->stream>>>(tmDZ_mn, tmH_mn, gp);
+             ctx->stream>>>(tmDZ_mn, rowscale ? tmHs_mn : tmH_mn, gp);
       ctx->launches += 3;
       AERO_CUDA_TRY(cudaGetLastError());
     }
