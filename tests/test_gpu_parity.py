@@ -393,8 +393,8 @@ def test_vocabulary_split_between_cta_pairs(ctx, vsplit, monkeypatch):
 @pytest.mark.parametrize("name", list(BF16_CASES) + ["tiny_fp32"])
 def test_forward_and_backward_in_one_call(ctx, name):
     """aero_grpo_loss_fwd_bwd (the forward leaves exp(z - c_t) of each chunk, the backward rescales it
-    instead of recomputing the logits) against the oracle, in one chunk and in 128-row chunks, with and
-    without a forced vocabulary split."""
+    instead of recomputing the logits) against the oracle, in one chunk and in 128-row chunks, with the
+    row factors applied in the backward GEMMs or by the rewriting pass, and with a forced vocabulary split."""
     if name == "tiny_fp32":
         wl, cover, peak, dtype = synth.WORKLOADS[0], {}, 0.0, "fp32"
     else:
@@ -410,9 +410,12 @@ def test_forward_and_backward_in_one_call(ctx, name):
     rho = ref["rho"]
     edge = (np.abs(rho - (1 + batch.ocfg.clip_hi)) < 1e-3) | (np.abs(rho - (1 - batch.ocfg.clip_lo)) < 1e-3)
     import os
-    for chunk, vsplit in ((None, None), (128, None), (128, "2")):
+    # (one split: row factors in the backward GEMMs; AERO_ROWSCALE=0 or two splits: the pass that rewrites the block)
+    for chunk, vsplit, rowscale in ((None, None, None), (128, None, None), (128, None, "0"), (128, "2", None)):
         if vsplit:
             os.environ["AERO_VSPLIT"] = vsplit
+        if rowscale:
+            os.environ["AERO_ROWSCALE"] = rowscale
         try:
             ws = None
             if chunk:
@@ -422,6 +425,7 @@ def test_forward_and_backward_in_one_call(ctx, name):
             torch.cuda.synchronize()
         finally:
             os.environ.pop("AERO_VSPLIT", None)
+            os.environ.pop("AERO_ROWSCALE", None)
         assert ctx.last_status() == 0
         check_fwd(batch, f, ref, tol[0], tol[1], 2e-2 if dtype == "bf16" else 1e-3)
         assert TL.rel_l2(dH.float().cpu().numpy()[~edge], rdH[~edge]) < tol[2]
