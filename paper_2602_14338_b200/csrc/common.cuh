@@ -112,12 +112,14 @@ static inline int aero_nsync() {
   if (const char* e = getenv("AERO_NSYNC")) return atoi(e) > 0 ? atoi(e) : 0;
   return 32;
 }
-// One-call step with one vocabulary split: the backward GEMMs take p~ as it is, with the row
-// factors applied to the dH tiles and to a scaled copy of the chunk's H rows, instead of a
-// pass that rewrites the block (AERO_ROWSCALE=0 keeps that pass).
+// One-call step: the backward GEMMs take p~ as it is, with the row factors applied to the dH
+// tiles and to a scaled copy of the chunk's H rows, instead of a pass that rewrites the block
+// (AERO_ROWSCALE=0 keeps that pass).  With several vocabulary splits this needs one shift per
+// row for all of them (lmhead::Params::common_shift).
 static inline bool aero_rowscale(int32_t d) {
+  (void)d;
   if (const char* e = getenv("AERO_ROWSCALE")) { if (atoi(e) == 0) return false; }
-  return aero_vsplit(d) == 1;
+  return true;
 }
 size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t d, int32_t R);
 int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,

@@ -99,6 +99,8 @@ struct Params {
   float* g_out;
   float* ent_out;               // entropy per row (entropy modes)
   float* shift_out;             // MODE_FWD_P: c_t * log2(e) per split and row, [vsplit][T]
+  int common_shift;             // MODE_FWD_P with vsplit > 1: every split takes c_t from the row's first 32 logits
+                                // of the whole vocabulary (the later splits compute that tile once more for it)
   double* partials;             // [tile][4 epilogue warps][kPartialStride]
   // dz modes
   const float* lse_in;
@@ -232,6 +234,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
   auto unit_first = [&](int k) { return p.tile_begin + 2 * ((pair + k * npairs) / vsplit); };
   auto unit_j0 = [&](int k) { return (int)((long long)((pair + k * npairs) % vsplit) * nvt / vsplit); };
   auto unit_j1 = [&](int k) { return (int)((long long)((pair + k * npairs) % vsplit + 1) * nvt / vsplit); };
+  // with a common shift, a unit of a later split starts with vocabulary tile 0, used for the shift alone
+  auto unit_pre = [&](int k) { return (MODE == MODE_FWD_P && p.common_shift && (pair + k * npairs) % vsplit != 0) ? 1 : 0; };
 
   if (warp == 4) {
     // ---------------- TMA producer ----------------
@@ -246,8 +250,9 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
         const int mine = unit_first(k) + (int)rank;
         const int row0 = p.tile_row[mine < n_tiles ? mine : unit_first(k)];
         int next_meet = 0;
-        for (int j = unit_j0(k), j0 = j, j1 = unit_j1(k); ok && j < j1; ++j) {
-          if (p.nsync > 0 && next_meet < p.nsync && j - j0 >= (int)((long long)next_meet * (j1 - j0) / p.nsync)) {
+        for (int j0 = unit_j0(k), jj = j0 - unit_pre(k), j1 = unit_j1(k); ok && jj < j1; ++jj) {
+          const int j = jj < j0 ? 0 : jj;
+          if (p.nsync > 0 && next_meet < p.nsync && jj - j0 >= (int)((long long)next_meet * (j1 - j0) / p.nsync)) {
             ++next_meet;
             ++meetings;
             atomicAdd(p.sync_ctr, 1u);
@@ -286,7 +291,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
       uint32_t it = 0, at = 0;
       bool ok = true;
       for (int k = 0; ok && unit_first(k) < n_tiles; ++k) {
-        for (int j = unit_j0(k), j1 = unit_j1(k); ok && j < j1; ++j, ++at) {
+        for (int j = unit_j0(k) - unit_pre(k), j1 = unit_j1(k); ok && j < j1; ++j, ++at) {
           const uint32_t buf = at & 1u, aph = (at >> 1) & 1u;
           if (!tc::mbar_wait(&ctl->tempty[buf], aph ^ 1u, abort_flag)) { ok = false; break; }
           tc::tc_fence_after();
@@ -330,6 +335,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
 
       float m2 = -INFINITY, l = 0.f, zy = 0.f, sz = 0.f;   // forward running state (log2 domain); sz = sum e^(z-m) z
       float c2 = 0.f;                                      // MODE_FWD_P: shift of the stored exponentials, log2 domain
+      bool c2_set = false;                                 // ... taken from vocabulary tile 0 by a later split
       float lse2 = 0.f, coef = 0.f, et = 0.f, c0 = 0.f;     // dz per-row constants: dz = 1[y] coef + p (c0 + et z)
       if (IS_DZ) {
         if (live) {
@@ -344,13 +350,30 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
         }
       }
 
-      for (int j = unit_j0(k), j1 = unit_j1(k); ok && j < j1; ++j, ++at) {
+      for (int j0 = unit_j0(k), jj = j0 - unit_pre(k), j1 = unit_j1(k); ok && jj < j1; ++jj, ++at) {
+        const int j = jj < j0 ? 0 : jj;
         const uint32_t buf = at & 1u, aph = (at >> 1) & 1u;
         // the TMEM loads below are warp-collective: take the decision for the whole warp
         if (!__all_sync(0xffffffffu, tc::mbar_wait(&ctl->tfull[buf], aph, abort_flag))) { ok = false; break; }
         tc::tc_fence_after();
         if (!have_tile) {
           // nothing to read: hand the accumulator straight back
+          tc::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) tc::mbar_arrive_cluster(tc::mapa_shared(tc::smem_u32(&ctl->tempty[buf]), 0));
+          continue;
+        }
+        if (jj < j0) {
+          // vocabulary tile 0 again, for the shift alone: the row's first 32 logits
+          uint32_t r0[32];
+          __syncwarp();
+          tc::tmem_ld_32x32(tmem_base + ((uint32_t)(warp * 32) << 16) + buf * BN, r0);
+          tc::tmem_ld_wait();
+          float cmax = __uint_as_float(r0[0]);
+#pragma unroll
+          for (int q = 1; q < 32; ++q) cmax = fmaxf(cmax, q < p.V ? __uint_as_float(r0[q]) : kMasked);
+          c2 = fmaf(cmax + kShiftMargin, kLog2e, 0.f);
+          c2_set = true;
           tc::tc_fence_before();
           __syncwarp();
           if (lane == 0) tc::mbar_arrive_cluster(tc::mapa_shared(tc::smem_u32(&ctl->tempty[buf]), 0));
@@ -404,7 +427,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
 #pragma unroll
             for (int q = 1; q < 32; ++q) cmax = fmaxf(cmax, z[q]);
             const float m2n = fmaxf(m2, cmax * kLog2e);
-            if (STORE_P && m2 == -INFINITY) c2 = fmaf(cmax + kShiftMargin, kLog2e, 0.f);   // first chunk of the row
+            if (STORE_P && !c2_set && m2 == -INFINITY) c2 = fmaf(cmax + kShiftMargin, kLog2e, 0.f);   // first chunk of the row
             float acc = 0.f, accz = 0.f;
             if (STORE_P) {
               // e^(z - c) = e^(z - m) * 2^(m2 - c2): one extra multiply per logit

@@ -5,8 +5,8 @@
 //   merge_kernel               (large d only) merges the running states of the vocabulary splits
 //   scale_dz_kernel            dz = gs (g_t 1[v = y_t] - g_t exp(c_t - lse_t) p~), in place
 //   gemm_kernel<DH>, <DW>      dH rows of the chunk, dW += dz^T H
-// With one vocabulary split every row has one factor s_t = -gs g_t exp(c_t - lse_t), and the
-// rewriting pass is replaced by
+// When every row has one shift c_t (one vocabulary split, or several that share the shift) it has
+// one factor s_t = -gs g_t exp(c_t - lse_t), and the rewriting pass is replaced by
 //   row_factors_kernel         p~[t, y_t] -= exp(lse_t - c_t) (so that dz = s_t p~), s_t, and the
 //                              chunk's rows of H times s_t
 //   gemm_kernel<DH>, <DW>      dH = s_t (p~ W) with the factor applied to the finished tile,
@@ -274,6 +274,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
       p.clip_lo = cfg->clip_lo; p.clip_hi = cfg->clip_hi;
       p.logp = logp; p.lse_out = lse; p.g_out = g; p.partials = f.partials;
       p.shift_out = f.shift; p.dz = f.dz; p.ldz = ldz;
+      p.common_shift = rowscale && vs > 1 ? 1 : 0;
       AERO_CUDA_TRY(cudaMemsetAsync(f.sync_ctr, 0, 256, ctx->stream));
       const long long pairs = (tpc + 1) / 2 * vs;
       const int grid = 2 * (int)(pairs < max_pairs ? pairs : max_pairs);

@@ -410,8 +410,9 @@ def test_forward_and_backward_in_one_call(ctx, name):
     rho = ref["rho"]
     edge = (np.abs(rho - (1 + batch.ocfg.clip_hi)) < 1e-3) | (np.abs(rho - (1 - batch.ocfg.clip_lo)) < 1e-3)
     import os
-    # (one split: row factors in the backward GEMMs; AERO_ROWSCALE=0 or two splits: the pass that rewrites the block)
-    for chunk, vsplit, rowscale in ((None, None, None), (128, None, None), (128, None, "0"), (128, "2", None)):
+    # (row factors in the backward GEMMs, with two splits sharing one shift per row; AERO_ROWSCALE=0: the pass
+    # that rewrites the block, with a shift per split)
+    for chunk, vsplit, rowscale in ((None, None, None), (128, None, None), (128, None, "0"), (128, "2", None), (128, "2", "0")):
         if vsplit:
             os.environ["AERO_VSPLIT"] = vsplit
         if rowscale:
