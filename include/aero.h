@@ -356,6 +356,10 @@ int aero_logprob_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, i
  * rollout batch lives in host memory.  The call copies the batch to the device,
  * runs aero_group_stats and aero_grpo_loss_fwd_bwd on the context's
  * stream, copies the scalars back and synchronises the stream before returning.
+ * H, the bulk of the bytes, is copied in 16 slices on a second stream that the context
+ * owns; each chunk of the forward waits only for the slices its token rows lie in (the
+ * call reads the chunks' row ranges back once, after the group stage), so with pinned
+ * host memory most of the transfer runs under the first chunks' kernels.
  *
  * HOST inputs (pinned memory makes the copies asynchronous): go_h [P+1] i32,
  *   reward_h [R] f32, cs_h [R+1] i64, key_h [R] u32 or NULL, alpha_h/beta_h [P] f32 or

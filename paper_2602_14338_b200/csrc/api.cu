@@ -91,6 +91,9 @@ int aero_destroy(aero_ctx* ctx) {
     if (ctx->ev0[i]) cudaEventDestroy(ctx->ev0[i]);
     if (ctx->ev1[i]) cudaEventDestroy(ctx->ev1[i]);
   }
+  for (int i = 0; i < 16; ++i)
+    if (ctx->slice_ev[i]) cudaEventDestroy(ctx->slice_ev[i]);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
   delete ctx;
   return AERO_OK;
 }

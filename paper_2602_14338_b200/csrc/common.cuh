@@ -22,6 +22,12 @@ struct aero_ctx {
   int timing;
   int n_timed;
   cudaEvent_t ev0[256], ev1[256];
+  // aero_grpo_step_host stages H in slices on a stream of its own; while it runs the fused
+  // step, every chunk waits only for the slices its token rows lie in (n_slices > 0)
+  cudaStream_t copy_stream;
+  cudaEvent_t slice_ev[16];
+  int n_slices;
+  long long rows_per_slice;
 };
 
 #define AERO_CUDA_TRY(expr)                          \

@@ -16,6 +16,8 @@
 #include "lmhead_kernel.cuh"
 #include "tmap.cuh"
 
+#include <vector>
+
 namespace {
 
 inline long long ldz_of(int32_t V) { return ((long long)V + 63) / 64 * 64; }
@@ -223,6 +225,17 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
   if (!accumulate_dW) AERO_CUDA_TRY(cudaMemsetAsync(dW, 0, (size_t)V * d * sizeof(float), ctx->stream));
   int rc = aero_build_tiles(ctx, T, R, cs, keep, lmhead::BM, f.tiles);
   if (rc) return rc;
+  // H still arriving in slices (aero_grpo_step_host): the tile list comes to the host once, so
+  // that each chunk can wait for just the slices its rows lie in
+  std::vector<int32_t> tile_row_h;
+  int32_t n_tiles_h = 0;
+  if (ctx->n_slices > 0 && T > 0 && R > 0) {
+    tile_row_h.resize((size_t)f.tiles.max_tiles);
+    AERO_CUDA_TRY(cudaMemcpyAsync(tile_row_h.data(), f.tiles.tile_row, sizeof(int32_t) * (size_t)f.tiles.max_tiles,
+                                  cudaMemcpyDeviceToHost, ctx->stream));
+    AERO_CUDA_TRY(cudaMemcpyAsync(&n_tiles_h, f.tiles.n_tiles, sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream));
+    AERO_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
+  }
   if (T > 0 && R > 0) {
     const long long ldz = ldz_of(V);
     long long tpc = (long long)((ws_bytes - f.head_bytes) / chunk_tile_bytes(d, V));
@@ -264,6 +277,14 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
     const long long dw_units = (long long)((V + gemmbwd::BM - 1) / gemmbwd::BM) * n_nt;
     const long long max_pairs = ctx->sm_count / 2 > 0 ? ctx->sm_count / 2 : 1;
     for (long long begin = 0; begin < f.tiles.max_tiles; begin += tpc) {
+      if (ctx->n_slices > 0) {
+        if (begin >= n_tiles_h) break;                        // the tile list is known: no empty chunks
+        const long long last_tile = (begin + tpc < n_tiles_h ? begin + tpc : (long long)n_tiles_h) - 1;
+        const long long last_row = (long long)tile_row_h[(size_t)last_tile] + lmhead::BM - 1;
+        long long slice = last_row / ctx->rows_per_slice;
+        if (slice > ctx->n_slices - 1) slice = ctx->n_slices - 1;
+        AERO_CUDA_TRY(cudaStreamWaitEvent(ctx->stream, ctx->slice_ev[slice], 0));
+      }
       lmhead::Params p = {};
       p.T = T; p.d = d; p.V = V; p.R = R;
       p.tile_row = f.tiles.tile_row; p.tile_valid = f.tiles.tile_valid; p.n_tiles = f.tiles.n_tiles;

@@ -79,7 +79,8 @@ int aero_grpo_step_host(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R
   // chunk size: whatever the given workspace affords beyond the fixed part
   const size_t fixed = carve_step(nullptr, P, R, T, d, V, 128, cfg->dtype).total;
   if (workspace_bytes < fixed) return AERO_ERR_WORKSPACE;
-  const size_t per_tile = cfg->dtype == AERO_FP32 ? 1 : (size_t)128 * (((size_t)V + 63) / 64 * 64) * 2;
+  const size_t per_tile = cfg->dtype == AERO_FP32 ? 1 : (size_t)128 * ((((size_t)V + 63) / 64 * 64) * 2 +
+                                                                        (aero_rowscale(d) ? (size_t)d * 2 : 0));
   int64_t chunk_tokens = 128 + (int64_t)((workspace_bytes - fixed) / per_tile) * 128;
   StepWs s = carve_step(workspace, P, R, T, d, V, chunk_tokens, cfg->dtype);
   while (s.total > workspace_bytes && chunk_tokens > 128) {     // alignment slack
@@ -98,18 +99,52 @@ int aero_grpo_step_host(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R
     AERO_CUDA_TRY(cudaMemcpyAsync(s.alpha, alpha_h, (size_t)P * 4, H2D, st));
     AERO_CUDA_TRY(cudaMemcpyAsync(s.beta, beta_h, (size_t)P * 4, H2D, st));
   }
+  // H, the bulk of the bytes, goes in slices on a stream of its own (tensor-core path): the group
+  // stage and the first chunks of the fused step run while the later slices arrive
+  const bool sliced = T > 0 && cfg->dtype != AERO_FP32;
   if (T > 0) {
-    AERO_CUDA_TRY(cudaMemcpyAsync(s.H, H_h, (size_t)T * d * esz, H2D, st));
     AERO_CUDA_TRY(cudaMemcpyAsync(s.y, y_h, (size_t)T * 4, H2D, st));
     AERO_CUDA_TRY(cudaMemcpyAsync(s.old_logp, old_logp_h, (size_t)T * 4, H2D, st));
+  }
+  if (sliced) {
+    constexpr int kSlices = 16;
+    if (!ctx->copy_stream) AERO_CUDA_TRY(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < kSlices; ++i)
+      if (!ctx->slice_ev[i]) AERO_CUDA_TRY(cudaEventCreateWithFlags(&ctx->slice_ev[i], cudaEventDisableTiming));
+    const long long rows = ((T + kSlices - 1) / kSlices + 127) / 128 * 128;
+    // whatever ran before on the caller's stream may still read the staging area
+    AERO_CUDA_TRY(cudaEventRecord(ctx->slice_ev[0], st));
+    AERO_CUDA_TRY(cudaStreamWaitEvent(ctx->copy_stream, ctx->slice_ev[0], 0));
+    for (int i = 0; i < kSlices; ++i) {
+      const long long r0 = (long long)i * rows, r1 = r0 + rows < T ? r0 + rows : T;
+      if (r0 < r1)
+        AERO_CUDA_TRY(cudaMemcpyAsync(s.H + (size_t)r0 * d * esz, static_cast<const char*>(H_h) + (size_t)r0 * d * esz,
+                                      (size_t)(r1 - r0) * d * esz, H2D, ctx->copy_stream));
+      AERO_CUDA_TRY(cudaEventRecord(ctx->slice_ev[i], ctx->copy_stream));
+    }
+    ctx->n_slices = kSlices;
+    ctx->rows_per_slice = rows;
+  } else if (T > 0) {
+    AERO_CUDA_TRY(cudaMemcpyAsync(s.H, H_h, (size_t)T * d * esz, H2D, st));
   }
   int rc = aero_group_stats(ctx, cfg, P, R, s.go, s.reward, s.cs, key_h ? s.key : nullptr, nullptr,
                             alpha_h ? s.alpha : nullptr, alpha_h ? s.beta : nullptr, s.adv, s.w, s.keep, s.gmask,
                             s.cat, s.u, s.ao, s.bo, s.kept_ids, s.kept_tok_off, s.counters, s.metrics, s.sub,
                             s.sub_bytes);
-  if (rc) return rc;
+  if (rc) {
+    ctx->n_slices = 0;
+    if (sliced) cudaStreamSynchronize(ctx->copy_stream);      // the caller may free the workspace next
+    return rc;
+  }
   rc = aero_grpo_loss_fwd_bwd(ctx, cfg, T, d, V, R, s.H, W, s.y, s.old_logp, s.cs, s.adv, s.w, s.keep, s.logp, s.lse,
                               s.g, s.loss, s.metrics + 4, 1.0f, dH, dW, accumulate_dW, s.sub, s.sub_bytes);
+  if (sliced) {
+    // the last slice may lie past the last kept row: the call still ends with all of H on the device
+    ctx->n_slices = 0;
+    const cudaError_t e = cudaStreamWaitEvent(st, ctx->slice_ev[15], 0);
+    if (rc == AERO_OK && e != cudaSuccess) rc = AERO_ERR_CUDA;
+    if (rc) cudaStreamSynchronize(ctx->copy_stream);
+  }
   if (rc) return rc;
   if (loss_h) AERO_CUDA_TRY(cudaMemcpyAsync(loss_h, s.loss, 4, D2H, st));
   if (counters_h) AERO_CUDA_TRY(cudaMemcpyAsync(counters_h, s.counters, 64, D2H, st));
