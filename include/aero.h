@@ -309,6 +309,18 @@ int aero_grpo_loss_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_
                            float grad_scale, void* dH, float* dW, int accumulate_dW,
                            void* workspace, size_t workspace_bytes);
 
+/* aero_grpo_loss_fwd_bwd with Eq. 2's KL term: ref_logp [T] f32 (NULL: no KL term, the call is
+ * aero_grpo_loss_fwd_bwd) and cfg->kl_beta, defined as for aero_grpo_loss_reg_fwd below.  The term
+ * only changes loss and g_t, so it costs nothing in the backward.  (The entropy bonus needs the
+ * logits again in the backward and is available through aero_grpo_loss_reg_fwd / _reg_bwd only.) */
+int aero_grpo_loss_kl_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                              const void* H, const void* W, const int32_t* y, const float* old_logp,
+                              const float* ref_logp,
+                              const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                              float* logp, float* lse, float* g, float* loss, float* metrics,
+                              float grad_scale, void* dH, float* dW, int accumulate_dW,
+                              void* workspace, size_t workspace_bytes);
+
 /* ------------------------------------------------------------------------------
  * Stage (b) with the regularisers of Eq. 2 and Table 9.
  *

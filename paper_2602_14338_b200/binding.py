@@ -30,7 +30,7 @@ EXPORTS = [
     "aero_step_workspace_bytes", "aero_grpo_step_host", "aero_launch_count", "aero_group_stats_static",
     "aero_grpo_loss_reg_fwd", "aero_grpo_loss_reg_bwd", "aero_logprob_fwd",
     "aero_alloc_cfg_default", "aero_allocate_workspace_bytes", "aero_allocate_sim",
-    "aero_fwd_bwd_workspace_bytes", "aero_grpo_loss_fwd_bwd", "aero_enable_kernel_timing", "aero_kernel_timing_ms",
+    "aero_fwd_bwd_workspace_bytes", "aero_grpo_loss_fwd_bwd", "aero_grpo_loss_kl_fwd_bwd", "aero_enable_kernel_timing", "aero_kernel_timing_ms",
 ]
 
 
@@ -100,6 +100,8 @@ def load_library():
     lib.aero_fwd_bwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i64]
     lib.aero_grpo_loss_fwd_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 13 + [f32] +
                                            [vp, vp, C.c_int, vp, sz])
+    lib.aero_grpo_loss_kl_fwd_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 14 + [f32] +
+                                              [vp, vp, C.c_int, vp, sz])
     lib.aero_enable_kernel_timing.argtypes = [vp, C.c_int]
     lib.aero_kernel_timing_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
     lib.aero_step_workspace_bytes.restype = sz
@@ -362,9 +364,9 @@ class Context:
         return self.lib.aero_fwd_bwd_workspace_bytes(T, d, V, R, chunk_tokens)
 
     def grpo_loss_fwd_bwd(self, cfg, H, W, y, old_logp, cs, adv, w, keep, out=None, grad_scale=1.0, dH=None, dW=None,
-                          accumulate_dW=False, chunk_tokens=None, workspace=None):
-        """aero_grpo_loss_fwd_bwd: forward and backward of stage (b) in one call (no recompute of the logits).
-        Returns (forward outputs dict, dH, dW)."""
+                          accumulate_dW=False, chunk_tokens=None, workspace=None, ref_logp=None):
+        """aero_grpo_loss_fwd_bwd (aero_grpo_loss_kl_fwd_bwd when ref_logp is given): forward and backward of
+        stage (b) in one call (no recompute of the logits).  Returns (forward outputs dict, dH, dW)."""
         T, d = H.shape
         V = W.shape[0]
         R = cs.numel() - 1
@@ -385,14 +387,17 @@ class Context:
             if chunk_tokens is None:
                 chunk_tokens = min(max(128, (T + 127) // 128 * 128), 2 * 148 * 128)
             workspace = self.workspace(self.fwd_bwd_workspace_bytes(T, d, V, R, chunk_tokens))
-        rc = self.lib.aero_grpo_loss_fwd_bwd(
-            self.h, C.byref(cfg), T, d, V, R, _ptr(H, dt, T * d, "H"), _ptr(W, dt, V * d, "W"),
-            _ptr(y, torch.int32, T, "y"), _ptr(old_logp, torch.float32, T, "old_logp"),
-            _ptr(cs, torch.int64, R + 1, "cs"), _ptr(adv, torch.float32, R, "adv"), _ptr(w, torch.float32, R, "w"),
-            _ptr(keep, torch.uint8, R, "keep"), _ptr(o["logp"]), _ptr(o["lse"]), _ptr(o["g"]), _ptr(o["loss"]),
-            _ptr(o["metrics"]), C.c_float(grad_scale), _ptr(dH, dt, T * d, "dH"), _ptr(dW, torch.float32, V * d, "dW"),
-            1 if accumulate_dW else 0, workspace.data_ptr(), workspace.numel())
-        _check(rc, "aero_grpo_loss_fwd_bwd")
+        head = (self.h, C.byref(cfg), T, d, V, R, _ptr(H, dt, T * d, "H"), _ptr(W, dt, V * d, "W"),
+                _ptr(y, torch.int32, T, "y"), _ptr(old_logp, torch.float32, T, "old_logp"))
+        tail = (_ptr(cs, torch.int64, R + 1, "cs"), _ptr(adv, torch.float32, R, "adv"), _ptr(w, torch.float32, R, "w"),
+                _ptr(keep, torch.uint8, R, "keep"), _ptr(o["logp"]), _ptr(o["lse"]), _ptr(o["g"]), _ptr(o["loss"]),
+                _ptr(o["metrics"]), C.c_float(grad_scale), _ptr(dH, dt, T * d, "dH"), _ptr(dW, torch.float32, V * d, "dW"),
+                1 if accumulate_dW else 0, workspace.data_ptr(), workspace.numel())
+        if ref_logp is None:
+            _check(self.lib.aero_grpo_loss_fwd_bwd(*head, *tail), "aero_grpo_loss_fwd_bwd")
+        else:
+            _check(self.lib.aero_grpo_loss_kl_fwd_bwd(*head, _ptr(ref_logp, torch.float32, T, "ref_logp"), *tail),
+                   "aero_grpo_loss_kl_fwd_bwd")
         return o, dH, dW
 
     def grpo_loss_bwd(self, cfg, H, W, y, cs, keep, lse, g, grad_scale=1.0, dH=None, dW=None,

@@ -212,6 +212,7 @@ size_t aero_fwd_bwd_ws_bytes_tc(int64_t T, int32_t d, int32_t V, int32_t R, int6
 
 int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                     const void* H, const void* W, const int32_t* y, const float* old_logp,
+                    const float* ref_logp, float kl_beta,
                     const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
                     float* logp, float* lse, float* g, float* loss, float* metrics,
                     float grad_scale, void* dH, float* dW, int accumulate_dW, void* ws, size_t ws_bytes) {
@@ -292,6 +293,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
       p.y = y; p.status = ctx->d_status;
       p.vsplit = vs; p.xstate = f.xstate; p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync();
       p.old_logp = old_logp; p.cs = cs; p.adv = adv; p.w = w;
+      p.ref_logp = ref_logp; p.kl_beta = ref_logp ? kl_beta : 0.f;
       p.clip_lo = cfg->clip_lo; p.clip_hi = cfg->clip_hi;
       p.logp = logp; p.lse_out = lse; p.g_out = g; p.partials = f.partials;
       p.shift_out = f.shift; p.dz = f.dz; p.ldz = ldz;

@@ -584,6 +584,46 @@ def test_regularised_objective(ctx, name):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_kl_term_in_the_one_call_step(ctx, dtype):
+    """aero_grpo_loss_kl_fwd_bwd: Eq. 2's KL term through the one-call step (it only changes loss and g_t)
+    against the oracle, and against the two-call path with the same term."""
+    base = synth.WORKLOADS[0] if dtype == "fp32" else synth.scaled(
+        synth.WORKLOADS[1], P=6, n_lo=3, n_hi=9, d=256, V=3001, len_median=50.0, len_cap=200, dtype="bf16", seed=31)
+    batch = TL.Batch(base, O.Cfg(seed=base.seed, kl_beta=0.5), peak=0.0)
+    ocfg, rg = batch.ocfg, batch.ref_g
+    rng = np.random.default_rng(6)
+    ref_lp = (batch.old.astype(np.float64) + 0.3 * rng.standard_normal(batch.T)).astype(np.float32)
+    adv32 = rg["adv"].astype(np.float32).astype(np.float64)
+    w32 = rg["w"].astype(np.float32).astype(np.float64)
+    ref = O.grpo_loss_reg_fwd(ocfg, batch.H, batch.W, batch.st.y, batch.old, ref_lp, batch.st.cs, adv32, w32, rg["keep"])
+    rdH, rdW = O.grpo_loss_reg_bwd(ocfg, batch.H, batch.W, batch.st.y, batch.st.cs, rg["keep"], ref["lse"], ref["g"],
+                                   ref["entropy"], w32)
+    cfg = TL.lib_cfg(ocfg, dtype)
+    dv = batch.to_device()
+    f, dH, dW = ctx.grpo_loss_fwd_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"], dv["keep"],
+                                      ref_logp=TL.dev(ref_lp))
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    tol = (1e-4, 1e-4, 1e-4) if dtype == "fp32" else (LOGP_ABS, LOSS_REL, GRAD_L2)
+    assert np.abs(f["logp"][:batch.T].cpu().numpy() - ref["logp"]).max() <= tol[0]
+    assert abs(f["loss"].item() - ref["loss"]) <= tol[1] * abs(ref["loss"]) + 1e-7
+    rho = ref["rho"]
+    edge = (np.abs(rho - (1 + ocfg.clip_hi)) < 1e-3) | (np.abs(rho - (1 - ocfg.clip_lo)) < 1e-3)
+    np.testing.assert_allclose(f["g"][:batch.T].cpu().numpy()[~edge], ref["g"][~edge], rtol=2e-2, atol=1e-9)
+    assert TL.rel_l2(dH.float().cpu().numpy()[~edge], rdH[~edge]) < tol[2]
+    if not edge.any():
+        assert TL.rel_l2(dW.cpu().numpy(), rdW) < tol[2]
+    # the term is not vacuous: without it the gradient differs by far more than the tolerance
+    plain = O.grpo_loss_fwd(ocfg, batch.H, batch.W, batch.st.y, batch.old, batch.st.cs, adv32, w32, rg["keep"])
+    pdH, _ = O.grpo_loss_bwd(batch.H, batch.W, batch.st.y, batch.st.cs, rg["keep"], plain["lse"], plain["g"])
+    assert TL.rel_l2(pdH, rdH) > 5 * tol[2]
+    # the two-call path with the same term gives the same per-token coefficients
+    f2 = ctx.grpo_loss_reg_fwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], TL.dev(ref_lp), dv["cs"], dv["adv"], dv["w"],
+                               dv["keep"], entropy=False)
+    np.testing.assert_allclose(f["g"][:batch.T].cpu().numpy(), f2["g"][:batch.T].cpu().numpy(), rtol=1e-4, atol=1e-9)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_logprob_pass_alone(ctx, dtype):
     """aero_logprob_fwd over all rows (no groups, no objective): the pass that produces old and
     reference log-probs, against log_softmax of the oracle's logits; entropy output included."""
