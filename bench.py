@@ -356,8 +356,8 @@ def run_ours(args):
 
 
 def variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, g, dH, dW, ws_b, T_kept, pk):
-    """The step with Eq. 2's KL term and the entropy bonus (aero_grpo_loss_reg_fwd/_bwd), and the
-    log-prob pass alone (aero_logprob_fwd) that produces old / reference log-probs."""
+    """The step with Eq. 2's KL term and the entropy bonus (aero_grpo_loss_reg_fwd/_bwd), the one-call step
+    with the KL term (aero_grpo_loss_kl_fwd_bwd), and the log-prob pass alone (aero_logprob_fwd) that produces old / reference log-probs."""
     import copy
     import torch
 
@@ -384,6 +384,11 @@ def variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, g, dH, dW, ws_b, T_kept,
                               workspace=ws_b)
 
     ms_reg = timed(reg_step)
+    kcfg = copy.copy(cfg)
+    kcfg.kl_beta = 0.04
+    kb = {}
+    ms_kl = timed(lambda: ctx.grpo_loss_fwd_bwd(kcfg, H, W, y, old, cs, g["adv"], g["w"], g["keep"], out=kb, dH=dH, dW=dW,
+                                                workspace=ws_b, ref_logp=ref))
     ms_lp = timed(lambda: ctx.logprob_fwd(rcfg, H, W, y, out=lb))
     # allocation controller on 2^22 simulated prompts with success rates ~ Beta(0.5, 0.5)
     from paper_2602_14338_b200 import binding as B
@@ -414,6 +419,9 @@ def variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, g, dH, dW, ws_b, T_kept,
             "regularised_step": {"kl_beta": 0.04, "ent_coef": 1e-3, "ms": ms_reg, "tokens_per_s": T_kept / (ms_reg * 1e-3),
                                  "executed_tflops": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12,
                                  "frac_of_sustained": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12 / pk["sustained"]},
+            "kl_step_one_call": {"kl_beta": 0.04, "ms": ms_kl, "tokens_per_s": T_kept / (ms_kl * 1e-3),
+                                 "executed_tflops": 3 * fl * T_kept / (ms_kl * 1e-3) / 1e12,
+                                 "frac_of_sustained": 3 * fl * T_kept / (ms_kl * 1e-3) / 1e12 / pk["sustained"]},
             "logprob_pass": {"rows": T, "ms": ms_lp, "tokens_per_s": T / (ms_lp * 1e-3),
                              "tflops": fl * T / (ms_lp * 1e-3) / 1e12, "frac_of_burst": fl * T / (ms_lp * 1e-3) / 1e12 / pk["burst"]}}
 
