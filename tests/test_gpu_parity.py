@@ -442,6 +442,35 @@ def test_forward_and_backward_in_one_call(ctx, name):
             assert TL.rel_l2(soft_gpu[live], soft_ref[live]) < 3e-2
 
 
+def test_one_call_step_reports_a_logit_out_of_range(ctx):
+    """The one-call step stores exp(z - c_t) in bf16 with c_t taken from the row's first 32 logits; a logit more
+    than about 127 above them cannot be held and raises AERO_ST_RANGE (nothing traps, the other rows are
+    unaffected); the two-call path takes the same batch without a status bit."""
+    wl = synth.scaled(synth.WORKLOADS[1], P=4, n_lo=3, n_hi=6, d=128, V=2000, len_median=40.0, len_cap=120, dtype="bf16",
+                      seed=57)
+    batch = TL.Batch(wl, O.Cfg(seed=wl.seed), peak=0.0)
+    cfg = TL.lib_cfg(batch.ocfg, "bf16")
+    dv = batch.to_device()
+    owner = O.token_rollout(batch.st.cs, batch.T)
+    t = int(np.nonzero(batch.ref_g["keep"][owner] != 0)[0][3])
+    H, W = dv["H"].clone(), dv["W"].clone()
+    H[t] = 2.0                                 # z[t, 1500] = 128 * 2 * 1.5 = 384; the first 32 logits of the row stay small
+    W[1500] = 1.5
+    W[:32] *= 0.01
+    good, _, _ = ctx.grpo_loss_fwd_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"], dv["keep"])
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    f, dH, dW = ctx.grpo_loss_fwd_bwd(cfg, H, W, dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"], dv["keep"])
+    torch.cuda.synchronize()
+    assert ctx.last_status() & B.AERO_ST_RANGE
+    assert ctx.last_status() == 0
+    assert torch.isfinite(f["logp"]).all() and torch.isfinite(dH.float()).all()
+    f2 = ctx.grpo_loss_fwd(cfg, H, W, dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"], dv["keep"])
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    np.testing.assert_allclose(f["logp"][:batch.T].cpu().numpy(), f2["logp"][:batch.T].cpu().numpy(), atol=2e-5)
+
+
 def test_bwd_chunking_and_accumulation(ctx):
     over, cover, _ = BF16_CASES["aero_dropped"]
     wl = synth.scaled(synth.WORKLOADS[1], **over)
