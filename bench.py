@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 METRIC = "rollout tokens/sec, fused GRPO logprob+loss fwd+bwd"
 # dram__bytes_read.sum + dram__bytes_write.sum of one lmhead_kernel<MODE_FWD> launch on the full-size workload,
 # from the one-pass ncu captures summarised in profiles/lmhead_fwd_full_size_dram.md (per workload index).
-NCU_FWD_TRAFFIC = {1: {"bytes": 5.795e9, "tokens": 204780}, 2: {"bytes": 85.26e9, "tokens": 468700}}
+NCU_FWD_TRAFFIC = {1: {"bytes": 6.057e9, "tokens": 204780}, 2: {"bytes": 197.6e9, "tokens": 468700}}
 # the same for the launches of lmhead_kernel<MODE_FWD_P> of one step (they also write the chunk blocks)
 NCU_FWDP_TRAFFIC = {1: {"bytes": 71.87e9, "tokens": 204780}, 2: {"bytes": 315.6e9, "tokens": 468700}}
 NCU_FWD_TRAFFIC_SOURCE = "ncu capture of the full-size launch (dram__bytes_read.sum + dram__bytes_write.sum)"
