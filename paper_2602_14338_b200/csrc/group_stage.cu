@@ -195,8 +195,10 @@ __device__ __forceinline__ Rule decide(const Args& a, int p, int n, int c) {
 // a warp's share).
 struct PromptRule {
   float adv_correct, adv_incorrect;   // advantage of a kept rollout by its reward bit
-  unsigned range;      // first rollout | one past the last << 16, relative to the share's first rollout
-  unsigned sel;        // bit 0: keep none; bit 1: the incorrect rollouts are ranked; bit 2: the correct ones are; quota << 4
+  unsigned range;      // first rollout | one past the last << 16, relative to the share's first rollout; or, with
+                       // bit 3 of sel, the high word of the largest sort word a selection keeps
+  unsigned sel;        // bit 0: keep none; bit 1: the incorrect rollouts are ranked; bit 2: the correct ones are;
+                       // bit 3: a ranked rollout is kept iff its sort word's high half is at most `range`; quota << 4
 };
 
 // Staging of one warp's share.  `ck` orders the candidates of a selection and carries the
@@ -319,6 +321,45 @@ __device__ __forceinline__ void group_moments(const Args& a, const Rule& ru, int
   *inv_out = 1.f / (sd + a.cfg.eps_std);
 }
 
+// Selection in a group of at most N rollouts by threshold: the high halves of the group's sort
+// words (correct << 31 | key >> 1; all ones for an absent rollout and past the group's end) go
+// through Batcher's odd-even merge sort as a fixed network of min/max on registers, every index a
+// compile-time constant.  With v the sorted halves, a rollout of rank below `idx + 1` has a half
+// at most v[idx]; the converse holds when v[idx + 1] > v[idx].  Returns whether it does (else
+// the group is ranked by the loop, which compares whole words) and v[idx] in *thr.
+template <int N>
+__device__ __forceinline__ bool threshold_half(const unsigned long long* grp, int n, int idx, unsigned* thr) {
+  unsigned v[N];
+  const unsigned* half = reinterpret_cast<const unsigned*>(grp) + 1;
+#pragma unroll
+  for (int t = 0; t < N; ++t) v[t] = t < n ? half[2 * t] : 0xffffffffu;
+  // pass (p, k) compares a with a + k for every a whose offset from k % p, taken modulo 2k, is
+  // below k, when both lie in the same block of 2p
+#pragma unroll
+  for (int p = 1; p < N; p <<= 1) {
+#pragma unroll
+    for (int k = p; k >= 1; k >>= 1) {
+#pragma unroll
+      for (int a = 0; a < N; ++a) {
+        const int r = k % p, b = a + k;
+        if (a >= r && (a - r) % (2 * k) < k && b < N && a / (2 * p) == b / (2 * p)) {
+          const unsigned x = v[a], y = v[b];
+          v[a] = min(x, y);
+          v[b] = max(x, y);
+        }
+      }
+    }
+  }
+  unsigned lo = v[0], up = v[1];
+#pragma unroll
+  for (int t = 1; t + 1 < N; ++t) {
+    lo = idx == t ? v[t] : lo;
+    up = idx == t ? v[t + 1] : up;
+  }
+  *thr = lo;
+  return up > lo;
+}
+
 // A share whose rollouts fit the warp's staging area, have between 1 and 2^22 - 1 tokens each
 // and rewards of exactly 0 or 1.  Rewards enter as the bit r > 0.5, so per-prompt sums are bit counts and mean and deviation are closed
 // forms of the counts; the number of rollouts a selection keeps is known from the rule alone,
@@ -365,6 +406,7 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
   __syncwarp();
 
   // ---- per prompt: counts, category, posterior, curation rule, moments of the base set ----
+  int sort_n = 0, sort_idx = 0;      // a selection in a group of at most 16: its size and the place of its threshold
   if (lane < sh.np) {
     const int p = sh.p0 + lane;
     const int n = HAS_KEEP_IN ? range_popc(S.pmask, sh.lo, sh.hi) : sh.hi - sh.lo;
@@ -395,8 +437,10 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
     // every incorrect rollout orders before every correct one: when the correct ones are the
     // candidates, the n - c incorrect ones are counted by each rank and the quota allows for them
     const bool sel = ru.mode == 2;
+    const int quota = (int)ru.quota + (ru.reject == 2 ? n - c : 0);
+    if (sel && sh.hi - sh.lo <= 16 && quota > 0 && quota < sh.hi - sh.lo) { sort_n = sh.hi - sh.lo; sort_idx = quota - 1; }
     pr.sel = (ru.mode == 1 ? 1u : 0u) | (sel && ru.reject != 2 ? 2u : 0u) | (sel && ru.reject != 1 ? 4u : 0u) |
-             ((unsigned)((int)ru.quota + (ru.reject == 2 ? n - c : 0)) << 4);
+             ((unsigned)quota << 4);
     S.rule[lane] = pr;
     mine.present_roll = n;
 #pragma unroll
@@ -404,9 +448,20 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
     mine.surv = nk > 0 ? 1 : 0;
     mine.abs_adv = ((float)ck * fabsf(1.f - mu) + (float)(nk - ck) * fabsf(mu)) * inv;
   }
+  // ---- per prompt with a selection in a small group: its threshold, where that decides exactly ----
+  const int widest = (int)__reduce_max_sync(0xffffffffu, (unsigned)sort_n);
+  if (widest > 0) {
+    unsigned thr = 0;
+    const bool exact = widest > 8 ? threshold_half<16>(S.ck + sh.lo, sort_n, sort_idx, &thr)
+                                  : threshold_half<8>(S.ck + sh.lo, sort_n, sort_idx, &thr);
+    if (sort_n > 0 && exact) {
+      S.rule[lane].range = thr;
+      S.rule[lane].sel |= 8u;
+    }
+  }
   __syncwarp();
 
-  // ---- per rollout: keep decision (rank among the group's candidates), advantage ----
+  // ---- per rollout: keep decision (threshold, or rank among the group's candidates), advantage ----
   int cnt = 0;
   unsigned ktok = 0;       // at most kWChunks lengths below 2^22 per lane
   for (int c = 0; c * 32 < nroll; ++c) {
@@ -418,9 +473,12 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
     const bool corr = (S.cmask[c] >> lane) & 1u;
     bool kp = pres && !(pr.sel & 1u);
     const bool ranked = pres && (pr.sel & (corr ? 4u : 2u));
-    // the loop runs as long as the longest group among the chunk's ranked rollouts, the same for all lanes
-    const int lo = (int)(pr.range & 0xffffu);
-    const int span = ranked ? (int)(pr.range >> 16) - lo : 0;
+    const bool by_half = (pr.sel & 8u) != 0;
+    if (ranked && by_half) kp = (unsigned)(mykey >> 32) <= pr.range;
+    // the others: the loop runs as long as the longest group among the chunk's rollouts ranked by it, the
+    // same for all lanes
+    const int lo = by_half ? 0 : (int)(pr.range & 0xffffu);
+    const int span = ranked && !by_half ? (int)(pr.range >> 16) - lo : 0;
     const int longest = (int)__reduce_max_sync(0xffffffffu, (unsigned)span);
     if (longest > 0) {
       // (reads past the lane's own group stay inside the block's shared memory and are not counted)
@@ -431,7 +489,7 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
         const unsigned long long other = grp[d];
         rank += (d < span && other < mykey) ? 1 : 0;
       }
-      if (ranked) kp = rank < (int)(pr.sel >> 4);
+      if (span > 0) kp = rank < (int)(pr.sel >> 4);
     }
     const unsigned km = __ballot_sync(0xffffffffu, kp);
     if (valid) {
