@@ -784,17 +784,20 @@ __global__ void __launch_bounds__(kThreads) emit_kernel(Args a, Workspace ws, in
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int tile = blockIdx.x;
   uint32_t st = 0;      // bad offsets were reported by the first launch
-  const Share sh = load_share(a, tile * kWarps + warp, pw, st);
-  if (sh.np == 0 || sh.nroll == 0) return;
+  // kept rollouts and tokens before this share: earlier runs, earlier tiles of the run, earlier warps of
+  // the tile (these loads do not depend on the share's offsets and are issued ahead of them)
   const Globals g = *ws.glob;
-  // kept rollouts and tokens before this share: earlier runs, earlier tiles of the run, earlier warps of the tile
   int pos0 = lane < warp ? ws.share_cnt[tile * kWarps + lane] : 0;
   long long tok0 = lane < warp ? ws.share_tok[tile * kWarps + lane] : 0;
+  const int before_cnt = ws.run_cnt[tile / kRunTiles] + ws.tile_cnt[tile];
+  const long long before_tok = ws.run_tok[tile / kRunTiles] + ws.tile_tok[tile];
+  const Share sh = load_share(a, tile * kWarps + warp, pw, st);
+  if (sh.np == 0 || sh.nroll == 0) return;
   pos0 = __reduce_add_sync(0xffffffffu, pos0);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) tok0 += __shfl_xor_sync(0xffffffffu, tok0, o);
-  pos0 += ws.run_cnt[tile / kRunTiles] + ws.tile_cnt[tile];
-  tok0 += ws.run_tok[tile / kRunTiles] + ws.tile_tok[tile];
+  pos0 += before_cnt;
+  tok0 += before_tok;
   const unsigned below = (1u << lane) - 1u;
   // one chunk of 32 rollouts, its keep flags and lengths already loaded
   auto emit_chunk = [&](int c0, int i, bool valid, bool kp, int len) {
