@@ -3,11 +3,14 @@
 //
 //   curate_kernel   one warp per share of up to 32 consecutive prompts, eight shares to a tile.
 //                   A warp stages its share's rollouts with coalesced loads (sort words with
-//                   the lengths in shared memory, presence and correctness as bit masks) and runs the per-prompt steps (counts, category, posterior, curation
-//                   rule, mean/std) one lane per prompt and the per-rollout steps (rank among
-//                   (key, index), keep, advantage) one lane per rollout.  Warps never wait for
-//                   one another; each leaves its totals of kept rollouts and tokens, each tile
-//                   its sums of them and its metrics record.
+//                   the lengths in shared memory, presence and correctness as bit masks) and
+//                   runs the per-prompt steps (counts, category, posterior, curation rule,
+//                   mean/std, and for a selection in a group of at most 16 its threshold from
+//                   a sorting network on registers) one lane per prompt and the per-rollout
+//                   steps (keep by threshold or by rank among (key, index), advantage) one
+//                   lane per rollout.  Warps never wait for one another; each leaves its
+//                   totals of kept rollouts and tokens, each tile its sums of them and its
+//                   metrics record.
 //   run_prefix_kernel, totals_kernel
 //                   exclusive prefixes of the tiles' totals in two levels (runs of 1024 tiles,
 //                   then the runs), the batch totals, counters and metrics (fixed order).
