@@ -15,12 +15,12 @@
 //                   exclusive prefixes of the tiles' totals in two levels (runs of 1024 tiles,
 //                   then the runs), the batch totals, counters and metrics (fixed order).
 //   emit_kernel     the same shares again: compacted ids and token offsets of the kept rollouts
-//                   from the keep flags and the prefixes, per-rollout weights (which need the
+//                   from the first pass's kept bits and lengths and the prefixes, per-rollout weights (which need the
 //                   batch totals), and the tails of the compacted arrays.
 //
-// Splitting where the batch-wide prefix is needed costs a second read of the keep flags and the
-// token offsets (9 bytes per rollout) and saves every wait between blocks: no launch depends on
-// the order in which its blocks run.  A share whose rollouts do not fit the warp's staging area
+// Splitting where the batch-wide prefix is needed costs the second pass a read of 4 bytes per
+// rollout (the first pass leaves kept bit | length where the weight will go) and saves every wait
+// between blocks: no launch depends on the order in which its blocks run.  A share whose rollouts do not fit the warp's staging area
 // (a huge group, or a rollout of 2^22 tokens or more) runs the first launch's steps straight from
 // global memory, one lane per prompt.
 #include "common.cuh"
@@ -36,6 +36,7 @@ constexpr int kWCap = 416;             // rollouts a warp can stage
 constexpr int kWChunks = kWCap / 32;
 constexpr int kLenBits = 22;           // staged rollouts are shorter than 2^22 tokens
 constexpr unsigned kLenMask = (1u << kLenBits) - 1u;
+constexpr unsigned kKeptBit = 1u << 31;    // first pass -> second pass, in w: kept bit | length (at most 2^31 - 1)
 constexpr int kMaxPW = 32;             // prompts per warp: one lane each in the per-prompt steps
 constexpr int kWTarget = 300;          // mean rollouts per warp the host aims at
 constexpr int kRunThreads = 256;
@@ -498,6 +499,7 @@ __device__ __forceinline__ bool curate_staged(const Args& a, const Workspace& ws
     if (valid) {
       a.adv[r0 + j] = kp ? (corr ? pr.adv_correct : pr.adv_incorrect) : 0.f;
       a.keep[r0 + j] = kp ? 1 : 0;
+      a.w[r0 + j] = __uint_as_float(kp ? kKeptBit | ((unsigned)mykey & kLenMask) : 0u);     // for the second pass
     }
     cnt += __popc(km);
     ktok += kp ? (unsigned)mykey & kLenMask : 0u;
@@ -561,8 +563,10 @@ __device__ void curate_global(const Args& a, const Workspace& ws, const Share& s
         }
         kp = rank < ru.quota;
       }
+      const int len = clamped_len(a.cs[r0 + j + 1] - a.cs[r0 + j]);
       a.keep[r0 + j] = kp ? 1 : 0;
-      if (kp) { nk += 1; ck += corr ? 1 : 0; ktok += clamped_len(a.cs[r0 + j + 1] - a.cs[r0 + j]); }
+      a.w[r0 + j] = __uint_as_float(kp ? kKeptBit | (unsigned)len : 0u);                    // for the second pass
+      if (kp) { nk += 1; ck += corr ? 1 : 0; ktok += len; }
     }
     const bool over_kept = a.cfg.stats_over == AERO_STATS_KEPT;
     float mu, inv;
@@ -861,10 +865,10 @@ __global__ void __launch_bounds__(kThreads) emit_kernel(Args a, Workspace ws, in
     const int j0 = c0 + lane, j1 = j0 + 32;
     const bool v0 = j0 < sh.nroll, v1 = j1 < sh.nroll;
     const int i0 = sh.r0 + min(j0, sh.nroll - 1), i1 = sh.r0 + min(j1, sh.nroll - 1);
-    const uint8_t k0 = a.keep[i0], k1 = a.keep[i1];
-    const long long b0 = a.cs[i0], e0 = a.cs[i0 + 1], b1 = a.cs[i1], e1 = a.cs[i1 + 1];
-    emit_chunk(c0, i0, v0, v0 && k0 != 0, clamped_len(e0 - b0));
-    if (c0 + 32 < sh.nroll) emit_chunk(c0 + 32, i1, v1, v1 && k1 != 0, clamped_len(e1 - b1));
+    // what the first pass left in w: the kept bit and the rollout's length
+    const unsigned k0 = __float_as_uint(a.w[i0]), k1 = __float_as_uint(a.w[i1]);
+    emit_chunk(c0, i0, v0, v0 && (k0 & kKeptBit), (int)(k0 & ~kKeptBit));
+    if (c0 + 32 < sh.nroll) emit_chunk(c0 + 32, i1, v1, v1 && (k1 & kKeptBit), (int)(k1 & ~kKeptBit));
   }
 }
 
