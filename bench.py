@@ -5,16 +5,22 @@ forward + backward, in rollout tokens per second.
     python bench.py --gpus 1 --steps 10 --warmup 3            # CUDA library (default)
     python bench.py --impl reference --steps 2 --warmup 1     # the fp64 CPU oracle, timed
 
-One step = one pass of the whole path over one synthetic batch of the workload
-(default: the Qwen2.5-Math-1.5B shaped batch).  Prints one JSON line on rank 0.
-With N > 1 ranks (torchrun) every rank runs an independent replica of the step on
-its own batch; there is no data-path collective.
+One step = one pass of the whole path over one synthetic batch of the workload.  The
+default workload is the largest one that fits one GPU, the stress batch at the Qwen2.5-7B
+shape (d = 3584, V = 152064, about 4.5 M input tokens); the three smaller bf16 workloads
+are timed with a few steps each and reported as sub-records.  Prints one JSON line on
+rank 0.  With N > 1 ranks (torchrun, or `--gpus N`, which starts the ranks itself) every
+rank takes its own batch of prompts against a replicated W, and the step includes the
+exchange of a data-parallel step: all-reduce of the group counters, weights brought to the
+batch-wide denominators, all-reduce of dW and of the loss.
 """
 from __future__ import annotations
 
 import argparse
+import gc
 import json
 import os
+import socket
 import subprocess
 import sys
 import tempfile
@@ -27,13 +33,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "rollout tokens/sec, fused GRPO logprob+loss fwd+bwd"
-# dram__bytes_read.sum + dram__bytes_write.sum of one lmhead_kernel<MODE_FWD> launch on the full-size workload,
-# from the one-pass ncu captures summarised in profiles/lmhead_fwd_full_size_dram.md (per workload index).
-NCU_FWD_TRAFFIC = {1: {"bytes": 6.057e9, "tokens": 204780}, 2: {"bytes": 197.6e9, "tokens": 468700}}
-# the same for the launches of lmhead_kernel<MODE_FWD_P> of one step (they also write the chunk blocks)
-NCU_FWDP_TRAFFIC = {1: {"bytes": 71.87e9, "tokens": 204780}, 2: {"bytes": 315.6e9, "tokens": 468700}}
-NCU_FWD_TRAFFIC_SOURCE = "ncu capture of the full-size launch (dram__bytes_read.sum + dram__bytes_write.sum)"
 UNIT = "tokens/s"
+NOMINAL_BF16_TFLOPS = 2250.0          # dense bf16 of the data sheet; the targets are stated against it
+TARGET_STAGE_B, TARGET_STAGE_A = 0.60, 0.70
 
 
 def parse_args():
@@ -42,16 +44,18 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1, help="workload index 0..4")
+    ap.add_argument("--config", type=int, default=4, help="workload index 0..4 of the headline line")
     ap.add_argument("--chunk-tokens", type=int, default=4 * 148 * 128)
     ap.add_argument("--prompts", type=int, default=0, help="override the number of prompts (reduced runs for profiling)")
+    ap.add_argument("--sub-workloads", default="1,2,3", help="workloads timed briefly and reported as sub-records")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-group-leg", action="store_true")
     ap.add_argument("--no-variants-leg", action="store_true",
-                    help="skip the timings of the regularised step (KL + entropy) and of the log-prob pass alone")
+                    help="skip the regularised step, the log-prob pass alone, the allocation simulation and the k sweep")
     ap.add_argument("--only-group-leg", action="store_true",
                     help="run only the large-input group-stage measurement (for profiling that stage alone)")
+    ap.add_argument("--only-main", action="store_true", help="only the timed steps of the headline workload")
     return ap.parse_args()
 
 
@@ -117,7 +121,6 @@ class ClockSampler:
 def oracle_sample(wl, st, n_tokens):
     """The first n_tokens token rows of the workload as one group (rollouts truncated at the
     sample boundary), as fp64 arrays for the oracle.  Inputs only; no result of the CUDA path."""
-    import torch
     from paper_2602_14338_b200 import synth
 
     n_tokens = int(min(n_tokens, st.cs[-1]))
@@ -193,68 +196,127 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- CUDA arm
+class Prepared:
+    """One workload resident on the device: inputs, outputs and the workspace of the step."""
+
+    def __init__(self, ctx, dev, idx, rank, chunk_tokens, prompts=0):
+        import torch
+        from paper_2602_14338_b200 import binding as B
+        from paper_2602_14338_b200 import synth
+
+        self.ctx, self.dev = ctx, dev
+        self.base = synth.WORKLOADS[idx]
+        wl = synth.scaled(self.base, seed=self.base.seed + 100 * rank)      # an independent batch of prompts per rank
+        if prompts > 0:
+            wl = synth.scaled(wl, P=prompts)
+        self.wl = wl
+        self.st = st = synth.make_structure(wl)
+        self.P, self.R, self.T = len(st.go) - 1, len(st.reward), int(st.cs[-1])
+        self.H, self.W = synth.make_tensors(wl, self.T, device=dev)
+        over = dict(seed=wl.seed, dtype=B.AERO_BF16 if wl.dtype == "bf16" else B.AERO_FP32)
+        if wl.aero:
+            over.update(uniform_policy=B.AERO_UNIFORM_BAYES, rejection=1, k_ratio=1)
+        self.cfg_over = over
+        self.cfg = B.cfg_default(**over)
+        t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+        self.go, self.reward, self.cs, self.key, self.y = t(st.go), t(st.reward), t(st.cs), t(st.key.view(np.int32)), t(st.y)
+        self.alpha = t(st.alpha) if st.alpha is not None else None
+        self.beta = t(st.beta) if st.beta is not None else None
+        self.noise = t(st.noise)
+        self.gbuf, self.fbuf = {}, {}
+        self.dH = torch.empty_like(self.H)
+        self.dW = torch.empty((wl.V, wl.d), dtype=torch.float32, device=dev)
+        self.chunk = min(chunk_tokens, (self.T + 127) // 128 * 128)
+        T, R = self.T, self.R
+        self.ws = torch.empty(max(ctx.bwd_workspace_bytes(T, wl.d, wl.V, R, self.chunk),
+                                  ctx.fwd_bwd_workspace_bytes(T, wl.d, wl.V, R, self.chunk)), dtype=torch.uint8, device=dev)
+        # old log-probs: the current policy's own log-probs (the log-prob pass alone) plus seeded noise
+        f0 = ctx.logprob_fwd(self.cfg, self.H, self.W, self.y)
+        self.old = (f0["logp"][:T] + self.noise).contiguous()
+        del f0
+
+    def step(self, cfg=None):
+        """Group stage, then forward and backward of stage (b) in one call (no recompute of the logits)."""
+        cfg = cfg or self.cfg
+        g = self.ctx.group_stats(cfg, self.go, self.reward, self.cs, key=self.key, alpha_in=self.alpha, beta_in=self.beta,
+                                 out=self.gbuf)
+        f, _, _ = self.ctx.grpo_loss_fwd_bwd(cfg, self.H, self.W, self.y, self.old, self.cs, g["adv"], g["w"], g["keep"],
+                                             out=self.fbuf, dH=self.dH, dW=self.dW, workspace=self.ws)
+        return g, f
+
+    def step_dp(self, P_global):
+        """The same step as one rank of a data-parallel job (counters, weights, dW and loss exchanged)."""
+        from paper_2602_14338_b200 import dist as D
+        g, f, _ = D.data_parallel_step(self.ctx, self.cfg, self.go, self.reward, self.cs, self.key, self.alpha, self.beta,
+                                       self.H, self.W, self.y, self.old, self.gbuf, self.fbuf, self.dH, self.dW, self.ws,
+                                       P_global=P_global)
+        return g, f
+
+    def step_two_calls(self):
+        """The same step through the separate forward and backward calls (the backward recomputes the logits)."""
+        c = self.ctx
+        g = c.group_stats(self.cfg, self.go, self.reward, self.cs, key=self.key, alpha_in=self.alpha, beta_in=self.beta,
+                          out=self.gbuf)
+        f = c.grpo_loss_fwd(self.cfg, self.H, self.W, self.y, self.old, self.cs, g["adv"], g["w"], g["keep"], out=self.fbuf)
+        c.grpo_loss_bwd(self.cfg, self.H, self.W, self.y, self.cs, g["keep"], f["lse"], f["g"], dH=self.dH, dW=self.dW,
+                        workspace=self.ws, logp=f["logp"])
+
+    def release(self):
+        import torch
+        for k in list(self.__dict__):
+            if k not in ("base", "wl", "st", "P", "R", "T", "chunk", "cfg_over"):
+                self.__dict__[k] = None
+        gc.collect()
+        torch.cuda.empty_cache()
+
+
+def timed(fn, n, warm=1):
+    """Mean milliseconds of fn over n calls after `warm` untimed ones (CUDA events on the current stream)."""
+    import torch
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(n):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / n
+
+
+def step_record(wl, T_kept, ms, pk, flops_per_token_factor):
+    """tokens/s and the step's FLOP rate (factor * d * V FLOP per kept token) against the three peaks."""
+    tf = flops_per_token_factor * T_kept * wl.d * wl.V / (ms * 1e-3) / 1e12
+    return {"ms": ms, "tokens_per_s": T_kept / (ms * 1e-3), "tflops": tf, "frac_of_sustained": tf / pk["sustained"],
+            "frac_of_burst": tf / pk["burst"], "frac_of_nominal_peak": tf / NOMINAL_BF16_TFLOPS}
+
+
 def run_ours(args):
     import torch
     from paper_2602_14338_b200 import binding as B
     from paper_2602_14338_b200 import dist as D
-    from paper_2602_14338_b200 import synth
 
     rank, world, local = D.init_from_env()
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device (the library has no CPU path)")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     pk = peaks()
+    ctx = B.Context(local)
     if args.only_group_leg:
-        ctx = B.Context(local)
         print(json.dumps({"group_stage": group_stage_leg(ctx, pk, dev)}), flush=True)
         return
 
-    base = synth.WORKLOADS[args.config]
-    wl = synth.scaled(base, seed=base.seed + 100 * rank)      # an independent batch per replica
-    if args.prompts > 0:
-        wl = synth.scaled(wl, P=args.prompts)
-    st = synth.make_structure(wl)
-    P, R, T = len(st.go) - 1, len(st.reward), int(st.cs[-1])
-    H, W = synth.make_tensors(wl, T, device=dev)
-    ctx = B.Context(local)
-    over = dict(seed=wl.seed, dtype=B.AERO_BF16 if wl.dtype == "bf16" else B.AERO_FP32)
-    if wl.aero:
-        over.update(uniform_policy=B.AERO_UNIFORM_BAYES, rejection=1, k_ratio=1)
-    cfg = B.cfg_default(**over)
-
-    t = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
-    go, reward, cs, key, y = t(st.go), t(st.reward), t(st.cs), t(st.key.view(np.int32)), t(st.y)
-    alpha = t(st.alpha) if st.alpha is not None else None
-    beta = t(st.beta) if st.beta is not None else None
-    noise = t(st.noise)
-
-    gbuf, fbuf = {}, {}
-    dH = torch.empty_like(H)
-    dW = torch.empty((wl.V, wl.d), dtype=torch.float32, device=dev)
-    chunk = min(args.chunk_tokens, (T + 127) // 128 * 128)
-    ws_b = torch.empty(max(ctx.bwd_workspace_bytes(T, wl.d, wl.V, R, chunk), ctx.fwd_bwd_workspace_bytes(T, wl.d, wl.V, R, chunk)),
-                       dtype=torch.uint8, device=dev)
-
-    # old log-probs: the current policy's own log-probs (the log-prob pass alone) plus seeded noise
-    f0 = ctx.logprob_fwd(cfg, H, W, y)
-    old = (f0["logp"][:T] + noise).contiguous()
-    del f0
-
-    def step():
-        # group stage, then forward and backward of stage (b) in one call (no recompute of the logits)
-        g = ctx.group_stats(cfg, go, reward, cs, key=key, alpha_in=alpha, beta_in=beta, out=gbuf)
-        f, _, _ = ctx.grpo_loss_fwd_bwd(cfg, H, W, y, old, cs, g["adv"], g["w"], g["keep"], out=fbuf, dH=dH, dW=dW,
-                                        workspace=ws_b)
-        return g, f
-
-    def step_two_calls():
-        # the same step through the separate forward and backward calls (the backward recomputes the logits)
-        g = ctx.group_stats(cfg, go, reward, cs, key=key, alpha_in=alpha, beta_in=beta, out=gbuf)
-        f = ctx.grpo_loss_fwd(cfg, H, W, y, old, cs, g["adv"], g["w"], g["keep"], out=fbuf)
-        ctx.grpo_loss_bwd(cfg, H, W, y, cs, g["keep"], f["lse"], f["g"], dH=dH, dW=dW, workspace=ws_b)
-
-    for _ in range(max(args.warmup, 1)):
+    t_start = time.perf_counter()
+    main = Prepared(ctx, dev, args.config, rank, args.chunk_tokens, args.prompts)
+    wl = main.wl
+    P_global = D.total_over_ranks(main.P)
+    step = (lambda: main.step_dp(P_global)) if world > 1 else main.step
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
         g, f = step()
     torch.cuda.synchronize()
     T_kept = int(g["counters"][1].item())
@@ -276,152 +338,173 @@ def run_ours(args):
     units, ms_total = D.aggregate(T_kept * args.steps, ms_local, device=dev)
     ms_step = ms_total / args.steps
     value = units / (ms_total * 1e-3)
+    long_step = ms_step > 1000.0
 
     # dominant kernel of the timed step: lmhead_kernel<MODE_FWD_P> (one launch per chunk), timed with CUDA events
-    # that the library records around its launches, over three more steps
+    # that the library records around its launches on the context's stream, over further steps
+    n_kt = 1 if long_step else 3
     ctx.enable_kernel_timing(True)
     fp_total_ms, fp_launches = 0.0, 0
-    for _ in range(3):
-        step()
+    for _ in range(n_kt):
+        main.step()
         ms_i, n_i = ctx.kernel_timing_ms()          # read out per step: the library keeps at most 256 pairs of events
         fp_total_ms += ms_i
         fp_launches += n_i
     ctx.enable_kernel_timing(False)
-    fwdp_ms_step = fp_total_ms / 3.0
-    # the plain forward kernel (MODE_FWD, used by the separate forward call and the log-prob pass), timed over its call
-    fw = []
-    for _ in range(max(3, min(args.steps, 10))):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        ctx.grpo_loss_fwd(cfg, H, W, y, old, cs, gbuf["adv"], gbuf["w"], gbuf["keep"], out=fbuf)
-        b.record()
-        torch.cuda.synchronize()
-        fw.append(a.elapsed_time(b))
-    fwd_ms = float(np.mean(fw))
+    fwdp_ms_step = fp_total_ms / n_kt
     clocks = sampler.stop()
+    # the plain forward kernel (MODE_FWD, used by the separate forward call and the log-prob pass), timed over its call
+    fwd_ms = timed(lambda: ctx.grpo_loss_fwd(main.cfg, main.H, main.W, main.y, main.old, main.cs, main.gbuf["adv"],
+                                             main.gbuf["w"], main.gbuf["keep"], out=main.fbuf), 2 if long_step else 5)
     flops_launch = 2.0 * T_kept * wl.d * wl.V
-    cap = NCU_FWD_TRAFFIC.get(args.config) if args.prompts == 0 else None
-    traffic = cap["bytes"] * T_kept / cap["tokens"] if cap else None
     achieved = flops_launch / (fwdp_ms_step * 1e-3) / 1e12
-    capp = NCU_FWDP_TRAFFIC.get(args.config) if args.prompts == 0 else None
+    ldz = (wl.V + 63) // 64 * 64
+    one_call = step_record(wl, T_kept, ms_local / args.steps, pk, 6.0)
     # the kernel is timed inside whole steps, under the power cap they run into: the sustained GEMM rate is its peak
     roofline = {"bound": "tensor", "kernel": "lmhead_kernel<MODE_FWD_P>", "achieved": achieved, "peak": pk["sustained"],
                 "unit": "TFLOP/s", "frac": achieved / pk["sustained"],
                 "peak_source": pk["src"] + " sustained bf16 (kernel timed inside the step)",
                 "frac_of_burst": achieved / pk["burst"], "peak_burst": pk["burst"],
-                "traffic": capp["bytes"] * T_kept / capp["tokens"] if capp else None,
-                "traffic_source": NCU_FWD_TRAFFIC_SOURCE.replace("launch", "launches of one step") if capp else None,
-                "launches_per_step": fp_launches / 3.0, "ms_per_step_all_launches": fwdp_ms_step,
+                "frac_of_nominal_peak": achieved / NOMINAL_BF16_TFLOPS,
+                "traffic": None,
+                "traffic_note": "no DRAM counters for this kernel at this size: counters are taken on reduced cases only "
+                                "(profiles/); algorithmic_bytes = kept rows of H + W + the chunk blocks of exp(z - c_t) "
+                                "written, each once per step",
+                "algorithmic_bytes": float(T_kept * wl.d * 2 + wl.V * wl.d * 2 + T_kept * ldz * 2),
+                "launches_per_step": fp_launches / n_kt, "ms_per_step_all_launches": fwdp_ms_step,
+                "share_of_step": fwdp_ms_step / (ms_local / args.steps),
                 "plain_forward_kernel": {"kernel": "lmhead_kernel<MODE_FWD>", "ms_per_launch": fwd_ms,
                                          "achieved": flops_launch / (fwd_ms * 1e-3) / 1e12,
                                          "frac": flops_launch / (fwd_ms * 1e-3) / 1e12 / pk["burst"],
                                          "peak_source": pk["src"] + " burst bf16 (kernel timed in a call of its own)",
                                          "frac_of_sustained": flops_launch / (fwd_ms * 1e-3) / 1e12 / pk["sustained"],
-                                         "traffic": traffic},
-                "step_executed_tflops": 6.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12,
-                "step_frac_of_sustained": 6.0 * T_kept * wl.d * wl.V / (ms_local / args.steps * 1e-3) / 1e12 / pk["sustained"]}
+                                         "algorithmic_bytes": float(T_kept * wl.d * 2 + wl.V * wl.d * 2)},
+                "step_executed_tflops": one_call["tflops"], "step_frac_of_sustained": one_call["frac_of_sustained"],
+                "step_frac_of_burst": one_call["frac_of_burst"], "step_frac_of_nominal_peak": one_call["frac_of_nominal_peak"],
+                "target": {"stage_b_frac_of_nominal_peak": TARGET_STAGE_B,
+                           "met": bool(one_call["frac_of_nominal_peak"] >= TARGET_STAGE_B)}}
     # the two-call step (8 d V executed FLOPs per token), for comparison
-    step_two_calls()
-    torch.cuda.synchronize()
-    a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a2.record()
-    for _ in range(2):
-        step_two_calls()
-    b2.record()
-    torch.cuda.synchronize()
-    ms2 = a2.elapsed_time(b2) / 2
-    roofline["two_call_step"] = {"ms": ms2, "tokens_per_s": T_kept / (ms2 * 1e-3),
-                                 "executed_tflops": 8.0 * T_kept * wl.d * wl.V / (ms2 * 1e-3) / 1e12,
-                                 "frac_of_sustained": 8.0 * T_kept * wl.d * wl.V / (ms2 * 1e-3) / 1e12 / pk["sustained"]}
+    ms2 = timed(main.step_two_calls, 1 if long_step else 2)
+    two_call = step_record(wl, T_kept, ms2, pk, 8.0)
+    roofline["two_call_step"] = two_call
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 1), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
-        "config": {"workload": wl.name, "P": P, "R": R, "T_input": T, "T_kept": T_kept, "d": wl.d, "V": wl.V,
-                   "parallelism": f"replicas x{world}", "chunk_tokens": int(chunk),
+        "config": {"workload": wl.name, "P": main.P, "R": main.R, "T_input": main.T, "T_kept": T_kept, "d": wl.d, "V": wl.V,
+                   "parallelism": "single GPU" if world == 1 else f"data parallel x{world}: prompts sharded, W replicated, "
+                                  "all-reduce of counters, dW and loss",
+                   "chunk_tokens": int(main.chunk), "step": "aero_group_stats + aero_grpo_loss_fwd_bwd (one-call step: the "
+                   "forward leaves one chunk of exp(z - c_t) in bf16 for the backward)",
                    "l2": "inputs larger than L2 (H+W > 1 GB per step)", "tokens_counted": "kept tokens",
-                   "input_tokens_per_s": T * world / (ms_step * 1e-3), "status_word": status},
+                   "input_tokens_per_s": main.T * world / (ms_step * 1e-3), "status_word": status},
+        "two_call_value": two_call["tokens_per_s"],
+        "two_call_note": "the same step through aero_grpo_loss_fwd + aero_grpo_loss_bwd (logits recomputed, nothing but "
+                         "dz of one chunk stored)",
         "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons")},
         "gpu_launches": int(launches),
         "roofline": roofline,
     }
+    single = rank == 0 and world == 1
+    if not args.no_e2e and not args.only_main:
+        line["e2e"] = e2e_leg(ctx, main, args, T_kept, world, dev)
+    main.release()
 
-    if rank == 0 and world == 1 and not args.no_variants_leg:
-        line["variants"] = variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, gbuf, dH, dW, ws_b, T_kept, pk)
-    if rank == 0 and world == 1 and not args.no_group_leg:
-        line["group_stage"] = group_stage_leg(ctx, pk, dev)
-    if rank == 0 and not args.no_e2e:
-        line["e2e"] = e2e_leg(ctx, cfg, wl, st, H, W, old, dH, dW, chunk, args, T_kept)
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        val, cores, sample, _ = time_oracle(base, synth.make_structure(base), 20.0)
-        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+    if single and not args.only_main:
+        subs, keep3, keep1 = {}, None, None
+        for idx in [int(x) for x in args.sub_workloads.split(",") if x.strip()]:
+            if idx == args.config or args.prompts > 0:
+                continue
+            pw = Prepared(ctx, dev, idx, rank, args.chunk_tokens)
+            n = 3 if idx <= 2 else 2
+            ms1 = timed(pw.step, n, warm=2)
+            tk = int(pw.gbuf["counters"][1].item())
+            rec = {"T_input": pw.T, "T_kept": tk, "d": pw.wl.d, "V": pw.wl.V, "steps": n,
+                   "one_call": step_record(pw.wl, tk, ms1, pk, 6.0),
+                   "two_call": step_record(pw.wl, tk, timed(pw.step_two_calls, 2 if idx <= 2 else 1), pk, 8.0)}
+            rec["value"] = rec["one_call"]["tokens_per_s"]
+            subs[pw.wl.name] = rec
+            if idx == 3 and not args.no_variants_leg:
+                line["k_ratio_sweep"] = k_sweep_leg(ctx, pw, pk)
+            if idx == 1 and not args.no_variants_leg:
+                line["variants"] = variants_leg(ctx, pw, tk, pk)
+            pw.release()
+        line["workloads"] = subs
+        if not args.no_group_leg:
+            line["group_stage"] = group_stage_leg(ctx, pk, dev)
+        if not args.no_cpu_baseline:
+            from paper_2602_14338_b200 import synth
+            val, cores, sample, _ = time_oracle(main.base, synth.make_structure(main.base), 20.0)
+            line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+    line["bench_wall_s"] = time.perf_counter() - t_start
     if rank == 0:
         print(json.dumps(line), flush=True)
     D.barrier()
 
 
-def variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, g, dH, dW, ws_b, T_kept, pk):
+def k_sweep_leg(ctx, pw, pk):
+    """Cost of the down-sampling ratio k (Sec. 5 and the appendix give +7 / +13 / +16 % training time for k = 2, 3, 4
+    on 2 x A10 with a 1.5B model): the AERO-curated batch with k = 1..4, the whole step timed per k."""
+    import torch
+    from paper_2602_14338_b200 import binding as B
+
+    out, base_ms = {}, None
+    for k in (1, 2, 3, 4):
+        kc = B.cfg_default(**{**pw.cfg_over, "k_ratio": k})
+        ms = timed(lambda: pw.step(kc), 2, warm=1)
+        ck = pw.gbuf["counters"].cpu().tolist()
+        base_ms = base_ms or ms
+        out[str(k)] = {"kept_rollouts": ck[0], "kept_tokens": ck[1], "kept_token_fraction": ck[1] / max(ck[7], 1), "ms": ms,
+                       "tokens_per_s": ck[1] / (ms * 1e-3), "time_vs_k1": ms / base_ms}
+    out["paper"] = {"time_vs_k1": {"2": 1.07, "3": 1.13, "4": 1.16},
+                    "context": "whole RL training step (rollout generation included) of a 1.5B model on 2 x A10; here only the "
+                               "policy-objective step, whose cost follows the kept tokens"}
+    return out
+
+
+def variants_leg(ctx, pw, T_kept, pk):
     """The step with Eq. 2's KL term and the entropy bonus (aero_grpo_loss_reg_fwd/_bwd), the one-call step
-    with the KL term (aero_grpo_loss_kl_fwd_bwd), and the log-prob pass alone (aero_logprob_fwd) that produces old / reference log-probs."""
+    with the KL term (aero_grpo_loss_kl_fwd_bwd), the log-prob pass alone (aero_logprob_fwd) that produces old /
+    reference log-probs, and the allocation controller on simulated prompts; on the workload passed in."""
     import copy
     import torch
-
-    T = H.shape[0]
-    rcfg = copy.copy(cfg)
-    rcfg.kl_beta, rcfg.ent_coef = 0.04, 1e-3
-    ref = (old + 0.5 * noise).contiguous()
-    fb, lb = {}, {}
-
-    def timed(fn, n=3):
-        fn()
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(n):
-            fn()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / n
-
-    def reg_step():
-        f = ctx.grpo_loss_reg_fwd(rcfg, H, W, y, old, ref, cs, g["adv"], g["w"], g["keep"], out=fb)
-        ctx.grpo_loss_reg_bwd(rcfg, H, W, y, cs, g["keep"], f["lse"], f["g"], f["entropy"], g["w"], dH=dH, dW=dW,
-                              workspace=ws_b)
-
-    ms_reg = timed(reg_step)
-    kcfg = copy.copy(cfg)
-    kcfg.kl_beta = 0.04
-    kb = {}
-    ms_kl = timed(lambda: ctx.grpo_loss_fwd_bwd(kcfg, H, W, y, old, cs, g["adv"], g["w"], g["keep"], out=kb, dH=dH, dW=dW,
-                                                workspace=ws_b, ref_logp=ref))
-    ms_lp = timed(lambda: ctx.logprob_fwd(rcfg, H, W, y, out=lb))
-    # allocation controller on 2^22 simulated prompts with success rates ~ Beta(0.5, 0.5)
     from paper_2602_14338_b200 import binding as B
     from paper_2602_14338_b200 import synth
+
+    wl, g = pw.wl, pw.gbuf
+    rcfg = copy.copy(pw.cfg)
+    rcfg.kl_beta, rcfg.ent_coef = 0.04, 1e-3
+    ref = (pw.old + 0.5 * pw.noise).contiguous()
+    fb, lb, kb, ab = {}, {}, {}, {}
+
+    def reg_step():
+        f = ctx.grpo_loss_reg_fwd(rcfg, pw.H, pw.W, pw.y, pw.old, ref, pw.cs, g["adv"], g["w"], g["keep"], out=fb)
+        ctx.grpo_loss_reg_bwd(rcfg, pw.H, pw.W, pw.y, pw.cs, g["keep"], f["lse"], f["g"], f["entropy"], g["w"], dH=pw.dH,
+                              dW=pw.dW, workspace=pw.ws, logp=f["logp"])
+
+    ms_reg = timed(reg_step, 3)
+    kcfg = copy.copy(pw.cfg)
+    kcfg.kl_beta = 0.04
+    ms_kl = timed(lambda: ctx.grpo_loss_fwd_bwd(kcfg, pw.H, pw.W, pw.y, pw.old, pw.cs, g["adv"], g["w"], g["keep"], out=kb,
+                                                dH=pw.dH, dW=pw.dW, workspace=pw.ws, ref_logp=ref), 3)
+    ms_lp = timed(lambda: ctx.logprob_fwd(rcfg, pw.H, pw.W, pw.y, out=lb), 3)
+    # allocation controller on 2^22 simulated prompts with success rates ~ Beta(0.5, 0.5)
     Pn = 1 << 22
-    thr = torch.from_numpy(synth.success_thresholds(Pn, 0.5, 0.5, seed=4301).view(np.int32)).to(H.device)
+    thr = torch.from_numpy(synth.success_thresholds(Pn, 0.5, 0.5, seed=4301).view(np.int32)).to(pw.H.device)
     acfg = B.cfg_default(uniform_policy=B.AERO_UNIFORM_BAYES, rejection=1, k_ratio=1, seed=4302)
-    ab = {}
-    ms_alloc = timed(lambda: ctx.allocate_sim(acfg, B.alloc_cfg_default(), thr, out=ab), n=5)
+    l0 = ctx.launch_count()
+    ctx.allocate_sim(acfg, B.alloc_cfg_default(), thr, out=ab)
+    alloc_launches = ctx.launch_count() - l0
+    ms_alloc = timed(lambda: ctx.allocate_sim(acfg, B.alloc_cfg_default(), thr, out=ab), 5)
     cnt = ab["counters"].cpu().tolist()
-    # down-sampling ratio k = 1..4 on the AERO-curated batch (workload 3): what the backward has to process
-    st3 = synth.make_structure(synth.WORKLOADS[3])
-    t3 = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(H.device)
-    go3, rw3, cs3, key3 = t3(st3.go), t3(st3.reward), t3(st3.cs), t3(st3.key.view(np.int32))
-    al3, be3 = t3(st3.alpha), t3(st3.beta)
-    ksweep = {}
-    for k in (1, 2, 3, 4):
-        kc = B.cfg_default(uniform_policy=B.AERO_UNIFORM_BAYES, rejection=1, k_ratio=k, seed=synth.WORKLOADS[3].seed)
-        gk = ctx.group_stats(kc, go3, rw3, cs3, key=key3, alpha_in=al3, beta_in=be3)
-        ck = gk["counters"].cpu().tolist()
-        ksweep[str(k)] = {"kept_rollouts": ck[0], "kept_tokens": ck[1], "kept_token_fraction": ck[1] / max(ck[7], 1)}
     fl = 2.0 * wl.d * wl.V
-    return {"allocation_sim": {"prompts": Pn, "ms": ms_alloc, "prompts_per_s": Pn / (ms_alloc * 1e-3),
-                               "launches": 23, "mean_rollouts_generated": cnt[0] / Pn, "mean_rollouts_trained": cnt[1] / Pn,
-                               "zero_accuracy_before": cnt[2] / Pn, "zero_accuracy_after": cnt[3] / Pn,
-                               "iterations": cnt[5]},
-            "k_ratio_sweep_workload3": ksweep,
+    T = pw.T
+    return {"workload": wl.name,
+            "allocation_sim": {"prompts": Pn, "ms": ms_alloc, "prompts_per_s": Pn / (ms_alloc * 1e-3),
+                               "launches": int(alloc_launches), "mean_rollouts_generated": cnt[0] / Pn,
+                               "mean_rollouts_trained": cnt[1] / Pn, "zero_accuracy_before": cnt[2] / Pn,
+                               "zero_accuracy_after": cnt[3] / Pn, "iterations": cnt[5]},
             "regularised_step": {"kl_beta": 0.04, "ent_coef": 1e-3, "ms": ms_reg, "tokens_per_s": T_kept / (ms_reg * 1e-3),
                                  "executed_tflops": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12,
                                  "frac_of_sustained": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12 / pk["sustained"]},
@@ -434,7 +517,7 @@ def variants_leg(ctx, cfg, wl, H, W, y, old, noise, cs, g, dH, dW, ws_b, T_kept,
 
 def group_stage_leg(ctx, pk, dev):
     """Stage (a) alone on an input large enough to be bandwidth-bound (2^22 prompts of 2..16 rollouts):
-    algorithmic bytes (37 per rollout + 26 per prompt) over the duration of the stage's four launches."""
+    algorithmic bytes (37 per rollout + 26 per prompt) over the duration of the stage's launches."""
     import torch
     from paper_2602_14338_b200 import binding as B
     from paper_2602_14338_b200 import synth
@@ -463,38 +546,73 @@ def group_stage_leg(ctx, pk, dev):
     gbs = nbytes / (ms * 1e-3) / 1e9
     return {"P": P, "R": R, "ms": ms, "bound": "hbm", "achieved": gbs, "peak": pk["hbm"], "unit": "GB/s",
             "frac": gbs / pk["hbm"], "algorithmic_bytes": nbytes,
+            "target": {"stage_a_frac_of_hbm": TARGET_STAGE_A, "met": bool(gbs / pk["hbm"] >= TARGET_STAGE_A)},
             "kept_rollout_frac": float(out["metrics"][2].item())}
 
 
-def e2e_leg(ctx, cfg, wl, st, H, W, old, dH, dW, chunk, args, T_kept):
-    """Same step through the host-buffer entry point: inputs in pinned host memory, copies inside the timed region."""
+def e2e_leg(ctx, pw, args, T_kept, world, dev):
+    """Same step through the host-buffer entry point: inputs in pinned host memory, copies inside the timed region.
+    With several ranks every rank runs it on its own batch and dW is all-reduced afterwards (the host-buffer call
+    normalises over the rank's own batch)."""
     import torch
+    from paper_2602_14338_b200 import dist as D
 
-    P, R, T = len(st.go) - 1, len(st.reward), int(st.cs[-1])
+    st, wl, cfg = pw.st, pw.wl, pw.cfg
+    P, R, T = pw.P, pw.R, pw.T
+    pw.ws = None                                   # the host-buffer call has a workspace of its own
+    gc.collect()
+    torch.cuda.empty_cache()
     pin = lambda x: x.pin_memory()
     go_h, rw_h, cs_h = pin(torch.from_numpy(st.go)), pin(torch.from_numpy(st.reward)), pin(torch.from_numpy(st.cs))
     key_h = pin(torch.from_numpy(st.key.view(np.int32)))
     al_h = pin(torch.from_numpy(st.alpha)) if st.alpha is not None else None
     be_h = pin(torch.from_numpy(st.beta)) if st.beta is not None else None
-    H_h, y_h, old_h = pin(H.cpu()), pin(torch.from_numpy(st.y)), pin(old.cpu())
-    ws = torch.empty(ctx.step_workspace_bytes(P, R, T, wl.d, wl.V, chunk, cfg.dtype), dtype=torch.uint8, device=H.device)
+    H_h = torch.empty(pw.H.shape, dtype=pw.H.dtype, pin_memory=True)
+    H_h.copy_(pw.H)
+    y_h, old_h = pin(torch.from_numpy(st.y)), pin(pw.old.cpu())
+    ws = torch.empty(ctx.step_workspace_bytes(P, R, T, wl.d, wl.V, pw.chunk, cfg.dtype), dtype=torch.uint8, device=dev)
     h2d = H_h.numel() * H_h.element_size() + 8 * T + 4 * (P + 1) + 16 * R + 8 + (8 * P if al_h is not None else 0)
     d2h = 4 + 64 + 32
-    n = max(2, min(args.steps, 5))
-    ctx.grpo_step_host(cfg, go_h, rw_h, cs_h, key_h, al_h, be_h, H_h, y_h, old_h, W, dH, dW, ws)
+    n = 2 if T > 2_000_000 else max(2, min(args.steps, 5))
+
+    def host_step():
+        out = ctx.grpo_step_host(cfg, go_h, rw_h, cs_h, key_h, al_h, be_h, H_h, y_h, old_h, pw.W, pw.dH, pw.dW, ws)
+        if world > 1:
+            D.reduce_sum_(pw.dW)
+            torch.cuda.synchronize()
+        return out
+
+    host_step()
     torch.cuda.synchronize()
+    D.barrier()
     t0 = time.perf_counter()
     for _ in range(n):
-        loss, counters, _ = ctx.grpo_step_host(cfg, go_h, rw_h, cs_h, key_h, al_h, be_h, H_h, y_h, old_h, W, dH, dW, ws)
+        loss, counters, _ = host_step()
     dt = (time.perf_counter() - t0) / n
     assert int(counters[1]) == T_kept
-    return {"value": T_kept / dt, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-            "ms_per_step": dt * 1e3, "loss": float(loss.item())}
+    units, ms_total = D.aggregate(T_kept, dt * 1e3, device=dev)
+    del ws, H_h
+    return {"value": units / (ms_total * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "ms_per_step": ms_total, "steps": n, "loss": float(loss.item()),
+            "api": "aero_grpo_step_host (pinned host inputs; H copied in slices under the first chunks' kernels)"}
+
+
+def spawn_ranks(args):
+    """`--gpus N` without a launcher: start N ranks of this script under torch.distributed.run."""
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
 
 
 if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(a)
     else:
         run_ours(a)

@@ -36,6 +36,11 @@
  *     dW are descent directions.
  *   - There is no CPU fallback: without a CUDA device every compute call fails with
  *     AERO_ERR_CUDA.
+ *   - Every call that takes a context makes the context's device the calling thread's
+ *     current CUDA device (cudaSetDevice) and leaves it so.
+ *   - Argument checks come first and need no device: a call with a bad argument returns
+ *     its error code whether or not the device is usable.
+ *   - Each compute call is wrapped in an NVTX range named after the entry point.
  */
 #ifndef AERO_H_
 #define AERO_H_
@@ -61,9 +66,10 @@ extern "C" {
 #define AERO_ST_BAD_REWARD     4u   /* reward not exactly 0 or 1                       */
 #define AERO_ST_EMPTY_ROLLOUT  8u   /* cs[i+1] == cs[i] for a present rollout          */
 #define AERO_ST_TIMEOUT       16u   /* a bounded wait inside a kernel ran out          */
-#define AERO_ST_RANGE         32u   /* aero_grpo_loss_fwd_bwd: a logit lies more than 125 octaves above  */
-                                    /* the shift taken from the row's first logits; that row's gradient   */
-                                    /* is saturated (use aero_grpo_loss_fwd + aero_grpo_loss_bwd instead) */
+#define AERO_ST_RANGE         32u   /* aero_grpo_loss_fwd_bwd: more than 1024 rows of one chunk have a   */
+                                    /* logit over 125 octaves above the shift taken from the row's first  */
+                                    /* logits; the rows beyond the 1024 the call redoes have a saturated   */
+                                    /* gradient (use aero_grpo_loss_fwd + aero_grpo_loss_bwd instead)      */
 
 /* ---- enumerations ------------------------------------------------------------- */
 #define AERO_UNIFORM_MASK   0   /* all-correct / all-incorrect groups are dropped (Sec. 3.2)      */
@@ -136,9 +142,21 @@ int aero_create(aero_ctx** out, int device, void* cuda_stream);
 int aero_destroy(aero_ctx* ctx);
 int aero_set_stream(aero_ctx* ctx, void* cuda_stream);
 
-/* Synchronise the stream, return the OR of all status bits raised since the last
- * call in *bits (host pointer) and clear them. */
+/* Return the OR of all status bits raised since the last call in *bits (host pointer)
+ * and clear them.  The read and the clear are enqueued on the context's stream, which is
+ * then synchronised, so they are ordered against the context's kernels on any stream. */
 int aero_last_status(aero_ctx* ctx, uint32_t* bits);
+
+/* Tuning hook (no passage of the paper: it only selects between equivalent schedules of
+ * stage (b); results agree within rounding).  vsplit: CTA pairs that share a pair of token
+ * tiles and split the vocabulary between them, 1, 2 or 4, or 0 to let the library choose
+ * by d (the default).  nsync: meeting points per unit at which the lm_head kernel's
+ * producers wait for one another, 0 for none, negative for the default.  rowscale: in
+ * aero_grpo_loss_fwd_bwd, 1 (or negative, the default) applies the row factors inside the
+ * backward products, 0 rewrites the chunk block in a pass of its own.  The workspace sizes
+ * the *_workspace_bytes functions return cover every setting.  Returns AERO_ERR_INVALID
+ * for any other value. */
+int aero_set_tuning(aero_ctx* ctx, int vsplit, int nsync, int rowscale);
 
 /* ------------------------------------------------------------------------------
  * Stage (a).  Group statistics, curation and weights (Eq. 1; Sec. 3.2; Sec. 4.2
@@ -192,6 +210,18 @@ int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
                      int32_t* kept_ids, int64_t* kept_tok_off, int64_t* counters,
                      float* metrics, void* workspace, size_t workspace_bytes);
 
+/* Weights of a data-parallel shard (Eq. 2's normalisers 1/G and 1/|o_i|, and the token-level
+ * mean of Appendix C, run over the whole batch; the paper trains with 2-4 data-parallel ranks,
+ * Appendix C).  A rank that ran aero_group_stats on its own prompts only holds weights over its
+ * local denominator.  Given its own counters and the element-wise sum of all ranks' counters
+ * (both [8] i64 on the device, e.g. after an all-reduce), this call rescales w [R] in place by
+ * local / global denominator: T_kept (TOKEN_MEAN) or P_surv (SEQ_MEAN), resp. T_present or
+ * P_local / P_global under DENOM_ALL.  Advantages and the keep-mask are per prompt and need
+ * nothing.  The loss and dW of the ranks then add up to those of the unsharded batch.  Nothing is
+ * read back to the host. */
+int aero_finalize_weights(aero_ctx* ctx, const aero_cfg* cfg, int32_t R, int32_t P_local, int64_t P_global,
+                          float* w, const int64_t* counters_local, const int64_t* counters_global);
+
 /* aero_group_stats for callers that cannot allocate device memory.  (The paper has no
  * counterpart to this call: it computes exactly what aero_group_stats computes; only the
  * origin of the scratch memory differs.)
@@ -200,8 +230,8 @@ int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
  * workspace at the point of the call -- a plug-in inside a host program that owns all
  * device memory, or a latency-bound loop that must not call the allocator because an
  * allocation can synchronise the whole device.  Instead of a caller workspace, the scratch
- * is a fixed array in device memory that belongs to the loaded library itself: about
- * 1.6 MB per GPU that loads the library, held until the process exits, sized for at most
+ * is a fixed array in device memory that belongs to the loaded library itself: 1,476,096
+ * bytes (1.41 MiB) per GPU that loads the library, held until the process exits, sized for at most
  * AERO_STATIC_MAX_PROMPTS prompts whatever their group sizes (R itself is not limited).
  * A batch beyond that limit returns AERO_ERR_TOO_LARGE and launches nothing.  The call,
  * and everything it calls, performs no cudaMalloc/cudaFree and uses no allocating library
@@ -266,8 +296,13 @@ int aero_grpo_loss_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d,
  * dz is rounded to bf16 before the two products (fp32 accumulation).  Token rows
  * are processed in chunks whose dz block lives in `workspace`; a larger workspace
  * means fewer passes over dW.  Rows of dropped rollouts get dH = 0.
+ * The target column is formed as -grad_scale g_t expm1(logp_t): for a confident token
+ * (p close to 1, where Eq. 3's factor 1 - p is tiny) this keeps the relative accuracy of
+ * the log-prob, which 1 - exp(z - lse_t) loses to the rounding of lse_t.  logp is the
+ * forward's output; NULL falls back to z_{t,y_t} - lse_t recomputed in fp32 (relative error
+ * of that entry about 4e-6 / (1 - p)).
  *
- * Inputs   as the forward, plus lse and g from it.
+ * Inputs   as the forward, plus lse, g and (optionally) logp from it.
  * Outputs  dH [T,d] (cfg->dtype); dW [V,d] f32, overwritten or, when
  *          accumulate_dW != 0, added to.
  * workspace: at least aero_bwd_workspace_bytes(T, d, V, R, chunk_tokens); chunk_tokens
@@ -280,7 +315,7 @@ size_t aero_bwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R, int6
 int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                        const void* H, const void* W, const int32_t* y,
                        const int64_t* cs, const uint8_t* keep,
-                       const float* lse, const float* g, float grad_scale,
+                       const float* lse, const float* g, const float* logp, float grad_scale,
                        void* dH, float* dW, int accumulate_dW,
                        void* workspace, size_t workspace_bytes);
 
@@ -291,11 +326,16 @@ int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d,
  * The two separate calls must recompute the logits in the backward (8 d V FLOP per token).
  * Called together, the forward of each chunk of token rows also leaves
  * p~_tv = exp(z_tv - c_t) in bf16 in the chunk's scratch block, c_t being a per-row shift taken
- * from the row's first logits; when lse_t and g_t are known the block is rescaled in place to
- * dz_tv = grad_scale (g_t 1[v == y_t] - g_t exp(c_t - lse_t) p~_tv), and dH, dW follow as in
+ * from the row's first logits; when lse_t and g_t are known the block stands for
+ * dz_tv = grad_scale (g_t 1[v == y_t] - g_t exp(c_t - lse_t) p~_tv) (the row factor is applied inside
+ * the backward products, or by a pass that rewrites the block), and dH, dW follow as in
  * aero_grpo_loss_bwd: 6 d V FLOP per token.  bf16 shares fp32's exponent range, so p~ carries the
- * same 2^-9 relative rounding dz has in the two-call path.  Neither the logits nor anything of
- * size [T,V] is stored: the scratch block is one chunk of rows, as in the backward.
+ * same 2^-9 relative rounding dz has in the two-call path; the target column is written from the
+ * fp32 log-prob as -grad_scale g_t expm1(logp_t), never by subtracting from the rounded p~.  A row
+ * with a logit too far above its shift for bf16 to hold (about 87 above the largest of the row's
+ * first 32 logits) is redone from H and W by a kernel of its own, up to 1024 such rows per chunk
+ * (beyond: AERO_ST_RANGE).  Neither the logits nor anything of size [T,V] is stored: the scratch
+ * block is one chunk of rows of unnormalised probabilities, where the backward's holds dz.
  *
  * workspace: at least aero_fwd_bwd_workspace_bytes(T, d, V, R, chunk_tokens), 256-byte aligned.
  * fp32 inputs run the two plain calls one after the other.
@@ -337,8 +377,8 @@ int aero_grpo_loss_kl_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int
  * aero_grpo_loss_reg_fwd: arguments of aero_grpo_loss_fwd plus ref_logp [T] f32 (NULL:
  *   no KL term, kl_beta ignored) and entropy [T] f32 out (NULL: no entropy term,
  *   ent_coef ignored).  With both NULL it is aero_grpo_loss_fwd.
- * aero_grpo_loss_reg_bwd: arguments of aero_grpo_loss_bwd plus entropy [T] from the
- *   forward and w [R] (both NULL: no entropy term).
+ * aero_grpo_loss_reg_bwd: arguments of aero_grpo_loss_bwd (logp included, may be NULL) plus
+ *   entropy [T] from the forward and w [R] (both NULL: no entropy term).
  * aero_logprob_fwd: the log-prob pass alone over all T rows (what produces old_logp and
  *   ref_logp, Appendix C "Rollout"/"GRPO Training"): logp, lse [T] f32 and, if not NULL,
  *   entropy [T] f32.  Workspace: aero_fwd_workspace_bytes(T, d, V, 0).
@@ -353,7 +393,8 @@ int aero_grpo_loss_reg_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_
 int aero_grpo_loss_reg_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                            const void* H, const void* W, const int32_t* y,
                            const int64_t* cs, const uint8_t* keep,
-                           const float* lse, const float* g, const float* entropy, const float* w,
+                           const float* lse, const float* g, const float* logp,
+                           const float* entropy, const float* w,
                            float grad_scale, void* dH, float* dW, int accumulate_dW,
                            void* workspace, size_t workspace_bytes);
 
@@ -437,6 +478,13 @@ int aero_allocate_sim(aero_ctx* ctx, const aero_cfg* cfg, const aero_alloc_cfg* 
  * pointers) and starts over.  Off by default; meant for benchmarks. */
 int aero_enable_kernel_timing(aero_ctx* ctx, int on);
 int aero_kernel_timing_ms(aero_ctx* ctx, float* total_ms, int* launches);
+
+/* Self-test of the bounded waits (no passage of the paper).  Every wait inside the tensor-core
+ * kernels gives up after a time limit, raises AERO_ST_TIMEOUT and lets the kernel end normally.
+ * This call launches a one-warp kernel of its own that waits, for at most limit_us microseconds
+ * (1 .. 1000000), on a barrier nobody arrives at: afterwards aero_last_status must report
+ * AERO_ST_TIMEOUT and the context must be usable as before.  Nothing else is touched. */
+int aero_selftest_bounded_wait(aero_ctx* ctx, uint32_t limit_us);
 
 /* Number of kernels the library has launched through this context since it was created
  * (copies and memsets are not counted).  Host-side counter, no synchronisation. */

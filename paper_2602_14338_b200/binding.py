@@ -31,6 +31,7 @@ EXPORTS = [
     "aero_grpo_loss_reg_fwd", "aero_grpo_loss_reg_bwd", "aero_logprob_fwd",
     "aero_alloc_cfg_default", "aero_allocate_workspace_bytes", "aero_allocate_sim",
     "aero_fwd_bwd_workspace_bytes", "aero_grpo_loss_fwd_bwd", "aero_grpo_loss_kl_fwd_bwd", "aero_enable_kernel_timing", "aero_kernel_timing_ms",
+    "aero_set_tuning", "aero_finalize_weights", "aero_selftest_bounded_wait",
 ]
 
 
@@ -74,21 +75,24 @@ def load_library():
     lib.aero_create.argtypes = [C.POINTER(vp), C.c_int, vp]
     lib.aero_destroy.argtypes = [vp]
     lib.aero_set_stream.argtypes = [vp, vp]
+    lib.aero_set_tuning.argtypes = [vp, C.c_int, C.c_int, C.c_int]
+    lib.aero_selftest_bounded_wait.argtypes = [vp, C.c_uint32]
     lib.aero_last_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.aero_group_workspace_bytes.restype = sz
     lib.aero_group_workspace_bytes.argtypes = [i32, i32]
     lib.aero_group_stats.argtypes = [vp, C.POINTER(AeroCfg), i32, i32] + [vp] * 19 + [vp, sz]
     lib.aero_group_stats_static.argtypes = [vp, C.POINTER(AeroCfg), i32, i32] + [vp] * 19
+    lib.aero_finalize_weights.argtypes = [vp, C.POINTER(AeroCfg), i32, i32, i64, vp, vp, vp]
     lib.aero_fwd_workspace_bytes.restype = sz
     lib.aero_fwd_workspace_bytes.argtypes = [i64, i32, i32, i32]
     lib.aero_grpo_loss_fwd.argtypes = [vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 13 + [C.c_int, vp, sz]
     lib.aero_bwd_workspace_bytes.restype = sz
     lib.aero_bwd_workspace_bytes.argtypes = [i64, i32, i32, i32, i64]
-    lib.aero_grpo_loss_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 7 + [f32] +
+    lib.aero_grpo_loss_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 8 + [f32] +
                                        [vp, vp, C.c_int, vp, sz])
     lib.aero_grpo_loss_reg_fwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 15 +
                                            [C.c_int, vp, sz])
-    lib.aero_grpo_loss_reg_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 9 + [f32] +
+    lib.aero_grpo_loss_reg_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 10 + [f32] +
                                            [vp, vp, C.c_int, vp, sz])
     lib.aero_logprob_fwd.argtypes = [vp, C.POINTER(AeroCfg), i64, i32, i32] + [vp] * 6 + [vp, sz]
     lib.aero_alloc_cfg_default.restype = None
@@ -191,6 +195,14 @@ class Context:
         self.stream = stream
         _check(self.lib.aero_set_stream(self.h, C.c_void_p(stream.cuda_stream)), "aero_set_stream")
 
+    def set_tuning(self, vsplit=0, nsync=-1, rowscale=-1):
+        """aero_set_tuning: schedule choices of stage (b); the defaults let the library decide."""
+        _check(self.lib.aero_set_tuning(self.h, int(vsplit), int(nsync), int(rowscale)), "aero_set_tuning")
+
+    def selftest_bounded_wait(self, limit_us=1000):
+        """aero_selftest_bounded_wait: a wait that cannot complete must end with AERO_ST_TIMEOUT."""
+        _check(self.lib.aero_selftest_bounded_wait(self.h, int(limit_us)), "aero_selftest_bounded_wait")
+
     def last_status(self) -> int:
         bits = C.c_uint32(0)
         _check(self.lib.aero_last_status(self.h, C.byref(bits)), "aero_last_status")
@@ -231,6 +243,15 @@ class Context:
             _ptr(u), _ptr(ao), _ptr(bo), _ptr(kid), _ptr(kto), _ptr(cnt), _ptr(met), ws.data_ptr(), ws.numel())
         _check(rc, "aero_group_stats")
         return o
+
+    def finalize_weights(self, cfg, w, counters_local, counters_global, P_local, P_global):
+        """aero_finalize_weights: rescale a shard's weights from its local to the batch-wide denominator."""
+        R = w.numel()
+        rc = self.lib.aero_finalize_weights(self.h, C.byref(cfg), R, P_local, P_global, _ptr(w, torch.float32, R, "w"),
+                                            _ptr(counters_local, torch.int64, 8, "counters_local"),
+                                            _ptr(counters_global, torch.int64, 8, "counters_global"))
+        _check(rc, "aero_finalize_weights")
+        return w
 
     GROUP_OUTPUTS = (("adv", "R", torch.float32), ("w", "R", torch.float32), ("keep", "R", torch.uint8),
                      ("gmask", "P", torch.uint8), ("cat", "P", torch.uint8), ("u_tilde", "P", torch.float32),
@@ -336,7 +357,7 @@ class Context:
         return o
 
     def grpo_loss_reg_bwd(self, cfg, H, W, y, cs, keep, lse, g, entropy, w, grad_scale=1.0, dH=None, dW=None,
-                          accumulate_dW=False, chunk_tokens=None, workspace=None):
+                          accumulate_dW=False, chunk_tokens=None, workspace=None, logp=None):
         """aero_grpo_loss_reg_bwd: the backward with the entropy term (entropy and w from the forward / group stage)."""
         T, d = H.shape
         V = W.shape[0]
@@ -353,7 +374,7 @@ class Context:
         rc = self.lib.aero_grpo_loss_reg_bwd(
             self.h, C.byref(cfg), T, d, V, R, _ptr(H, dt, T * d, "H"), _ptr(W, dt, V * d, "W"),
             _ptr(y, torch.int32, T, "y"), _ptr(cs, torch.int64, R + 1, "cs"), _ptr(keep, torch.uint8, R, "keep"),
-            _ptr(lse, torch.float32, T, "lse"), _ptr(g, torch.float32, T, "g"),
+            _ptr(lse, torch.float32, T, "lse"), _ptr(g, torch.float32, T, "g"), _ptr(logp, torch.float32, T, "logp"),
             _ptr(entropy, torch.float32, T, "entropy"), _ptr(w, torch.float32, R, "w"), C.c_float(grad_scale),
             _ptr(dH, dt, T * d, "dH"), _ptr(dW, torch.float32, V * d, "dW"), 1 if accumulate_dW else 0,
             workspace.data_ptr(), workspace.numel())
@@ -401,7 +422,7 @@ class Context:
         return o, dH, dW
 
     def grpo_loss_bwd(self, cfg, H, W, y, cs, keep, lse, g, grad_scale=1.0, dH=None, dW=None,
-                      accumulate_dW=False, chunk_tokens=None, workspace=None):
+                      accumulate_dW=False, chunk_tokens=None, workspace=None, logp=None):
         T, d = H.shape
         V = W.shape[0]
         R = cs.numel() - 1
@@ -417,7 +438,8 @@ class Context:
         rc = self.lib.aero_grpo_loss_bwd(
             self.h, C.byref(cfg), T, d, V, R, _ptr(H, dt, T * d, "H"), _ptr(W, dt, V * d, "W"),
             _ptr(y, torch.int32, T, "y"), _ptr(cs, torch.int64, R + 1, "cs"), _ptr(keep, torch.uint8, R, "keep"),
-            _ptr(lse, torch.float32, T, "lse"), _ptr(g, torch.float32, T, "g"), C.c_float(grad_scale),
+            _ptr(lse, torch.float32, T, "lse"), _ptr(g, torch.float32, T, "g"), _ptr(logp, torch.float32, T, "logp"),
+            C.c_float(grad_scale),
             _ptr(dH, dt, T * d, "dH"), _ptr(dW, torch.float32, V * d, "dW"), 1 if accumulate_dW else 0,
             workspace.data_ptr(), workspace.numel())
         _check(rc, "aero_grpo_loss_bwd")

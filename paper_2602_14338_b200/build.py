@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libaero_b200.so")
-SOURCES = ["api.cu", "group_stage.cu", "loss_common.cu", "loss_fp32.cu", "loss_fwd_tc.cu", "loss_bwd_tc.cu", "step_host.cu", "alloc_sim.cu", "step_fused_tc.cu"]
+SOURCES = ["api.cu", "group_stage.cu", "loss_common.cu", "loss_fp32.cu", "loss_fwd_tc.cu", "loss_bwd_tc.cu", "step_host.cu", "alloc_sim.cu", "step_fused_tc.cu", "selftest.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC"]
 

@@ -4,7 +4,15 @@
 
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 namespace {
+
+// NVTX range over one ABI call (visible in Nsight timelines; a no-op without a profiler attached)
+struct Range {
+  explicit Range(const char* name) { nvtxRangePushA(name); }
+  ~Range() { nvtxRangePop(); }
+};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
@@ -19,7 +27,7 @@ int check_ctx(aero_ctx* ctx) {
 
 extern "C" {
 
-int aero_version(void) { return 100; }
+int aero_version(void) { return 101; }
 
 const char* aero_error_string(int code) {
   switch (code) {
@@ -71,6 +79,9 @@ int aero_create(aero_ctx** out, int device, void* cuda_stream) {
   ctx->launches = 0;
   ctx->timing = 0;
   ctx->n_timed = 0;
+  ctx->tune_vsplit = 0;
+  ctx->tune_nsync = -1;
+  ctx->tune_rowscale = -1;
   for (int i = 0; i < 256; ++i) { ctx->ev0[i] = nullptr; ctx->ev1[i] = nullptr; }
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return AERO_ERR_CUDA; }
@@ -128,13 +139,25 @@ int aero_set_stream(aero_ctx* ctx, void* cuda_stream) {
   return AERO_OK;
 }
 
+int aero_set_tuning(aero_ctx* ctx, int vsplit, int nsync, int rowscale) {
+  if (!ctx) return AERO_ERR_INVALID;
+  if (vsplit != 0 && vsplit != 1 && vsplit != 2 && vsplit != 4) return AERO_ERR_INVALID;
+  if (nsync > 4096) return AERO_ERR_INVALID;
+  ctx->tune_vsplit = vsplit;
+  ctx->tune_nsync = nsync < 0 ? -1 : nsync;
+  ctx->tune_rowscale = rowscale < 0 ? -1 : (rowscale ? 1 : 0);
+  return AERO_OK;
+}
+
 int aero_last_status(aero_ctx* ctx, uint32_t* bits) {
   if (!ctx || !bits) return AERO_ERR_INVALID;
   int rc = check_ctx(ctx);
   if (rc) return rc;
+  // read and clear in stream order, so that neither can overtake (or be overtaken by) kernels of
+  // this context on a stream that does not synchronise with the default stream
+  AERO_CUDA_TRY(cudaMemcpyAsync(bits, ctx->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost, ctx->stream));
+  AERO_CUDA_TRY(cudaMemsetAsync(ctx->d_status, 0, sizeof(uint32_t), ctx->stream));
   AERO_CUDA_TRY(cudaStreamSynchronize(ctx->stream));
-  AERO_CUDA_TRY(cudaMemcpy(bits, ctx->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost));
-  AERO_CUDA_TRY(cudaMemset(ctx->d_status, 0, sizeof(uint32_t)));
   return AERO_OK;
 }
 
@@ -148,9 +171,8 @@ int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
                      float* u_tilde, float* alpha_out, float* beta_out,
                      int32_t* kept_ids, int64_t* kept_tok_off, int64_t* counters,
                      float* metrics, void* workspace, size_t workspace_bytes) {
-  int rc = check_ctx(ctx);
-  if (rc) return rc;
-  if (!cfg || P < 0 || R < 0) return AERO_ERR_INVALID;
+  Range nv("aero_group_stats");
+  if (!ctx || !cfg || P < 0 || R < 0) return AERO_ERR_INVALID;
   if (!go || !cs || !kept_tok_off || !counters) return AERO_ERR_INVALID;
   if (R > 0 && (!reward || !adv || !w || !keep || !kept_ids)) return AERO_ERR_INVALID;
   if (P > 0 && (!gmask || !cat || !u_tilde || !alpha_out || !beta_out)) return AERO_ERR_INVALID;
@@ -158,9 +180,21 @@ int aero_group_stats(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
   if (cfg->k_ratio < 1 || cfg->n_explore < 1 || cfg->rescue_S < 0) return AERO_ERR_INVALID;
   if (!workspace || !aligned256(workspace)) return AERO_ERR_INVALID;
   if (workspace_bytes < aero_group_ws_bytes_impl(P, R)) return AERO_ERR_WORKSPACE;
+  const int rc = check_ctx(ctx);
+  if (rc) return rc;
   return aero_group_stats_launch(ctx, cfg, P, R, go, reward, cs, key, keep_in, alpha_in, beta_in,
                                  adv, w, keep, gmask, cat, u_tilde, alpha_out, beta_out,
                                  kept_ids, kept_tok_off, counters, metrics, workspace);
+}
+
+int aero_finalize_weights(aero_ctx* ctx, const aero_cfg* cfg, int32_t R, int32_t P_local, int64_t P_global,
+                          float* w, const int64_t* counters_local, const int64_t* counters_global) {
+  Range nv("aero_finalize_weights");
+  if (!ctx || !cfg || R < 0 || P_local < 0 || P_global < P_local) return AERO_ERR_INVALID;
+  if (!counters_local || !counters_global || (R > 0 && !w)) return AERO_ERR_INVALID;
+  const int rc = check_ctx(ctx);
+  if (rc) return rc;
+  return aero_finalize_weights_launch(ctx, cfg, R, P_local, P_global, w, counters_local, counters_global);
 }
 
 size_t aero_fwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R) {
@@ -174,9 +208,7 @@ static int fwd_dispatch(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d
                         const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
                         float* logp, float* lse, float* g, float* loss, float* metrics,
                         int accumulate, void* workspace, size_t workspace_bytes, const aero_fwd_extra& ex) {
-  int rc = check_ctx(ctx);
-  if (rc) return rc;
-  if (!cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
+  if (!ctx || !cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
   if (!W) return AERO_ERR_INVALID;
   if (T > 0 && (!H || !y || !logp || !lse)) return AERO_ERR_INVALID;
   if (!ex.logprob_only) {
@@ -185,14 +217,16 @@ static int fwd_dispatch(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d
     if (R > 0 && (!adv || !w || !keep)) return AERO_ERR_INVALID;
   }
   if (!workspace || !aligned256(workspace)) return AERO_ERR_INVALID;
+  if (cfg->dtype != AERO_FP32 && cfg->dtype != AERO_BF16) return AERO_ERR_UNSUPPORTED;
+  if (cfg->dtype == AERO_BF16 && d % 64 != 0) return AERO_ERR_UNSUPPORTED;
+  if (cfg->dtype == AERO_BF16 && (!aligned16(H) || !aligned16(W))) return AERO_ERR_INVALID;
   if (workspace_bytes < aero_fwd_workspace_bytes(T, d, V, R)) return AERO_ERR_WORKSPACE;
+  const int rc = check_ctx(ctx);
+  if (rc) return rc;
   if (cfg->dtype == AERO_FP32) {
     return aero_fwd_fp32(ctx, cfg, T, d, V, R, static_cast<const float*>(H), static_cast<const float*>(W),
                          y, old_logp, cs, adv, w, keep, logp, lse, g, loss, metrics, accumulate, workspace, ex);
   }
-  if (cfg->dtype != AERO_BF16) return AERO_ERR_UNSUPPORTED;
-  if (d % 64 != 0) return AERO_ERR_UNSUPPORTED;
-  if (!aligned16(H) || !aligned16(W)) return AERO_ERR_INVALID;
   return aero_fwd_tc(ctx, cfg, T, d, V, R, H, W, y, old_logp, cs, adv, w, keep, logp, lse, g, loss,
                      metrics, accumulate, workspace, ex);
 }
@@ -202,6 +236,7 @@ int aero_grpo_loss_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d,
                        const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
                        float* logp, float* lse, float* g, float* loss, float* metrics,
                        int accumulate, void* workspace, size_t workspace_bytes) {
+  Range nv("aero_grpo_loss_fwd");
   const aero_fwd_extra ex = {nullptr, 0.f, 0.f, nullptr, 0};
   return fwd_dispatch(ctx, cfg, T, d, V, R, H, W, y, old_logp, cs, adv, w, keep, logp, lse, g, loss, metrics,
                       accumulate, workspace, workspace_bytes, ex);
@@ -213,6 +248,7 @@ int aero_grpo_loss_reg_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_
                            const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
                            float* logp, float* lse, float* g, float* entropy, float* loss, float* metrics,
                            int accumulate, void* workspace, size_t workspace_bytes) {
+  Range nv("aero_grpo_loss_reg_fwd");
   if (!cfg) return AERO_ERR_INVALID;
   const aero_fwd_extra ex = {ref_logp, ref_logp ? cfg->kl_beta : 0.f, entropy ? cfg->ent_coef : 0.f, entropy, 0};
   return fwd_dispatch(ctx, cfg, T, d, V, R, H, W, y, old_logp, cs, adv, w, keep, logp, lse, g, loss, metrics,
@@ -223,6 +259,7 @@ int aero_logprob_fwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, i
                      const void* H, const void* W, const int32_t* y,
                      float* logp, float* lse, float* entropy,
                      void* workspace, size_t workspace_bytes) {
+  Range nv("aero_logprob_fwd");
   const aero_fwd_extra ex = {nullptr, 0.f, 0.f, entropy, 1};
   return fwd_dispatch(ctx, cfg, T, d, V, 0, H, W, y, nullptr, nullptr, nullptr, nullptr, nullptr, logp, lse, nullptr,
                       nullptr, nullptr, 0, workspace, workspace_bytes, ex);
@@ -240,24 +277,25 @@ int aero_grpo_loss_kl_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int
                               float* logp, float* lse, float* g, float* loss, float* metrics,
                               float grad_scale, void* dH, float* dW, int accumulate_dW,
                               void* workspace, size_t workspace_bytes) {
-  int rc = check_ctx(ctx);
-  if (rc) return rc;
-  if (!cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
+  Range nv("aero_grpo_loss_fwd_bwd");
+  if (!ctx || !cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
   if (!W || !cs || !loss || !dW) return AERO_ERR_INVALID;
   if (T > 0 && (!H || !y || !old_logp || !logp || !lse || !g || !dH)) return AERO_ERR_INVALID;
   if (R > 0 && (!adv || !w || !keep)) return AERO_ERR_INVALID;
   if (!workspace || !aligned256(workspace)) return AERO_ERR_INVALID;
   if (cfg->dtype == AERO_FP32) {
-    rc = aero_grpo_loss_reg_fwd(ctx, cfg, T, d, V, R, H, W, y, old_logp, ref_logp, cs, adv, w, keep, logp, lse, g,
-                                nullptr, loss, metrics, 0, workspace, workspace_bytes);
+    int rc = aero_grpo_loss_reg_fwd(ctx, cfg, T, d, V, R, H, W, y, old_logp, ref_logp, cs, adv, w, keep, logp, lse, g,
+                                    nullptr, loss, metrics, 0, workspace, workspace_bytes);
     if (rc) return rc;
-    return aero_grpo_loss_bwd(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, grad_scale, dH, dW, accumulate_dW,
+    return aero_grpo_loss_bwd(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, logp, grad_scale, dH, dW, accumulate_dW,
                               workspace, workspace_bytes);
   }
   if (cfg->dtype != AERO_BF16) return AERO_ERR_UNSUPPORTED;
   if (d % 64 != 0) return AERO_ERR_UNSUPPORTED;
   if (!aligned16(H) || !aligned16(W) || !aligned16(dH) || !aligned16(dW)) return AERO_ERR_INVALID;
   if (workspace_bytes < aero_fwd_bwd_ws_bytes_tc(T, d, V, R, 128)) return AERO_ERR_WORKSPACE;
+  const int rc = check_ctx(ctx);
+  if (rc) return rc;
   return aero_fwd_bwd_tc(ctx, cfg, T, d, V, R, H, W, y, old_logp, ref_logp, cfg->kl_beta, cs, adv, w, keep, logp, lse, g,
                          loss, metrics, grad_scale, dH, dW, accumulate_dW, workspace, workspace_bytes);
 }
@@ -282,13 +320,13 @@ static int bwd_dispatch(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d
                         const float* lse, const float* g, float grad_scale,
                         void* dH, float* dW, int accumulate_dW,
                         void* workspace, size_t workspace_bytes, const aero_bwd_extra& ex) {
-  int rc = check_ctx(ctx);
-  if (rc) return rc;
-  if (!cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
+  if (!ctx || !cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
   if (!W || !cs || !dW) return AERO_ERR_INVALID;
   if (T > 0 && (!H || !y || !lse || !g || !dH)) return AERO_ERR_INVALID;
   if (R > 0 && !keep) return AERO_ERR_INVALID;
   if (cfg->dtype == AERO_FP32) {
+    const int rc = check_ctx(ctx);
+    if (rc) return rc;
     return aero_bwd_fp32(ctx, cfg, T, d, V, R, static_cast<const float*>(H), static_cast<const float*>(W),
                          y, cs, keep, lse, g, grad_scale, static_cast<float*>(dH), dW, accumulate_dW, ex);
   }
@@ -297,6 +335,8 @@ static int bwd_dispatch(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d
   if (!aligned16(H) || !aligned16(W) || !aligned16(dH) || !aligned16(dW)) return AERO_ERR_INVALID;
   if (!workspace || !aligned256(workspace)) return AERO_ERR_INVALID;
   if (workspace_bytes < aero_bwd_ws_bytes_tc(T, d, V, R, 128)) return AERO_ERR_WORKSPACE;
+  const int rc = check_ctx(ctx);
+  if (rc) return rc;
   return aero_bwd_tc(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, grad_scale, dH, dW, accumulate_dW,
                      workspace, workspace_bytes, ex);
 }
@@ -304,10 +344,11 @@ static int bwd_dispatch(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d
 int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                        const void* H, const void* W, const int32_t* y,
                        const int64_t* cs, const uint8_t* keep,
-                       const float* lse, const float* g, float grad_scale,
+                       const float* lse, const float* g, const float* logp, float grad_scale,
                        void* dH, float* dW, int accumulate_dW,
                        void* workspace, size_t workspace_bytes) {
-  const aero_bwd_extra ex = {nullptr, nullptr, 0.f};
+  Range nv("aero_grpo_loss_bwd");
+  const aero_bwd_extra ex = {nullptr, nullptr, 0.f, logp};
   return bwd_dispatch(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, grad_scale, dH, dW, accumulate_dW, workspace,
                       workspace_bytes, ex);
 }
@@ -315,12 +356,13 @@ int aero_grpo_loss_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d,
 int aero_grpo_loss_reg_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                            const void* H, const void* W, const int32_t* y,
                            const int64_t* cs, const uint8_t* keep,
-                           const float* lse, const float* g, const float* entropy, const float* w,
+                           const float* lse, const float* g, const float* logp, const float* entropy, const float* w,
                            float grad_scale, void* dH, float* dW, int accumulate_dW,
                            void* workspace, size_t workspace_bytes) {
+  Range nv("aero_grpo_loss_reg_bwd");
   if (!cfg) return AERO_ERR_INVALID;
   if ((entropy == nullptr) != (w == nullptr)) return AERO_ERR_INVALID;
-  const aero_bwd_extra ex = {entropy, w, entropy ? cfg->ent_coef : 0.f};
+  const aero_bwd_extra ex = {entropy, w, entropy ? cfg->ent_coef : 0.f, logp};
   return bwd_dispatch(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, grad_scale, dH, dW, accumulate_dW, workspace,
                       workspace_bytes, ex);
 }

@@ -6,7 +6,6 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
-#include <stdlib.h>
 
 #include "../../include/aero.h"
 
@@ -28,6 +27,10 @@ struct aero_ctx {
   cudaEvent_t slice_ev[16];
   int n_slices;
   long long rows_per_slice;
+  // tuning hooks (aero_set_tuning); the defaults mean "let the library decide"
+  int tune_vsplit;        // 0: by d (aero_vsplit_auto); else 1, 2 or 4 CTA pairs per pair of token tiles
+  int tune_nsync;         // < 0: the default number of meeting points; 0: no pacing; else that many
+  int tune_rowscale;      // < 0 or 1: row factors in the backward GEMMs; 0: the pass that rewrites the block
 };
 
 #define AERO_CUDA_TRY(expr)                          \
@@ -53,6 +56,9 @@ int aero_group_stats_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32
                             int32_t* kept_ids, int64_t* kept_tok_off, int64_t* counters,
                             float* metrics, void* ws);
 
+int aero_finalize_weights_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t R, int32_t P_local, int64_t P_global,
+                                 float* w, const int64_t* counters_local, const int64_t* counters_global);
+
 // Optional terms of the objective beyond the clipped surrogate: Eq. 2's KL to a reference
 // policy and the entropy bonus of Table 9.  All-zero / NULL means the plain objective.
 struct aero_fwd_extra {
@@ -66,6 +72,8 @@ struct aero_bwd_extra {
   const float* entropy;    // [T] from the forward, or NULL
   const float* w;          // [R] rollout weights (entropy term only)
   float ent_coef;
+  const float* logp;       // [T] log-probs from the forward, or NULL: the target column of dz is then
+                           // formed from exp(z_y - lse) recomputed in fp32
 };
 
 // ---- stage (b): helpers shared by the fp32 and the tensor-core paths ---------------
@@ -103,30 +111,28 @@ int aero_bwd_fp32(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int3
 // Number of CTA pairs that share a pair of token tiles and split the vocabulary between them:
 // the smallest power of two that brings the H tiles all 148 CTAs keep re-reading from L2
 // (148 * 128 * d * 2 bytes) under 72 MB, a bit over half of the 126 MB L2.
-static inline int aero_vsplit(int32_t d) {
-  if (const char* e = getenv("AERO_VSPLIT")) {          // override for tests and tuning: 1, 2, 4 or 8
-    const int v = atoi(e);
-    if (v == 1 || v == 2 || v == 4 || v == 8) return v;
-  }
+static inline int aero_vsplit_auto(int32_t d) {
   const double live = 148.0 * 128.0 * (double)d * 2.0;
   int s = 1;
   while (live / s > 72.0 * 1024 * 1024 && s < 8) s *= 2;
   return s;
 }
+// Largest split a context may be tuned to (aero_set_tuning); workspaces are sized for it.
+constexpr int kAeroMaxForcedVsplit = 4;
+static inline int aero_vsplit_cap(int32_t d) {
+  const int a = aero_vsplit_auto(d);
+  return a > kAeroMaxForcedVsplit ? a : kAeroMaxForcedVsplit;
+}
+static inline int aero_vsplit(const aero_ctx* ctx, int32_t d) {
+  return ctx->tune_vsplit > 0 ? ctx->tune_vsplit : aero_vsplit_auto(d);
+}
 // Meeting points per unit of the lm_head kernel's producers (0 switches the pacing off).
-static inline int aero_nsync() {
-  if (const char* e = getenv("AERO_NSYNC")) return atoi(e) > 0 ? atoi(e) : 0;
-  return 32;
-}
+static inline int aero_nsync(const aero_ctx* ctx) { return ctx->tune_nsync >= 0 ? ctx->tune_nsync : 32; }
 // One-call step: the backward GEMMs take p~ as it is, with the row factors applied to the dH
-// tiles and to a scaled copy of the chunk's H rows, instead of a pass that rewrites the block
-// (AERO_ROWSCALE=0 keeps that pass).  With several vocabulary splits this needs one shift per
-// row for all of them (lmhead::Params::common_shift).
-static inline bool aero_rowscale(int32_t d) {
-  (void)d;
-  if (const char* e = getenv("AERO_ROWSCALE")) { if (atoi(e) == 0) return false; }
-  return true;
-}
+// tiles and to a scaled copy of the chunk's H rows, instead of a pass that rewrites the block.
+// With several vocabulary splits this needs one shift per row for all of them
+// (lmhead::Params::common_shift).
+static inline bool aero_rowscale(const aero_ctx* ctx) { return ctx->tune_rowscale != 0; }
 size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t d, int32_t R);
 int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                 const void* H, const void* W, const int32_t* y, const float* old_logp,

@@ -920,6 +920,41 @@ int aero_group_stats_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32
   return AERO_OK;
 }
 
+// ---- weights of a data-parallel shard -----------------------------------------------------
+namespace {
+
+// Eq. 2's normalisers are batch-wide.  A rank that ran the group stage on its own prompts holds
+// weights over its local denominator; multiplying by local / global denominator (both read from
+// the counters on the device, so the host never waits) gives the weights of the whole batch.
+__global__ void __launch_bounds__(256) finalize_weights_kernel(aero_cfg cfg, int R, long long P_local, long long P_global,
+                                                               float* __restrict__ w,
+                                                               const int64_t* __restrict__ cl, const int64_t* __restrict__ cg) {
+  long long num, den;
+  if (cfg.agg == AERO_TOKEN_MEAN) {
+    const int k = cfg.denom == AERO_DENOM_SURVIVING ? AERO_CNT_T_KEPT : AERO_CNT_T_PRESENT;
+    num = cl[k]; den = cg[k];
+  } else if (cfg.denom == AERO_DENOM_SURVIVING) {
+    num = cl[AERO_CNT_P_SURV]; den = cg[AERO_CNT_P_SURV];
+  } else {
+    num = P_local; den = P_global;
+  }
+  const double f = den > 0 ? (double)num / (double)den : 0.0;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < R; i += gridDim.x * blockDim.x)
+    w[i] = (float)((double)w[i] * f);
+}
+
+}  // namespace
+
+int aero_finalize_weights_launch(aero_ctx* ctx, const aero_cfg* cfg, int32_t R, int32_t P_local, int64_t P_global,
+                                 float* w, const int64_t* counters_local, const int64_t* counters_global) {
+  if (R == 0) return AERO_OK;
+  const int blocks = (R + 255) / 256 < 4 * ctx->sm_count ? (R + 255) / 256 : 4 * ctx->sm_count;
+  finalize_weights_kernel<<<blocks, 256, 0, ctx->stream>>>(*cfg, R, P_local, P_global, w, counters_local, counters_global);
+  ctx->launches += 1;
+  AERO_CUDA_TRY(cudaGetLastError());
+  return AERO_OK;
+}
+
 // ---- variant with library-owned scratch ------------------------------------------------
 // The kernels above need a few bytes of scratch per prompt and per tile.  This entry point takes
 // them from a fixed array in device memory that is part of the loaded library image, so the

@@ -101,10 +101,16 @@ struct Params {
   float* shift_out;             // MODE_FWD_P: c_t * log2(e) per split and row, [vsplit][T]
   int common_shift;             // MODE_FWD_P with vsplit > 1: every split takes c_t from the row's first 32 logits
                                 // of the whole vocabulary (the later splits compute that tile once more for it)
+  // MODE_FWD_P: rows with a logit too far above c_t for bf16 to hold exp(z - c_t) are listed here (row index
+  // inside the chunk) so that the step can redo them; AERO_ST_RANGE is raised only if the list overflows
+  int* range_rows;
+  int* range_count;
+  int range_cap;
   double* partials;             // [tile][4 epilogue warps][kPartialStride]
   // dz modes
   const float* lse_in;
   const float* g_in;
+  const float* logp_in;         // NULL, or the forward's log-probs: the target column is then -coef expm1(logp_t)
   const float* ent_in;
   float grad_scale;
   __nv_bfloat16* dz;            // tiled: [tile - tile_begin][ldz / 64][128 rows][64 columns]
@@ -125,13 +131,27 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // End of a token row in the forward modes: log-sum-exp, log-prob, entropy, then Eq. 2 (with the
 // KL term when a reference is given) and the warp's record of loss partials.  Called by the four
 // epilogue warps of a tile (warp = 0..3), with the merged running state of the row.
+// The running state leaves the target's own column out: m2 is the largest of the other logits
+// (log2 domain), l = sum_{v != y} 2^(z_v log2e - m2), sz = sum_{v != y} 2^(..) z_v.  With
+// a = z_y log2e - m2 the log-prob is -log(1 + l 2^-a): for a confident token (l 2^-a tiny) this
+// keeps the relative accuracy of 1 - p_y = l / (l + 2^a), which z_y - lse loses to the rounding
+// of lse at the magnitude of the logits and to the rounding of a sum that sits next to 1.
 __device__ __forceinline__ void finish_rows(const Params& p, bool ent_mode, bool live, long long row, int tile, int warp,
                                             int lane, float m2, float l, float zy, float sz) {
   double part[kPartialStride] = {0.0, 0.0, 0.0, 0.0, 0.0};
   if (live) {
-    const float ls = (m2 + __log2f(l)) * kLn2;
-    const float lp = zy - ls;
-    const float ent = ent_mode ? ls - sz / l : 0.f;       // H = lse - E_p[z]
+    float ls, lp, ent = 0.f;
+    if (l > 0.f) {
+      const float a = fmaf(zy, kLog2e, -m2);               // the target's exponent relative to m2
+      const float big = fmaxf(a, 0.f);                     // everything below is scaled by 2^-big: no overflow
+      const float ey = exp2f(a - big), lr = l * exp2f(-big);
+      ls = (m2 + big + log2f(lr + ey)) * kLn2;
+      lp = a > -40.f ? -log1pf(l * exp2f(-a)) : (a - log2f(l + exp2f(a))) * kLn2;
+      if (ent_mode) ent = ls - (sz * exp2f(-big) + ey * zy) / (lr + ey);       // H = lse - E_p[z]
+    } else {                                               // no other column carries weight: p_y = 1
+      ls = zy;
+      lp = 0.f;
+    }
     p.logp[row] = lp;
     p.lse_out[row] = ls;
     if (ent_mode) p.ent_out[row] = ent;
@@ -337,18 +357,32 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
       float c2 = 0.f;                                      // MODE_FWD_P: shift of the stored exponentials, log2 domain
       bool c2_set = false;                                 // ... taken from vocabulary tile 0 by a later split
       float lse2 = 0.f, coef = 0.f, et = 0.f, c0 = 0.f;     // dz per-row constants: dz = 1[y] coef + p (c0 + et z)
+      float ls_nat = 0.f, lp_row = 0.f, ent_row = 0.f;      // ... and what the target column needs besides
+      bool have_lp = false;
       if (IS_DZ) {
         if (live) {
           const float ls = p.lse_in[row];
+          ls_nat = ls;
           lse2 = ls * kLog2e;
           coef = p.g_in[row] * p.grad_scale;
           c0 = -coef;
+          if (p.logp_in != nullptr) { lp_row = p.logp_in[row]; have_lp = true; }
           if (ENT) {
             et = p.ent_coef * p.w[aero_owner(p.cs, p.R, row)] * p.grad_scale;
-            c0 += et * (p.ent_in[row] - ls);
+            ent_row = p.ent_in[row];
+            c0 += et * (ent_row - ls);
           }
         }
       }
+      // Target column of a dz row: coef (1 - p_y) + et p_y (log p_y + H_t), with 1 - p_y = -expm1(log p_y)
+      // so that a confident token (p_y close to 1) keeps the relative accuracy of its log-prob.
+      auto dz_target = [&](float z) {
+        const float lpy = have_lp ? lp_row : z - ls_nat;
+        float v = -coef * expm1f(lpy);
+        if (ENT) v = fmaf(et * __expf(lpy), lpy + ent_row, v);
+        return v;
+      };
+      bool range_hit = false;                              // MODE_FWD_P: exp(z - c_t) saturated somewhere in this row
 
       for (int j0 = unit_j0(k), jj = j0 - unit_pre(k), j1 = unit_j1(k); ok && jj < j1; ++jj, ++at) {
         const int j = jj < j0 ? 0 : jj;
@@ -369,9 +403,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
           __syncwarp();
           tc::tmem_ld_32x32(tmem_base + ((uint32_t)(warp * 32) << 16) + buf * BN, r0);
           tc::tmem_ld_wait();
-          float cmax = __uint_as_float(r0[0]);
+          // (the same 32 logits the first split sees: columns past V and the target's own masked)
+          float cmax = yt == 0 ? kMasked : __uint_as_float(r0[0]);
 #pragma unroll
-          for (int q = 1; q < 32; ++q) cmax = fmaxf(cmax, q < p.V ? __uint_as_float(r0[q]) : kMasked);
+          for (int q = 1; q < 32; ++q) cmax = fmaxf(cmax, (q < p.V && q != yt) ? __uint_as_float(r0[q]) : kMasked);
           c2 = fmaf(cmax + kShiftMargin, kLog2e, 0.f);
           c2_set = true;
           tc::tc_fence_before();
@@ -423,6 +458,12 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
 #pragma unroll
               for (int q = 0; q < 32; ++q) if (col0 + q >= p.V) z[q] = kMasked;
             }
+            if ((unsigned)(yt - col0) < 32u) {
+              // the target's column is kept out of the running sums (see finish_rows)
+              const int sel = yt - col0;
+#pragma unroll
+              for (int q = 0; q < 32; ++q) if (q == sel) { zy = z[q]; z[q] = kMasked; }
+            }
             float cmax = z[0];
 #pragma unroll
             for (int q = 1; q < 32; ++q) cmax = fmaxf(cmax, z[q]);
@@ -432,7 +473,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
             if (STORE_P) {
               // e^(z - c) = e^(z - m) * 2^(m2 - c2): one extra multiply per logit
               const float d2 = m2n - c2;
-              if (live && d2 > 126.f) aero_raise(p.status, AERO_ST_RANGE);
+              range_hit |= live && d2 > 126.f;
               const float sc = live ? ex2(fminf(d2, 126.f)) : 0.f;
               uint32_t pk[16];
 #pragma unroll
@@ -454,11 +495,6 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
             l = fmaf(l, scale, acc);
             if (ENT) sz = fmaf(sz, scale, accz);
             m2 = m2n;
-            if ((unsigned)(yt - col0) < 32u) {
-              const int sel = yt - col0;
-#pragma unroll
-              for (int q = 0; q < 32; ++q) if (q == sel) zy = z[q];
-            }
           } else {
             // 32 columns -> 16 packed words -> half of this row's 128-byte line in the staging
             // buffer (16-byte chunks XOR-swizzled with the row, matching the store's tensor map)
@@ -474,7 +510,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
               if ((unsigned)(yt - col0) < 32u) {
                 const int sel = yt - col0;
 #pragma unroll
-                for (int q = 0; q < 32; ++q) if (q == sel) v[q] += coef;
+                for (int q = 0; q < 32; ++q) if (q == sel) v[q] = dz_target(__uint_as_float(r[q]));
               }
 #pragma unroll
               for (int q = 0; q < 32; q += 2) pk[q >> 1] = pack_bf16(v[q], v[q + 1]);
@@ -484,8 +520,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
                 const float z0 = __uint_as_float(r[q]), z1 = __uint_as_float(r[q + 1]);
                 float v0 = ex2(fmaf(z0, kLog2e, -lse2)) * (ENT ? fmaf(et, z0, c0) : c0);
                 float v1 = ex2(fmaf(z1, kLog2e, -lse2)) * (ENT ? fmaf(et, z1, c0) : c0);
-                if (col0 + q == yt) v0 += coef;
-                if (col0 + q + 1 == yt) v1 += coef;
+                if (col0 + q == yt) v0 = dz_target(z0);
+                if (col0 + q + 1 == yt) v1 = dz_target(z1);
                 if (!live || col0 + q >= p.V) v0 = 0.f;
                 if (!live || col0 + q + 1 >= p.V) v1 = 0.f;
                 pk[q >> 1] = pack_bf16(v0, v1);
@@ -516,6 +552,11 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
       }
 
       if (STORE_P && ok && have_tile && live) p.shift_out[(size_t)((pair + k * npairs) % vsplit) * p.T + row] = c2;
+      if (STORE_P && range_hit) {
+        const int slot = atomicAdd(p.range_count, 1);
+        if (slot < p.range_cap) p.range_rows[slot] = (tile - p.tile_begin) * BM + r_in_tile;
+        else aero_raise(p.status, AERO_ST_RANGE);
+      }
       if (!IS_DZ && ok && have_tile) {
         if (vsplit > 1) {
           if (live) p.xstate[(size_t)((pair + k * npairs) % vsplit) * p.T + row] = make_float4(m2, l, zy, sz);

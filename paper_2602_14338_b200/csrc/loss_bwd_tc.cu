@@ -93,10 +93,10 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     lp.tile_row = tiles.tile_row; lp.tile_valid = tiles.tile_valid; lp.n_tiles = tiles.n_tiles;
     lp.tile_begin = (int)begin; lp.tile_end = (int)(begin + tpc);
     lp.y = y; lp.status = ctx->d_status;
-    lp.lse_in = lse; lp.g_in = g; lp.grad_scale = grad_scale; lp.dz = dz; lp.ldz = ldz;
+    lp.lse_in = lse; lp.g_in = g; lp.logp_in = ex.logp; lp.grad_scale = grad_scale; lp.dz = dz; lp.ldz = ldz;
     lp.cs = cs; lp.w = ex.w; lp.ent_in = ex.entropy; lp.ent_coef = ex.ent_coef;
-    lp.vsplit = aero_vsplit(d);
-    lp.sync_ctr = sync_ctr; lp.nsync = aero_nsync();
+    lp.vsplit = aero_vsplit(ctx, d);
+    lp.sync_ctr = sync_ctr; lp.nsync = aero_nsync(ctx);
     AERO_CUDA_TRY(cudaMemsetAsync(sync_ctr, 0, 256, ctx->stream));
     const long long max_pairs = ctx->sm_count / 2 > 0 ? ctx->sm_count / 2 : 1;
     const long long dz_pairs = (tpc + 1) / 2 * lp.vsplit;

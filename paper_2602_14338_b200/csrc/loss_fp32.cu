@@ -53,8 +53,11 @@ fwd_fp32_kernel(aero_cfg cfg, long long T, int d, int V, int R,
       continue;
     }
     const float* h = H + (size_t)t * d;
-    float m = -INFINITY, l = 0.f, sz = 0.f;       // sz = sum_v exp(z_v - m) z_v, for the entropy
+    // running sums over every column but the target's own: with a = z_y - m the log-prob is
+    // -log(1 + l e^-a), which keeps the relative accuracy of 1 - p_y for a confident token
+    float m = -INFINITY, l = 0.f, sz = 0.f;       // sz = sum_{v != y} exp(z_v - m) z_v, for the entropy
     for (int v = lane; v < V; v += 32) {
+      if (v == yt) continue;
       const float z = dot_row(h, W + (size_t)v * d, d);
       const float mn = fmaxf(m, z);
       const float sc = __expf(m - mn), e = __expf(z - mn);
@@ -63,14 +66,19 @@ fwd_fp32_kernel(aero_cfg cfg, long long T, int d, int V, int R,
       m = mn;
     }
     const float M = warp_max(m);
-    const float sc = __expf(m - M);
+    const float sc = m > -INFINITY ? __expf(m - M) : 0.f;
     l = warp_sum(l * sc);
     sz = warp_sum(sz * sc);
-    const float ls = M + __logf(l);
     if (lane == 0) {
       const float zy = dot_row(h, W + (size_t)yt * d, d);
-      const float lp = zy - ls;
-      const float ent = ls - sz / l;              // H = lse - E_p[z]
+      float ls = zy, lp = 0.f, ent = 0.f;         // (a vocabulary of one: p_y = 1)
+      if (l > 0.f) {
+        const float a = zy - M, big = fmaxf(a, 0.f);
+        const float ey = expf(a - big), lr = l * expf(-big);
+        ls = M + big + logf(lr + ey);
+        lp = a > -30.f ? -log1pf(l * expf(-a)) : a - logf(l + expf(a));
+        ent = ls - (sz * expf(-big) + ey * zy) / (lr + ey);      // H = lse - E_p[z]
+      }
       logp[t] = lp; lse[t] = ls;
       if (ex.entropy) ex.entropy[t] = ent;
       for (int k = 0; k < kPartialStride; ++k) pr[k] = 0.0;
@@ -97,6 +105,14 @@ fwd_fp32_kernel(aero_cfg cfg, long long T, int d, int V, int R,
 
 // Per-row constants of dz = gs * (g (1[v=y] - p) + e p (z - lse + H)) = 1[v=y] coef + p (c0 + et z).
 struct RowDz { float coef, c0, et; };
+// One entry of a dz row.  The target column is coef (1 - p_y) + et p_y (log p_y + H) with
+// 1 - p_y = -expm1(log p_y), log p_y being the forward's log-prob when it is given.
+__device__ __forceinline__ float dz_entry(const RowDz& rd, float z, float ls, bool is_target, const float* logp, long long t) {
+  const float base = __expf(z - ls) * fmaf(rd.et, z, rd.c0);
+  if (!is_target) return base;
+  const float lp = logp ? logp[t] : z - ls;
+  return -rd.coef * expm1f(lp) + __expf(lp) * (fmaf(rd.et, z, rd.c0) + rd.coef);
+}
 __device__ __forceinline__ RowDz row_dz(long long t, float gs, const float* __restrict__ g, const float* __restrict__ lse,
                                         const int64_t* __restrict__ cs, int R, const uint8_t* __restrict__ keep,
                                         const aero_bwd_extra& ex) {
@@ -142,7 +158,7 @@ bwd_dh_fp32_kernel(long long T, int d, int V, const float* __restrict__ H, const
         float part = 0.f;
         for (int k = lane; k < d; k += 32) part = fmaf(h[k], wv[k], part);
         const float z = warp_sum(part);
-        const float dz = (v == yt ? rd.coef : 0.f) + __expf(z - ls) * fmaf(rd.et, z, rd.c0);
+        const float dz = dz_entry(rd, z, ls, v == yt, ex.logp, t);
 #pragma unroll
         for (int q = 0; q < kChunk / 32; ++q) {
           const int k = c0 + q * 32 + lane;
@@ -181,7 +197,7 @@ bwd_dw_fp32_kernel(long long T, int d, int V, const float* __restrict__ H, const
         float part = 0.f;
         for (int k = lane; k < d; k += 32) part = fmaf(h[k], wv[k], part);
         const float z = warp_sum(part);
-        const float dz = (v == y[t] ? rd.coef : 0.f) + __expf(z - lse[t]) * fmaf(rd.et, z, rd.c0);
+        const float dz = dz_entry(rd, z, lse[t], v == y[t], ex.logp, t);
 #pragma unroll
         for (int q = 0; q < kChunk / 32; ++q) {
           const int k = c0 + q * 32 + lane;

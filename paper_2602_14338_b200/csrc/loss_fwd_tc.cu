@@ -32,8 +32,8 @@ FwdWs carve_fwd(void* ws, int64_t T, int32_t R) {
 }  // namespace
 
 size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t d, int32_t R) {
-  const int vs = aero_vsplit(d);
-  const size_t state = vs > 1 ? aero_align_up((size_t)vs * (size_t)(T > 0 ? T : 1) * sizeof(float4), 256) : 0;
+  const int vs = aero_vsplit_cap(d);
+  const size_t state = aero_align_up((size_t)vs * (size_t)(T > 0 ? T : 1) * sizeof(float4), 256);
   return aero_tiles_bytes(T, R, lmhead::BM) + partials_bytes(T, R) + 256 + state;
 }
 
@@ -66,8 +66,8 @@ int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     p.T = T; p.d = d; p.V = V; p.R = R;
     p.tile_row = f.tiles.tile_row; p.tile_valid = f.tiles.tile_valid; p.n_tiles = f.tiles.n_tiles;
     p.tile_begin = 0; p.tile_end = f.tiles.max_tiles;
-    p.vsplit = aero_vsplit(d); p.xstate = f.xstate;
-    p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync();
+    p.vsplit = aero_vsplit(ctx, d); p.xstate = f.xstate;
+    p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync(ctx);
     p.y = y; p.status = ctx->d_status;
     p.old_logp = ex.logprob_only ? nullptr : old_logp; p.cs = cs; p.adv = adv; p.w = w;
     p.ref_logp = ex.ref_logp; p.kl_beta = ex.kl_beta; p.ent_coef = ex.ent_coef; p.ent_out = ex.entropy;

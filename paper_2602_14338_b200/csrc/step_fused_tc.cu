@@ -3,14 +3,17 @@
 //   lmhead_kernel<MODE_FWD_P>  logits, online log-sum-exp, Eq. 2, and p~ = exp(z - c_t) in bf16 into
 //                              the chunk's tiled block (instead of recomputing the logits later)
 //   merge_kernel               (large d only) merges the running states of the vocabulary splits
-//   scale_dz_kernel            dz = gs (g_t 1[v = y_t] - g_t exp(c_t - lse_t) p~), in place
+//   scale_dz_kernel            dz = gs (g_t 1[v = y_t] - g_t exp(c_t - lse_t) p~), in place (the target's entry
+//                              as -gs g_t expm1(logp_t), not by subtraction from the rounded p~)
 //   gemm_kernel<DH>, <DW>      dH rows of the chunk, dW += dz^T H
 // When every row has one shift c_t (one vocabulary split, or several that share the shift) it has
 // one factor s_t = -gs g_t exp(c_t - lse_t), and the rewriting pass is replaced by
-//   row_factors_kernel         p~[t, y_t] -= exp(lse_t - c_t) (so that dz = s_t p~), s_t, and the
-//                              chunk's rows of H times s_t
+//   row_factors_kernel         p~[t, y_t] = expm1(logp_t) exp(lse_t - c_t), i.e. lowered by the row's sum of p~
+//                              (so that dz = s_t p~), s_t, and the chunk's rows of H times s_t
 //   gemm_kernel<DH>, <DW>      dH = s_t (p~ W) with the factor applied to the finished tile,
 //                              dW += p~^T (s H)
+//   range_fix_kernel           rows in which bf16 could not hold exp(z - c_t) (a logit more than ~87 above the
+//                              shift; the forward lists them) get their dz row recomputed from H and W
 // and once at the end the fixed-order reduction of the loss partials.
 #include "gemm_bwd_kernel.cuh"
 #include "lmhead_kernel.cuh"
@@ -23,8 +26,9 @@ namespace {
 inline long long ldz_of(int32_t V) { return ((long long)V + 63) / 64 * 64; }
 // bytes of one token tile in the chunk's blocks: 128 rows of p~ / dz, and of the scaled H rows if used
 inline size_t chunk_tile_bytes(int32_t d, int32_t V) {
-  return (size_t)128 * ((size_t)ldz_of(V) * 2 + (aero_rowscale(d) ? (size_t)d * 2 : 0));
+  return (size_t)128 * ((size_t)ldz_of(V) * 2 + (size_t)d * 2);
 }
+constexpr int kRangeCap = 1024;      // rows per chunk the step can redo after a saturated exp(z - c_t)
 
 struct ScaleArgs {
   __nv_bfloat16* dz;        // tiled: [tile - tile_begin][ldz / 64][128][64]
@@ -38,6 +42,7 @@ struct ScaleArgs {
   const int32_t* y;
   const float* lse;
   const float* g;
+  const float* logp;
   const float* shift;       // [vsplit][T], log2 domain
   float grad_scale;
 };
@@ -59,12 +64,13 @@ __global__ void __launch_bounds__(256) scale_dz_kernel(ScaleArgs a) {
     const int b = b0 + blk;
     const long long row = (long long)row0 + r;
     uint4* ptr = reinterpret_cast<uint4*>(a.dz + (((size_t)blockIdx.y * a.nblk + b) * 128 + r) * 64 + seg * 8);
-    float coef = 0.f, sc = 0.f;
+    float coef = 0.f, sc = 0.f, tgt = 0.f;
     int yt = -1;
     if (r < valid && row < a.T) {
       coef = a.g[row] * a.grad_scale;
       yt = a.y[row];
       if (coef != 0.f) {
+        tgt = -coef * expm1f(a.logp[row]);          // coef (1 - p_y), exact for p_y close to 1
         // the vocabulary split that produced this column block, and its shift
         const int j = b / (lmhead::BN / 64);
         int s = 0;
@@ -78,8 +84,8 @@ __global__ void __launch_bounds__(256) scale_dz_kernel(ScaleArgs a) {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       float2 f = __bfloat1622float2(h[q]);
-      f.x = (col0 + 2 * q == yt ? coef : 0.f) + sc * f.x;
-      f.y = (col0 + 2 * q + 1 == yt ? coef : 0.f) + sc * f.y;
+      f.x = col0 + 2 * q == yt ? tgt : sc * f.x;
+      f.y = col0 + 2 * q + 1 == yt ? tgt : sc * f.y;
       h[q] = __floats2bfloat162_rn(f.x, f.y);
     }
     *ptr = v;
@@ -98,6 +104,7 @@ struct RowArgs {
   const int32_t* y;
   const float* lse;
   const float* g;
+  const float* logp;
   const float* shift;       // [T], log2 domain
   float grad_scale;
   const __nv_bfloat16* H;   // [T, d]
@@ -107,7 +114,10 @@ struct RowArgs {
 
 // One warp per row of the chunk's token tiles.  dz_tv = gs g_t (1[v = y_t] - p_tv) with
 // p_tv = p~_tv exp(c_t - lse_t), so with s_t = -gs g_t exp(c_t - lse_t) and the target's entry
-// lowered by exp(lse_t - c_t) (the sum of the row's p~), dz = s_t p~ everywhere.
+// lowered by exp(lse_t - c_t) (the sum of the row's p~), dz = s_t p~ everywhere.  The lowered
+// entry is (p_y - 1) exp(lse_t - c_t); it is written as expm1(logp_t) exp(lse_t - c_t) from the
+// fp32 log-prob, because subtracting from the bf16-rounded p~_y would leave an error of
+// 2^-9 p_y / (1 - p_y) relative, which is everything for a confident token.
 __global__ void __launch_bounds__(256) row_factors_kernel(RowArgs a) {
   const int n_tiles = min(*a.n_tiles, a.tile_end);
   const int lt = blockIdx.x / 16;                       // 16 blocks of 8 rows per tile
@@ -130,7 +140,9 @@ __global__ void __launch_bounds__(256) row_factors_kernel(RowArgs a) {
       if (lane == 0) {
         const int yt = a.y[row];
         __nv_bfloat16* pt = a.dz + (((size_t)lt * a.nblk + yt / 64) * 128 + r) * 64 + yt % 64;
-        *pt = __float2bfloat16_rn(__bfloat162float(*pt) - exp2f(-e));
+        // (lse_t far above c_t: the factor s_t underflows with exp2(e) and the row's dz is zero to rounding;
+        // the clamp only keeps this entry finite, so that 0 * entry stays 0)
+        *pt = __float2bfloat16_rn(expm1f(a.logp[row]) * exp2f(fminf(-e, 126.f)));
       }
     }
     if (lane == 0) a.row_scale[row] = sc;
@@ -148,6 +160,75 @@ __global__ void __launch_bounds__(256) row_factors_kernel(RowArgs a) {
         h[q] = __floats2bfloat162_rn(sc * f.x, sc * f.y);
       }
       dst[k] = v;
+    }
+  }
+}
+
+struct RangeArgs {
+  const int* rows;          // chunk-local rows (tile in chunk * 128 + row in tile) listed by the forward
+  const int* count;
+  int cap;
+  __nv_bfloat16* dz;        // tiled as above
+  int nblk;
+  const int32_t* tile_row;
+  int tile_begin;
+  long long T;
+  int d, V;
+  const int32_t* y;
+  const float* lse;
+  const float* g;
+  const float* logp;
+  float grad_scale;
+  const __nv_bfloat16* H;   // [T, d]
+  const __nv_bfloat16* W;   // [V, d]
+  __nv_bfloat16* Hs;        // row-factor form: the row's copy of H (unscaled here); NULL otherwise
+  float* row_scale;         // row-factor form: set to 1 for a redone row
+};
+
+// The forward could not hold exp(z - c_t) of these rows in bf16: write their dz rows from the
+// definition, one warp per (row, vocabulary column), logits as fp32 dot products of the bf16
+// operands.  Rare by construction (a logit ~87 above the row's first ones), so speed is no concern;
+// without listed rows the kernel reads one word and returns.
+__global__ void __launch_bounds__(256) range_fix_kernel(RangeArgs a) {
+  const int n = min(*a.count, a.cap);
+  if (n == 0) return;
+  const int lane = threadIdx.x & 31;
+  const long long warp0 = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+  const long long nwarps = (long long)gridDim.x * 8;
+  const long long ldz = (long long)a.nblk * 64;
+  for (long long u = warp0; u < (long long)n * ldz; u += nwarps) {
+    const int e = (int)(u / ldz), v = (int)(u % ldz);
+    const int local = a.rows[e], lt = local / 128, r = local % 128;
+    const long long row = (long long)a.tile_row[a.tile_begin + lt] + r;
+    if (row >= a.T) continue;
+    const float coef = a.g[row] * a.grad_scale;
+    float val = 0.f;
+    if (v < a.V && coef != 0.f) {
+      const uint4* h = reinterpret_cast<const uint4*>(a.H + row * a.d);
+      const uint4* w = reinterpret_cast<const uint4*>(a.W + (long long)v * a.d);
+      float acc = 0.f;
+      for (int k = lane; k < a.d / 8; k += 32) {
+        const uint4 hv = h[k], wv = w[k];
+        const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&hv);
+        const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&wv);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float2 x = __bfloat1622float2(hp[q]), yv = __bfloat1622float2(wp[q]);
+          acc = fmaf(x.x, yv.x, acc);
+          acc = fmaf(x.y, yv.y, acc);
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      val = v == a.y[row] ? -coef * expm1f(a.logp[row]) : -coef * __expf(acc - a.lse[row]);
+    }
+    if (lane == 0) a.dz[(((size_t)lt * a.nblk + v / 64) * 128 + r) * 64 + v % 64] = __float2bfloat16_rn(val);
+    if (a.Hs != nullptr && v == 0) {
+      // the row's factor is already in its dz entries: unit factor, plain copy of the H row
+      if (lane == 0) a.row_scale[row] = 1.f;
+      const uint4* src = reinterpret_cast<const uint4*>(a.H + row * a.d);
+      uint4* dst = reinterpret_cast<uint4*>(a.Hs + ((size_t)lt * 128 + r) * a.d);
+      for (int k = lane; k < a.d / 8; k += 32) dst[k] = src[k];
     }
   }
 }
@@ -175,6 +256,8 @@ struct FusedWs {
   float4* xstate;
   float* shift;
   float* row_scale;
+  int* range_count;
+  int* range_rows;
   __nv_bfloat16* dz;
   size_t head_bytes;
 };
@@ -186,7 +269,7 @@ size_t partials_bytes(int64_t T, int32_t R) {
 
 FusedWs carve(void* ws, int64_t T, int32_t d, int32_t R) {
   FusedWs f;
-  const int vs = aero_vsplit(d);
+  const int vs = aero_vsplit_cap(d);
   const size_t Tn = (size_t)(T > 0 ? T : 1);
   char* p = static_cast<char*>(ws);
   f.tiles = aero_carve_tiles(ws, T, R, lmhead::BM);
@@ -194,9 +277,11 @@ FusedWs carve(void* ws, int64_t T, int32_t d, int32_t R) {
   f.partials = reinterpret_cast<double*>(p + off);             off += partials_bytes(T, R);
   f.n_partials = (size_t)f.tiles.max_tiles * 4;
   f.sync_ctr = reinterpret_cast<unsigned int*>(p + off);       off += 256;
-  f.xstate = reinterpret_cast<float4*>(p + off);               off += vs > 1 ? aero_align_up(vs * Tn * sizeof(float4), 256) : 0;
+  f.range_count = reinterpret_cast<int*>(p + off);             off += 256;
+  f.range_rows = reinterpret_cast<int*>(p + off);              off += aero_align_up(kRangeCap * sizeof(int), 256);
+  f.xstate = reinterpret_cast<float4*>(p + off);               off += aero_align_up(vs * Tn * sizeof(float4), 256);
   f.shift = reinterpret_cast<float*>(p + off);                 off += aero_align_up(vs * Tn * sizeof(float), 256);
-  f.row_scale = reinterpret_cast<float*>(p + off);             off += aero_rowscale(d) ? aero_align_up(Tn * sizeof(float), 256) : 0;
+  f.row_scale = reinterpret_cast<float*>(p + off);             off += aero_align_up(Tn * sizeof(float), 256);
   f.dz = reinterpret_cast<__nv_bfloat16*>(p + off);
   f.head_bytes = off;
   return f;
@@ -260,7 +345,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
     if ((rc = aero_make_tmap_dz(ctx, &tmDZ_mn, f.dz, (uint64_t)tpc, nblk, 64, gemmbwd::BM / 64))) return rc;
     if ((rc = aero_make_tmap_blocked(ctx, &tmW_mn, W, V, d, d, 64, gemmbwd::BN / 64))) return rc;
     if ((rc = aero_make_tmap_blocked(ctx, &tmH_mn, H, T, d, d, 64, gemmbwd::BN / 64))) return rc;
-    const bool rowscale = aero_rowscale(d);
+    const bool rowscale = aero_rowscale(ctx);
     __nv_bfloat16* Hs = f.dz + (size_t)tpc * lmhead::BM * (size_t)ldz;      // after the chunk's p~ block
     CUtensorMap tmHs_mn;
     if (rowscale && (rc = aero_make_tmap_blocked(ctx, &tmHs_mn, Hs, tpc * lmhead::BM, d, d, 64, gemmbwd::BN / 64))) return rc;
@@ -272,7 +357,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
     AERO_CUDA_TRY(cudaFuncSetAttribute(k_dh, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::SMEM_BYTES));
     AERO_CUDA_TRY(cudaFuncSetAttribute(k_dw, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::SMEM_BYTES));
 
-    const int vs = aero_vsplit(d);
+    const int vs = aero_vsplit(ctx, d);
     const int nvt = (V + lmhead::BN - 1) / lmhead::BN;
     const int n_nt = (d + gemmbwd::BN - 1) / gemmbwd::BN;
     const long long dw_units = (long long)((V + gemmbwd::BM - 1) / gemmbwd::BM) * n_nt;
@@ -291,14 +376,15 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
       p.tile_row = f.tiles.tile_row; p.tile_valid = f.tiles.tile_valid; p.n_tiles = f.tiles.n_tiles;
       p.tile_begin = (int)begin; p.tile_end = (int)(begin + tpc);
       p.y = y; p.status = ctx->d_status;
-      p.vsplit = vs; p.xstate = f.xstate; p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync();
+      p.vsplit = vs; p.xstate = f.xstate; p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync(ctx);
       p.old_logp = old_logp; p.cs = cs; p.adv = adv; p.w = w;
       p.ref_logp = ref_logp; p.kl_beta = ref_logp ? kl_beta : 0.f;
       p.clip_lo = cfg->clip_lo; p.clip_hi = cfg->clip_hi;
       p.logp = logp; p.lse_out = lse; p.g_out = g; p.partials = f.partials;
       p.shift_out = f.shift; p.dz = f.dz; p.ldz = ldz;
       p.common_shift = rowscale && vs > 1 ? 1 : 0;
-      AERO_CUDA_TRY(cudaMemsetAsync(f.sync_ctr, 0, 256, ctx->stream));
+      p.range_rows = f.range_rows; p.range_count = f.range_count; p.range_cap = kRangeCap;
+      AERO_CUDA_TRY(cudaMemsetAsync(f.sync_ctr, 0, 512, ctx->stream));      // pacing counter and the range list's count
       const long long pairs = (tpc + 1) / 2 * vs;
       const int grid = 2 * (int)(pairs < max_pairs ? pairs : max_pairs);
       const bool timed = ctx->timing && ctx->n_timed < 256;
@@ -323,17 +409,25 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
         RowArgs ra;
         ra.dz = f.dz; ra.nblk = (int)nblk; ra.tile_row = f.tiles.tile_row; ra.tile_valid = f.tiles.tile_valid;
         ra.n_tiles = f.tiles.n_tiles; ra.tile_begin = (int)begin; ra.tile_end = (int)(begin + tpc);
-        ra.T = T; ra.d = d; ra.y = y; ra.lse = lse; ra.g = g; ra.shift = f.shift; ra.grad_scale = grad_scale;
+        ra.T = T; ra.d = d; ra.y = y; ra.lse = lse; ra.g = g; ra.logp = logp; ra.shift = f.shift; ra.grad_scale = grad_scale;
         ra.H = static_cast<const __nv_bfloat16*>(H); ra.Hs = Hs; ra.row_scale = f.row_scale;
         row_factors_kernel<<<(unsigned)(tpc * 16), 256, 0, ctx->stream>>>(ra);
       } else {
         ScaleArgs sa;
         sa.dz = f.dz; sa.nblk = (int)nblk; sa.tile_row = f.tiles.tile_row; sa.tile_valid = f.tiles.tile_valid;
         sa.n_tiles = f.tiles.n_tiles; sa.tile_begin = (int)begin; sa.tile_end = (int)(begin + tpc);
-        sa.T = T; sa.V = V; sa.vsplit = vs; sa.nvt = nvt; sa.y = y; sa.lse = lse; sa.g = g; sa.shift = f.shift;
+        sa.T = T; sa.V = V; sa.vsplit = vs; sa.nvt = nvt; sa.y = y; sa.lse = lse; sa.g = g; sa.logp = logp; sa.shift = f.shift;
         sa.grad_scale = grad_scale;
         scale_dz_kernel<<<dim3((unsigned)((nblk + kBlocksPerCta - 1) / kBlocksPerCta), (unsigned)tpc), 256, 0, ctx->stream>>>(sa);
-
+      }
+      {
+        RangeArgs fa;
+        fa.rows = f.range_rows; fa.count = f.range_count; fa.cap = kRangeCap; fa.dz = f.dz; fa.nblk = (int)nblk;
+        fa.tile_row = f.tiles.tile_row; fa.tile_begin = (int)begin; fa.T = T; fa.d = d; fa.V = V; fa.y = y;
+        fa.lse = lse; fa.g = g; fa.logp = logp; fa.grad_scale = grad_scale;
+        fa.H = static_cast<const __nv_bfloat16*>(H); fa.W = static_cast<const __nv_bfloat16*>(W);
+        fa.Hs = rowscale ? Hs : nullptr; fa.row_scale = rowscale ? f.row_scale : nullptr;
+        range_fix_kernel<<<2 * ctx->sm_count, 256, 0, ctx->stream>>>(fa);
       }
 
       gemmbwd::Params gp = {};
@@ -348,7 +442,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
              ctx->stream>>>(tmDZ_k, tmW_mn, gp);
       k_dw<<<(int)(dw_units < ctx->sm_count ? dw_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
              ctx->stream>>>(tmDZ_mn, rowscale ? tmHs_mn : tmH_mn, gp);
-      ctx->launches += 3;
+      ctx->launches += 4;
       AERO_CUDA_TRY(cudaGetLastError());
     }
   }

@@ -79,8 +79,7 @@ int aero_grpo_step_host(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R
   // chunk size: whatever the given workspace affords beyond the fixed part
   const size_t fixed = carve_step(nullptr, P, R, T, d, V, 128, cfg->dtype).total;
   if (workspace_bytes < fixed) return AERO_ERR_WORKSPACE;
-  const size_t per_tile = cfg->dtype == AERO_FP32 ? 1 : (size_t)128 * ((((size_t)V + 63) / 64 * 64) * 2 +
-                                                                        (aero_rowscale(d) ? (size_t)d * 2 : 0));
+  const size_t per_tile = cfg->dtype == AERO_FP32 ? 1 : (size_t)128 * ((((size_t)V + 63) / 64 * 64) * 2 + (size_t)d * 2);
   int64_t chunk_tokens = 128 + (int64_t)((workspace_bytes - fixed) / per_tile) * 128;
   StepWs s = carve_step(workspace, P, R, T, d, V, chunk_tokens, cfg->dtype);
   while (s.total > workspace_bytes && chunk_tokens > 128) {     // alignment slack

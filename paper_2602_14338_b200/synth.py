@@ -112,14 +112,18 @@ def make_tensors(wl: Workload, T: int, device="cpu"):
     return H, W
 
 
-def peak_hidden(H, W, y, strength: float):
-    """Overwrite H so that logits are peaked at the target: H_t = strength * W[y_t]/|W[y_t]| + 0.25 * H_t.
-    Used for parity cases in which the softmax part of the gradient is not negligible."""
+def peak_hidden(H, W, y, strength):
+    """Overwrite H so that logits are peaked at the target: H_t = strength_t * W[y_t]/|W[y_t]| + 0.25 * H_t
+    (strength a number, or one value per row).  Used for parity cases in which the softmax part of the
+    gradient is not negligible, and for rows whose target probability is close to 1."""
     import torch
 
     Wy = W[torch.as_tensor(y, device=W.device).long()].float()
     Wy = Wy / Wy.norm(dim=1, keepdim=True).clamp_min(1e-12)
-    return (strength * Wy + 0.25 * H.float()).to(H.dtype)
+    s = torch.as_tensor(strength, dtype=torch.float32, device=W.device)
+    if s.ndim == 1:
+        s = s[:, None]
+    return (s * Wy + 0.25 * H.float()).to(H.dtype)
 
 
 def success_thresholds(P: int, beta_a: float, beta_b: float, seed: int) -> np.ndarray:

@@ -93,7 +93,7 @@ class Batch:
         self.st = st
         self.P, self.R, self.T = len(st.go) - 1, len(st.reward), int(st.cs[-1])
         H, W = synth.make_tensors(wl, self.T, device="cpu")
-        if peak > 0:
+        if np.ndim(peak) > 0 or peak > 0:          # a number, or one strength per token row
             H = synth.peak_hidden(H, W, st.y, peak)
         self.H_t, self.W_t = H, W
         self.H = H.double().numpy()

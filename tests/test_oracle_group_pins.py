@@ -247,6 +247,35 @@ def test_zero_accuracy_ratio_metric():
     assert list(out["counters"][3:7]) == [2, 0, 1, 1]
 
 
+def test_group_metrics_hand_values():
+    # Three prompts with token lengths chosen by hand; AERO curation with k = 1, Bayesian uniform groups keep 2.
+    #   prompt 0: rewards 1 0 0 0 (lengths 2 4 6 8), keys put rollout 3 first among the incorrect ones
+    #             -> keep rollouts 0 and 3, advantages +1 and -1
+    #   prompt 1: rewards 0 0 0 (lengths 1 1 1), flat prior -> u~ = 1/5, keep the two smallest keys (1 and 2),
+    #             advantage (0 - 0.2)/sqrt(0.2 * 0.8) = -0.5 each
+    #   prompt 2: rewards 1 1 0 (lengths 3 3 3): c = 2 of 3 is not low-success -> keep all;
+    #             mean 2/3, population std sqrt(2)/3 -> advantages +1/sqrt(2), +1/sqrt(2), -sqrt(2)
+    go = np.array([0, 4, 7, 10], np.int32)
+    reward = np.array([1, 0, 0, 0, 0, 0, 0, 1, 1, 0], np.float32)
+    lens = np.array([2, 4, 6, 8, 1, 1, 1, 3, 3, 3])
+    cs = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    key = np.array([9, 7, 8, 1, 5, 2, 3, 0, 0, 0], np.uint32)
+    cfg = O.Cfg(uniform_policy=O.UNIFORM_BAYES, rejection=1, n_keep_uniform=2, eps_std=0.0)
+    out = O.group_stats(cfg, go, reward, cs, key=key)
+    assert list(out["keep"]) == [1, 0, 0, 1, 0, 1, 1, 1, 1, 1]
+    abs_adv = [1.0, 1.0, 0.5, 0.5, 1 / math.sqrt(2), 1 / math.sqrt(2), math.sqrt(2)]
+    assert out["metrics"][1] == pytest.approx(sum(abs_adv) / 7, rel=1e-12)       # mean |advantage| over kept rollouts
+    assert out["metrics"][2] == pytest.approx(7 / 10, rel=1e-12)                 # kept rollouts / present rollouts
+    assert out["metrics"][3] == pytest.approx((2 + 8 + 1 + 1 + 9) / 32, rel=1e-12)   # kept tokens / present tokens
+    assert out["metrics"][0] == pytest.approx(1 / 3)
+    # absent rollouts leave the denominators of both fractions
+    keep_in = np.array([1, 1, 1, 1, 1, 1, 1, 1, 1, 0], np.uint8)                 # prompt 2 becomes all-correct
+    out = O.group_stats(cfg, go, reward, cs, key=key, keep_in=keep_in)
+    assert int(out["keep"].sum()) == 6
+    assert out["metrics"][2] == pytest.approx(6 / 9, rel=1e-12)
+    assert out["metrics"][3] == pytest.approx((2 + 8 + 1 + 1 + 6) / 29, rel=1e-12)
+
+
 def test_balance_factor_lemma():
     # Lemma 4.2: c*m/(c+m)^2 is maximal iff m = c; it equals the variance of the kept group.
     for c in range(1, 6):
@@ -271,6 +300,22 @@ def test_rescue_threshold_extends_low_set():
     assert out["keep"].sum() == 10
 
 
+def test_rescue_threshold_decides_between_the_two_rejection_rules():
+    # For k >= 1 a group with 2c >= n keeps all its incorrect rollouts under the low-success rule anyway
+    # (m = min(k c, n - c) = n - c), so the threshold S can only matter where another rule would apply
+    # instead: with the high-success down-sampling on, a group of 5 correct / 3 incorrect is cut to 3 + 3,
+    # unless S puts it into the low-success set (5 * 8 <= 5 * 8), where it keeps all 8.
+    go, reward, cs = _one_group(8, 5)
+    cut = O.group_stats(O.Cfg(rejection=1, reject_high=1, rescue_S=4, n_explore=8), go, reward, cs)
+    assert cut["keep"].sum() == 6                     # 5 * 8 > 4 * 8: not in the low-success set
+    low = O.group_stats(O.Cfg(rejection=1, reject_high=1, rescue_S=5, n_explore=8), go, reward, cs)
+    assert low["keep"].sum() == 8
+    # inside the range the paper gives (S <= n_explore / 2) the threshold adds only groups with u = 1/2 exactly
+    go, reward, cs = _one_group(8, 4)
+    at_half = O.group_stats(O.Cfg(rejection=1, reject_high=1, rescue_S=4, n_explore=8), go, reward, cs)
+    assert at_half["keep"].sum() == 8
+
+
 def test_empty_group_and_empty_batch():
     go = np.array([0, 0, 3], np.int32)
     reward = np.array([1, 0, 0], np.float32)
@@ -283,8 +328,8 @@ def test_empty_group_and_empty_batch():
 
 
 def test_high_success_downsampling_brute_force():
-    """reject_high: which correct rollouts survive, against a plain sort; low-success groups and
-    uniform groups are untouched by the switch."""
+    """reject_high: which correct rollouts survive, by counting predecessors in (key, index) order;
+    low-success groups and uniform groups are untouched by the switch."""
     rng = np.random.default_rng(11)
     for _ in range(40):
         n = int(rng.integers(2, 14))
@@ -302,8 +347,11 @@ def test_high_success_downsampling_brute_force():
             assert np.array_equal(out["keep"], base["keep"])
             continue
         m = min(k * (n - c), c)
-        corr = sorted([i for i in range(n) if reward[i] > 0.5], key=lambda i: (int(key[i]), i))[:m]
-        expect = np.zeros(n, np.uint8)
-        expect[corr] = 1
-        expect[reward < 0.5] = 1
-        assert np.array_equal(out["keep"], expect)
+        for i in range(n):
+            if reward[i] < 0.5:
+                assert out["keep"][i] == 1            # every incorrect rollout stays
+            else:
+                # counted, not sorted: kept iff fewer than m correct rollouts precede it in (key, index) order
+                before = sum(1 for j in range(n) if reward[j] > 0.5 and
+                             (key[j] < key[i] or (key[j] == key[i] and j < i)))
+                assert out["keep"][i] == (1 if before < m else 0)

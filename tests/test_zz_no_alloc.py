@@ -38,26 +38,36 @@ def _compare(a, b, P, R):
 def test_static_scratch_matches_workspace_entry_point_twice():
     ctx = B.Context(0)
     cases = [
-        (synth.scaled(synth.WORKLOADS[3], P=2000, seed=501), dict(uniform_policy=O.UNIFORM_BAYES, rejection=1)),
-        (synth.scaled(synth.WORKLOADS[1], P=37, seed=502), dict()),      # smaller: stale scratch beyond it
+        (synth.scaled(synth.WORKLOADS[3], P=2000, seed=501), dict(uniform_policy=O.UNIFORM_BAYES, rejection=1), False),
+        (synth.scaled(synth.WORKLOADS[1], P=37, seed=502), dict(), False),      # smaller: stale scratch beyond it
+        # per-prompt kept counts go through the array only under the sequence mean; absent rollouts too
+        (synth.scaled(synth.WORKLOADS[3], P=900, seed=503),
+         dict(uniform_policy=O.UNIFORM_BAYES, rejection=1, agg=O.AGG_SEQ_MEAN), True),
     ]
-    for wl, mode in cases:
+    for n_call, (wl, mode, with_keep_in) in enumerate(cases):
         st = synth.make_structure(wl)
         P, R = len(st.go) - 1, len(st.reward)
         cfg = TL.lib_cfg(O.Cfg(seed=wl.seed, **mode), "bf16")
         gi = TL.group_inputs_device(st)
-        ref = ctx.group_stats(cfg, gi["go"], gi["reward"], gi["cs"], key=gi["key"],
+        keep_in_h = (np.random.default_rng(9).random(R) < 0.85).astype(np.uint8) if with_keep_in else None
+        keep_in = TL.dev(keep_in_h) if with_keep_in else None
+        ref = ctx.group_stats(cfg, gi["go"], gi["reward"], gi["cs"], key=gi["key"], keep_in=keep_in,
                               alpha_in=gi["alpha"], beta_in=gi["beta"])
         out = _outputs(P, R)
         torch.cuda.synchronize()
-        before = torch.cuda.memory_allocated()
-        ctx.group_stats_static(cfg, gi["go"], gi["reward"], gi["cs"], out, key=gi["key"],
+        # free device memory as the driver reports it (it sees every allocation of the process, not only
+        # torch's); the first call on a device may load the kernels' module, so the check starts with the second
+        free_before = torch.cuda.mem_get_info()[0]
+        held_before = torch.cuda.memory_allocated()
+        ctx.group_stats_static(cfg, gi["go"], gi["reward"], gi["cs"], out, key=gi["key"], keep_in=keep_in,
                                alpha_in=gi["alpha"], beta_in=gi["beta"])
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before          # the binding allocated nothing either
+        assert torch.cuda.memory_allocated() == held_before      # the binding allocated nothing either
+        if n_call > 0:
+            assert torch.cuda.mem_get_info()[0] >= free_before
         _compare(out, ref, P, R)
         # and both agree with the oracle on what is exact
-        oref = O.group_stats(O.Cfg(seed=wl.seed, **mode), st.go, st.reward, st.cs, key=st.key,
+        oref = O.group_stats(O.Cfg(seed=wl.seed, **mode), st.go, st.reward, st.cs, key=st.key, keep_in=keep_in_h,
                              alpha_in=st.alpha, beta_in=st.beta)
         assert np.array_equal(out["keep"][:R].cpu().numpy(), oref["keep"])
         assert np.array_equal(out["counters"].cpu().numpy(), oref["counters"])
