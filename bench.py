@@ -56,6 +56,8 @@ def parse_args():
     ap.add_argument("--only-group-leg", action="store_true",
                     help="run only the large-input group-stage measurement (for profiling that stage alone)")
     ap.add_argument("--only-main", action="store_true", help="only the timed steps of the headline workload")
+    ap.add_argument("--gemm-sync", type=int, default=-1,
+                    help="meeting points per unit of the backward products' producers (aero_set_tuning); -1: the library's default")
     return ap.parse_args()
 
 
@@ -119,20 +121,22 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- oracle legs
 def oracle_sample(wl, st, n_tokens):
-    """The first n_tokens token rows of the workload as one group (rollouts truncated at the
-    sample boundary), as fp64 arrays for the oracle.  Inputs only; no result of the CUDA path."""
+    """A bounded sample of the workload for the oracle: its first rollouts (up to 8), each cut to its
+    first n_tokens / 8 token rows, as one group, in fp64.  Inputs only; no result of the CUDA path."""
     from paper_2602_14338_b200 import synth
 
-    n_tokens = int(min(n_tokens, st.cs[-1]))
-    R = int(np.searchsorted(st.cs, n_tokens, side="left"))
-    cs = np.minimum(st.cs[:R + 1], n_tokens).astype(np.int64)
-    go = np.array([0, R], np.int32)
-    reward = st.reward[:R].copy()
-    if R >= 2:                                   # make sure the sample group is a mixed one
+    G = int(min(8, len(st.reward)))
+    cap = max(1, int(n_tokens) // G)
+    lens = np.minimum(st.cs[1:G + 1] - st.cs[:G], cap).astype(np.int64)
+    rows = np.concatenate([np.arange(st.cs[i], st.cs[i] + lens[i]) for i in range(G)])
+    cs = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    go = np.array([0, G], np.int32)
+    reward = st.reward[:G].copy()
+    if G >= 2:                                   # make sure the sample group is a mixed one
         reward[0], reward[1] = 1.0, 0.0
-    H, W = synth.make_tensors(wl, n_tokens, device="cpu")
-    return dict(go=go, cs=cs, reward=reward, key=st.key[:R], y=st.y[:n_tokens], noise=st.noise[:n_tokens],
-                H=H.double().numpy(), W=W.double().numpy(), T=n_tokens)
+    H, W = synth.make_tensors(wl, int(st.cs[G]), device="cpu")
+    return dict(go=go, cs=cs, reward=reward, key=st.key[:G], y=st.y[rows], noise=st.noise[rows],
+                H=H[rows].double().numpy(), W=W.double().numpy(), T=int(cs[-1]))
 
 
 def oracle_step(O, s, old):
@@ -170,8 +174,9 @@ def time_oracle(wl, st, budget_s, steps=1, warmup=0):
     for _ in range(steps):
         _, kept = oracle_step(O, s, old)
     dt = (time.perf_counter() - t0) / steps
-    sample = (f"first {s['T']} token rows of the workload as one group of {len(s['reward'])} rollouts "
-              f"({kept} kept tokens per step), full d={wl.d} and V={wl.V}, fp64 numpy")
+    sample = (f"the workload's first {len(s['reward'])} rollouts, each cut to its first {int(s['cs'][1:].max() if s['T'] else 0)} "
+              f"token rows at most, as one group: {s['T']} rows, {kept} kept tokens per step, full d={wl.d} and V={wl.V}, "
+              f"fp64 numpy")
     return kept / dt, cores, sample, dt * 1e3
 
 
@@ -306,6 +311,7 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     pk = peaks()
     ctx = B.Context(local)
+    ctx.set_tuning(gemm_sync=args.gemm_sync)
     if args.only_group_leg:
         print(json.dumps({"group_stage": group_stage_leg(ctx, pk, dev)}), flush=True)
         return

@@ -153,10 +153,11 @@ int aero_last_status(aero_ctx* ctx, uint32_t* bits);
  * by d (the default).  nsync: meeting points per unit at which the lm_head kernel's
  * producers wait for one another, 0 for none, negative for the default.  rowscale: in
  * aero_grpo_loss_fwd_bwd, 1 (or negative, the default) applies the row factors inside the
- * backward products, 0 rewrites the chunk block in a pass of its own.  The workspace sizes
- * the *_workspace_bytes functions return cover every setting.  Returns AERO_ERR_INVALID
- * for any other value. */
-int aero_set_tuning(aero_ctx* ctx, int vsplit, int nsync, int rowscale);
+ * backward products, 0 rewrites the chunk block in a pass of its own.  gemm_sync: meeting
+ * points per unit of the two backward products' producers, 0 for none, negative for the
+ * default.  The workspace sizes the *_workspace_bytes functions return cover every setting.
+ * Returns AERO_ERR_INVALID for any other value. */
+int aero_set_tuning(aero_ctx* ctx, int vsplit, int nsync, int rowscale, int gemm_sync);
 
 /* ------------------------------------------------------------------------------
  * Stage (a).  Group statistics, curation and weights (Eq. 1; Sec. 3.2; Sec. 4.2
@@ -230,8 +231,8 @@ int aero_finalize_weights(aero_ctx* ctx, const aero_cfg* cfg, int32_t R, int32_t
  * workspace at the point of the call -- a plug-in inside a host program that owns all
  * device memory, or a latency-bound loop that must not call the allocator because an
  * allocation can synchronise the whole device.  Instead of a caller workspace, the scratch
- * is a fixed array in device memory that belongs to the loaded library itself: 1,476,096
- * bytes (1.41 MiB) per GPU that loads the library, held until the process exits, sized for at most
+ * is a fixed array in device memory that belongs to the loaded library itself:
+ * AERO_STATIC_SCRATCH_BYTES (1,476,096 bytes, 1.41 MiB) per GPU that loads the library, held until the process exits, sized for at most
  * AERO_STATIC_MAX_PROMPTS prompts whatever their group sizes (R itself is not limited).
  * A batch beyond that limit returns AERO_ERR_TOO_LARGE and launches nothing.  The call,
  * and everything it calls, performs no cudaMalloc/cudaFree and uses no allocating library
@@ -242,10 +243,11 @@ int aero_finalize_weights(aero_ctx* ctx, const aero_cfg* cfg, int32_t R, int32_t
  * All calls on a device share the one array: two calls whose kernels may overlap on the
  * GPU (different streams, or different contexts of this library on one device) race on
  * it -- order them on one stream or with events.  The array keeps the previous call's
- * contents; each call writes every word before reading it.  Arguments, outputs and status bits are
- * those of aero_group_stats.
+ * contents; nothing in it has to start at zero: each call writes every word before reading it.
+ * Arguments, outputs and status bits are those of aero_group_stats.
  */
 #define AERO_STATIC_MAX_PROMPTS 65536
+#define AERO_STATIC_SCRATCH_BYTES 1476096   /* size of that array */
 
 int aero_group_stats_static(aero_ctx* ctx, const aero_cfg* cfg, int32_t P, int32_t R,
                             const int32_t* go, const float* reward, const int64_t* cs,

@@ -31,6 +31,7 @@ struct aero_ctx {
   int tune_vsplit;        // 0: by d (aero_vsplit_auto); else 1, 2 or 4 CTA pairs per pair of token tiles
   int tune_nsync;         // < 0: the default number of meeting points; 0: no pacing; else that many
   int tune_rowscale;      // < 0 or 1: row factors in the backward GEMMs; 0: the pass that rewrites the block
+  int tune_gemm_sync;     // < 0: the default number of meeting points per unit of the backward GEMMs; 0: none
 };
 
 #define AERO_CUDA_TRY(expr)                          \
@@ -133,6 +134,8 @@ static inline int aero_nsync(const aero_ctx* ctx) { return ctx->tune_nsync >= 0 
 // With several vocabulary splits this needs one shift per row for all of them
 // (lmhead::Params::common_shift).
 static inline bool aero_rowscale(const aero_ctx* ctx) { return ctx->tune_rowscale != 0; }
+// Meeting points per unit of the backward GEMMs' producers (0: none).
+static inline int aero_gemm_sync(const aero_ctx* ctx) { return ctx->tune_gemm_sync >= 0 ? ctx->tune_gemm_sync : 1; }
 size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t d, int32_t R);
 int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                 const void* H, const void* W, const int32_t* y, const float* old_logp,

@@ -47,6 +47,13 @@ struct Params {
   uint32_t* status;
   const float* row_scale;       // dH: factor of each token row, applied to the finished tile (NULL: none)
   int h_local;                  // dW: operand B holds the chunk's rows tile after tile, not all T rows
+  // Pacing: CTAs that run at the same time share operand tiles through L2 (the units of one row tile read the
+  // same dz tiles, the units of one column tile the same W or H slab), which works only while they walk the
+  // reduction dimension in step; small rate differences between SMs add up over the dozens of units a CTA
+  // processes.  The producers therefore meet `nsync` times per unit on a counter in global memory (zeroed
+  // before the launch).  The wait is short and bounded: a CTA that is not there in time is not waited for.
+  unsigned int* sync_ctr;
+  int nsync;
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -89,9 +96,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
       uint32_t it = 0;
       bool ok = true;
       int row_cur = 0, row_next = 0;
+      unsigned int meetings = 0;
+      const int max_units = (n_units + (int)gridDim.x - 1) / (int)gridDim.x;     // of the longest schedule
       for (int u = blockIdx.x; ok && u < n_units; u += gridDim.x) {
         const int mt = u / n_nt, nt = u % n_nt;
+        int next_meet = 0;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
+          if (p.nsync > 0 && next_meet < p.nsync && kb >= (int)((long long)next_meet * nkb / p.nsync)) {
+            ++next_meet;
+            ++meetings;
+            atomicAdd(p.sync_ctr, 1u);
+            const unsigned int target = meetings * gridDim.x;
+            const unsigned long long t0 = tc::globaltimer_ns();
+            while (*reinterpret_cast<volatile unsigned int*>(p.sync_ctr) < target) {
+              if (tc::globaltimer_ns() - t0 > 50000ull) break;        // 50 us: go on alone
+              __nanosleep(100);
+            }
+          }
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1u;
           if (!tc::mbar_wait(&ctl->empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -117,7 +138,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             tc::tma_load_3d(b_s, &tmB, 0, hrow, nt * (BN / 64), &ctl->full[s]);
           }
         }
+        // a unit with fewer slabs than meeting points still counts them all
+        if (p.nsync > 0 && next_meet < p.nsync) {
+          atomicAdd(p.sync_ctr, (unsigned)(p.nsync - next_meet));
+          meetings += (unsigned)(p.nsync - next_meet);
+        }
       }
+      // out of units: stand in for the meetings the longest schedule still has
+      if (p.nsync > 0 && meetings < (unsigned)(max_units * p.nsync))
+        atomicAdd(p.sync_ctr, (unsigned)(max_units * p.nsync) - meetings);
     }
   } else if (warp == 5) {
     // ---------------- MMA issuer ----------------

@@ -964,6 +964,7 @@ namespace {
 constexpr int32_t kStaticMaxP = AERO_STATIC_MAX_PROMPTS;
 // room for kStaticMaxP prompts in the smallest tiles there are (one prompt per warp)
 constexpr size_t kStaticBytes = workspace_bytes((size_t)kStaticMaxP, ((size_t)kStaticMaxP + kWarps - 1) / kWarps);
+static_assert(kStaticBytes == AERO_STATIC_SCRATCH_BYTES, "the header states the size of the array");
 
 static __device__ __align__(256) unsigned char g_group_scratch[kStaticBytes];
 

@@ -508,20 +508,33 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
                 v[q] = ENT ? pr * fmaf(et, z, c0) : c0 * pr;
               }
               if ((unsigned)(yt - col0) < 32u) {
+                // (the target's logit is picked out first, so that its formula is instantiated once, not per column)
                 const int sel = yt - col0;
+                float zs = 0.f;
 #pragma unroll
-                for (int q = 0; q < 32; ++q) if (q == sel) v[q] = dz_target(__uint_as_float(r[q]));
+                for (int q = 0; q < 32; ++q) if (q == sel) zs = __uint_as_float(r[q]);
+                const float tv = dz_target(zs);
+#pragma unroll
+                for (int q = 0; q < 32; ++q) if (q == sel) v[q] = tv;
               }
 #pragma unroll
               for (int q = 0; q < 32; q += 2) pk[q >> 1] = pack_bf16(v[q], v[q + 1]);
             } else {
+              float tv = 0.f;
+              if (live && (unsigned)(yt - col0) < 32u) {
+                const int sel = yt - col0;
+                float zs = 0.f;
+#pragma unroll
+                for (int q = 0; q < 32; ++q) if (q == sel) zs = __uint_as_float(r[q]);
+                tv = dz_target(zs);
+              }
 #pragma unroll
               for (int q = 0; q < 32; q += 2) {
                 const float z0 = __uint_as_float(r[q]), z1 = __uint_as_float(r[q + 1]);
                 float v0 = ex2(fmaf(z0, kLog2e, -lse2)) * (ENT ? fmaf(et, z0, c0) : c0);
                 float v1 = ex2(fmaf(z1, kLog2e, -lse2)) * (ENT ? fmaf(et, z1, c0) : c0);
-                if (col0 + q == yt) v0 = dz_target(z0);
-                if (col0 + q + 1 == yt) v1 = dz_target(z1);
+                if (col0 + q == yt) v0 = tv;
+                if (col0 + q + 1 == yt) v1 = tv;
                 if (!live || col0 + q >= p.V) v0 = 0.f;
                 if (!live || col0 + q + 1 >= p.V) v1 = 0.f;
                 pk[q >> 1] = pack_bf16(v0, v1);

@@ -108,9 +108,12 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     gp.tile_row = tiles.tile_row; gp.tile_valid = tiles.tile_valid; gp.n_tiles = tiles.n_tiles;
     gp.tile_begin = (int)begin; gp.tpc = (int)tpc;
     gp.dH = static_cast<__nv_bfloat16*>(dH); gp.dW = dW; gp.status = ctx->d_status;
+    gp.nsync = aero_gemm_sync(ctx);
+    gp.sync_ctr = sync_ctr + 4;             // (the lm_head kernel's counter comes first; all zeroed above)
     const long long dh_units = tpc * n_nt;
     k_dh<<<(int)(dh_units < ctx->sm_count ? dh_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
            ctx->stream>>>(tmDZ_k, tmW_mn, gp);
+    gp.sync_ctr = sync_ctr + 8;
     k_dw<<<(int)(dw_units < ctx->sm_count ? dw_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
            ctx->stream>>>(tmDZ_mn, tmH_mn, gp);
     ctx->launches += 3;

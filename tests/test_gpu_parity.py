@@ -413,8 +413,10 @@ def test_forward_and_backward_in_one_call(ctx, name):
     edge = (np.abs(rho - (1 + batch.ocfg.clip_hi)) < 1e-3) | (np.abs(rho - (1 - batch.ocfg.clip_lo)) < 1e-3)
     # (row factors in the backward GEMMs, with two splits sharing one shift per row; rowscale 0: the pass
     # that rewrites the block, with a shift per split)
-    for chunk, vsplit, rowscale in ((None, 0, -1), (128, 0, -1), (128, 0, 0), (128, 2, -1), (128, 2, 0)):
-        ctx.set_tuning(vsplit=vsplit, rowscale=rowscale)
+    # (the last entries also pace the producers of the backward products: same results, another schedule)
+    for chunk, vsplit, rowscale, gsync in ((None, 0, -1, -1), (128, 0, -1, -1), (128, 0, 0, 3), (128, 2, -1, 2), (128, 2, 0, -1),
+                                           (None, 0, -1, 5)):
+        ctx.set_tuning(vsplit=vsplit, rowscale=rowscale, gemm_sync=gsync)
         try:
             ws = None
             if chunk:
