@@ -148,16 +148,20 @@ int aero_set_stream(aero_ctx* ctx, void* cuda_stream);
 int aero_last_status(aero_ctx* ctx, uint32_t* bits);
 
 /* Tuning hook (no passage of the paper: it only selects between equivalent schedules of
- * stage (b); results agree within rounding).  vsplit: CTA pairs that share a pair of token
- * tiles and split the vocabulary between them, 1, 2 or 4, or 0 to let the library choose
- * by d (the default).  nsync: meeting points per unit at which the lm_head kernel's
- * producers wait for one another, 0 for none, negative for the default.  rowscale: in
- * aero_grpo_loss_fwd_bwd, 1 (or negative, the default) applies the row factors inside the
- * backward products, 0 rewrites the chunk block in a pass of its own.  gemm_sync: meeting
- * points per unit of the two backward products' producers, 0 for none, negative for the
- * default.  The workspace sizes the *_workspace_bytes functions return cover every setting.
- * Returns AERO_ERR_INVALID for any other value. */
-int aero_set_tuning(aero_ctx* ctx, int vsplit, int nsync, int rowscale, int gemm_sync);
+ * stage (b); results agree within rounding).  One setting per call, by name; a negative value
+ * restores the library's own choice:
+ *   "vsplit"     CTA pairs that share a pair of token tiles and split the vocabulary between
+ *                them: 1, 2 or 4; 0 (the default) lets the library choose by d.
+ *   "nsync"      meeting points per unit at which the lm_head kernel's producers wait for one
+ *                another (bounded); 0 for none.
+ *   "rowscale"   aero_grpo_loss_fwd_bwd: 1 applies the row factors inside the backward products
+ *                (the default), 0 rewrites the chunk block in a pass of its own.
+ *   "gemm_sync"  meeting points per unit of the two backward products' producers; 0 for none.
+ *   "gemm_pairs" 1: the two backward products run on CTA pairs (units of 256 rows); 0: on
+ *                single CTAs; by default pairs for d > 2048.
+ * The workspace sizes the *_workspace_bytes functions return cover every setting.  Returns
+ * AERO_ERR_INVALID for an unknown name or a value outside the ones listed. */
+int aero_set_tuning(aero_ctx* ctx, const char* name, int value);
 
 /* ------------------------------------------------------------------------------
  * Stage (a).  Group statistics, curation and weights (Eq. 1; Sec. 3.2; Sec. 4.2

@@ -75,7 +75,7 @@ def load_library():
     lib.aero_create.argtypes = [C.POINTER(vp), C.c_int, vp]
     lib.aero_destroy.argtypes = [vp]
     lib.aero_set_stream.argtypes = [vp, vp]
-    lib.aero_set_tuning.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.c_int]
+    lib.aero_set_tuning.argtypes = [vp, C.c_char_p, C.c_int]
     lib.aero_selftest_bounded_wait.argtypes = [vp, C.c_uint32]
     lib.aero_last_status.argtypes = [vp, C.POINTER(C.c_uint32)]
     lib.aero_group_workspace_bytes.restype = sz
@@ -195,9 +195,11 @@ class Context:
         self.stream = stream
         _check(self.lib.aero_set_stream(self.h, C.c_void_p(stream.cuda_stream)), "aero_set_stream")
 
-    def set_tuning(self, vsplit=0, nsync=-1, rowscale=-1, gemm_sync=-1):
-        """aero_set_tuning: schedule choices of stage (b); the defaults let the library decide."""
-        _check(self.lib.aero_set_tuning(self.h, int(vsplit), int(nsync), int(rowscale), int(gemm_sync)), "aero_set_tuning")
+    def set_tuning(self, vsplit=0, nsync=-1, rowscale=-1, gemm_sync=-1, gemm_pairs=-1):
+        """aero_set_tuning for every setting: schedule choices of stage (b); the defaults let the library decide."""
+        for name, value in (("vsplit", vsplit), ("nsync", nsync), ("rowscale", rowscale), ("gemm_sync", gemm_sync),
+                            ("gemm_pairs", gemm_pairs)):
+            _check(self.lib.aero_set_tuning(self.h, name.encode(), int(value)), f"aero_set_tuning({name})")
 
     def selftest_bounded_wait(self, limit_us=1000):
         """aero_selftest_bounded_wait: a wait that cannot complete must end with AERO_ST_TIMEOUT."""

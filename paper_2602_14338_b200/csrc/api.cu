@@ -3,6 +3,7 @@
 #include "common.cuh"
 
 #include <new>
+#include <string>
 
 #include <nvtx3/nvToolsExt.h>
 
@@ -83,6 +84,7 @@ int aero_create(aero_ctx** out, int device, void* cuda_stream) {
   ctx->tune_nsync = -1;
   ctx->tune_rowscale = -1;
   ctx->tune_gemm_sync = -1;
+  ctx->tune_gemm_pairs = -1;
   for (int i = 0; i < 256; ++i) { ctx->ev0[i] = nullptr; ctx->ev1[i] = nullptr; }
   cudaDeviceProp prop;
   if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return AERO_ERR_CUDA; }
@@ -140,14 +142,25 @@ int aero_set_stream(aero_ctx* ctx, void* cuda_stream) {
   return AERO_OK;
 }
 
-int aero_set_tuning(aero_ctx* ctx, int vsplit, int nsync, int rowscale, int gemm_sync) {
-  if (!ctx) return AERO_ERR_INVALID;
-  if (vsplit != 0 && vsplit != 1 && vsplit != 2 && vsplit != 4) return AERO_ERR_INVALID;
-  if (nsync > 4096 || gemm_sync > 4096) return AERO_ERR_INVALID;
-  ctx->tune_vsplit = vsplit;
-  ctx->tune_nsync = nsync < 0 ? -1 : nsync;
-  ctx->tune_rowscale = rowscale < 0 ? -1 : (rowscale ? 1 : 0);
-  ctx->tune_gemm_sync = gemm_sync < 0 ? -1 : gemm_sync;
+int aero_set_tuning(aero_ctx* ctx, const char* name, int value) {
+  if (!ctx || !name) return AERO_ERR_INVALID;
+  const std::string n(name);
+  if (n == "vsplit") {
+    if (value != 0 && value != 1 && value != 2 && value != 4) return AERO_ERR_INVALID;
+    ctx->tune_vsplit = value;
+  } else if (n == "nsync") {
+    if (value > 4096) return AERO_ERR_INVALID;
+    ctx->tune_nsync = value < 0 ? -1 : value;
+  } else if (n == "rowscale") {
+    ctx->tune_rowscale = value < 0 ? -1 : (value ? 1 : 0);
+  } else if (n == "gemm_sync") {
+    if (value > 4096) return AERO_ERR_INVALID;
+    ctx->tune_gemm_sync = value < 0 ? -1 : value;
+  } else if (n == "gemm_pairs") {
+    ctx->tune_gemm_pairs = value < 0 ? -1 : (value ? 1 : 0);
+  } else {
+    return AERO_ERR_INVALID;
+  }
   return AERO_OK;
 }
 

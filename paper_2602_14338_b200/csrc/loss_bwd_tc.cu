@@ -73,6 +73,13 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
   if ((rc = aero_make_tmap_blocked(ctx, &tmW_mn, W, V, d, d, 64, gemmbwd::BN / 64))) return rc;
   if ((rc = aero_make_tmap_dz(ctx, &tmDZ_mn, dz, (uint64_t)tpc, (uint64_t)(ldz / 64), 64, gemmbwd::BM / 64))) return rc;
   if ((rc = aero_make_tmap_blocked(ctx, &tmH_mn, H, T, d, d, 64, gemmbwd::BN / 64))) return rc;
+  // CTA pairs: each CTA stages half of the B slab's columns
+  const bool pairs = aero_gemm_pairs(ctx, d);
+  CUtensorMap tmW_mn2, tmH_mn2;
+  if (pairs) {
+    if ((rc = aero_make_tmap_blocked(ctx, &tmW_mn2, W, V, d, d, 64, gemmbwd::PBNH / 64))) return rc;
+    if ((rc = aero_make_tmap_blocked(ctx, &tmH_mn2, H, T, d, d, 64, gemmbwd::PBNH / 64))) return rc;
+  }
   // store view of the dz block for the lm_head kernel's epilogue: 32 rows x 64 columns per copy
   CUtensorMap tmDZ_st;
   if ((rc = aero_make_tmap_dz(ctx, &tmDZ_st, dz, (uint64_t)tpc, (uint64_t)(ldz / 64), 32, 1))) return rc;
@@ -84,6 +91,12 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
   AERO_CUDA_TRY(cudaFuncSetAttribute(k_dz, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lmhead::SMEM_BYTES));
   AERO_CUDA_TRY(cudaFuncSetAttribute(k_dh, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::SMEM_BYTES));
   AERO_CUDA_TRY(cudaFuncSetAttribute(k_dw, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::SMEM_BYTES));
+  auto k_dh2 = gemmbwd::gemm_pair_kernel<gemmbwd::KIND_DH>;
+  auto k_dw2 = gemmbwd::gemm_pair_kernel<gemmbwd::KIND_DW>;
+  if (pairs) {
+    AERO_CUDA_TRY(cudaFuncSetAttribute(k_dh2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::PSMEM_BYTES));
+    AERO_CUDA_TRY(cudaFuncSetAttribute(k_dw2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::PSMEM_BYTES));
+  }
 
   const int n_nt = (d + gemmbwd::BN - 1) / gemmbwd::BN;
   const long long dw_units = (long long)((V + gemmbwd::BM - 1) / gemmbwd::BM) * n_nt;
@@ -111,11 +124,20 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     gp.nsync = aero_gemm_sync(ctx);
     gp.sync_ctr = sync_ctr + 4;             // (the lm_head kernel's counter comes first; all zeroed above)
     const long long dh_units = tpc * n_nt;
-    k_dh<<<(int)(dh_units < ctx->sm_count ? dh_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
-           ctx->stream>>>(tmDZ_k, tmW_mn, gp);
-    gp.sync_ctr = sync_ctr + 8;
-    k_dw<<<(int)(dw_units < ctx->sm_count ? dw_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
-           ctx->stream>>>(tmDZ_mn, tmH_mn, gp);
+    if (pairs) {
+      const long long dh_pu = (tpc + 1) / 2 * n_nt, dw_pu = ((long long)((V + gemmbwd::BM - 1) / gemmbwd::BM) + 1) / 2 * n_nt;
+      k_dh2<<<2 * (int)(dh_pu < max_pairs ? dh_pu : max_pairs), gemmbwd::THREADS, gemmbwd::PSMEM_BYTES, ctx->stream>>>(
+          tmDZ_k, tmW_mn2, gp);
+      gp.sync_ctr = sync_ctr + 8;
+      k_dw2<<<2 * (int)(dw_pu < max_pairs ? dw_pu : max_pairs), gemmbwd::THREADS, gemmbwd::PSMEM_BYTES, ctx->stream>>>(
+          tmDZ_mn, tmH_mn2, gp);
+    } else {
+      k_dh<<<(int)(dh_units < ctx->sm_count ? dh_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
+             ctx->stream>>>(tmDZ_k, tmW_mn, gp);
+      gp.sync_ctr = sync_ctr + 8;
+      k_dw<<<(int)(dw_units < ctx->sm_count ? dw_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
+             ctx->stream>>>(tmDZ_mn, tmH_mn, gp);
+    }
     ctx->launches += 3;
     AERO_CUDA_TRY(cudaGetLastError());
   }

@@ -349,6 +349,15 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
     __nv_bfloat16* Hs = f.dz + (size_t)tpc * lmhead::BM * (size_t)ldz;      // after the chunk's p~ block
     CUtensorMap tmHs_mn;
     if (rowscale && (rc = aero_make_tmap_blocked(ctx, &tmHs_mn, Hs, tpc * lmhead::BM, d, d, 64, gemmbwd::BN / 64))) return rc;
+    // CTA pairs: each CTA stages half of the B slab's columns
+    const bool gemm_pairs = aero_gemm_pairs(ctx, d);
+    CUtensorMap tmW_mn2, tmB_dw2;
+    if (gemm_pairs) {
+      if ((rc = aero_make_tmap_blocked(ctx, &tmW_mn2, W, V, d, d, 64, gemmbwd::PBNH / 64))) return rc;
+      if (rowscale) rc = aero_make_tmap_blocked(ctx, &tmB_dw2, Hs, tpc * lmhead::BM, d, d, 64, gemmbwd::PBNH / 64);
+      else rc = aero_make_tmap_blocked(ctx, &tmB_dw2, H, T, d, d, 64, gemmbwd::PBNH / 64);
+      if (rc) return rc;
+    }
 
     auto k_fwd = lmhead::lmhead_kernel<lmhead::MODE_FWD_P>;
     auto k_dh = gemmbwd::gemm_kernel<gemmbwd::KIND_DH>;
@@ -356,6 +365,12 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
     AERO_CUDA_TRY(cudaFuncSetAttribute(k_fwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lmhead::SMEM_BYTES));
     AERO_CUDA_TRY(cudaFuncSetAttribute(k_dh, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::SMEM_BYTES));
     AERO_CUDA_TRY(cudaFuncSetAttribute(k_dw, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::SMEM_BYTES));
+    auto k_dh2 = gemmbwd::gemm_pair_kernel<gemmbwd::KIND_DH>;
+    auto k_dw2 = gemmbwd::gemm_pair_kernel<gemmbwd::KIND_DW>;
+    if (gemm_pairs) {
+      AERO_CUDA_TRY(cudaFuncSetAttribute(k_dh2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::PSMEM_BYTES));
+      AERO_CUDA_TRY(cudaFuncSetAttribute(k_dw2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)gemmbwd::PSMEM_BYTES));
+    }
 
     const int vs = aero_vsplit(ctx, d);
     const int nvt = (V + lmhead::BN - 1) / lmhead::BN;
@@ -440,11 +455,20 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
       gp.nsync = aero_gemm_sync(ctx);
       gp.sync_ctr = f.sync_ctr + 4;           // (the lm_head kernel's counter comes first; all zeroed above)
       const long long dh_units = tpc * n_nt;
-      k_dh<<<(int)(dh_units < ctx->sm_count ? dh_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
-             ctx->stream>>>(tmDZ_k, tmW_mn, gp);
-      gp.sync_ctr = f.sync_ctr + 8;
-      k_dw<<<(int)(dw_units < ctx->sm_count ? dw_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
-             ctx->stream>>>(tmDZ_mn, rowscale ? tmHs_mn : tmH_mn, gp);
+      if (gemm_pairs) {
+        const long long dh_pu = (tpc + 1) / 2 * n_nt, dw_pu = ((long long)((V + gemmbwd::BM - 1) / gemmbwd::BM) + 1) / 2 * n_nt;
+        k_dh2<<<2 * (int)(dh_pu < max_pairs ? dh_pu : max_pairs), gemmbwd::THREADS, gemmbwd::PSMEM_BYTES, ctx->stream>>>(
+            tmDZ_k, tmW_mn2, gp);
+        gp.sync_ctr = f.sync_ctr + 8;
+        k_dw2<<<2 * (int)(dw_pu < max_pairs ? dw_pu : max_pairs), gemmbwd::THREADS, gemmbwd::PSMEM_BYTES, ctx->stream>>>(
+            tmDZ_mn, tmB_dw2, gp);
+      } else {
+        k_dh<<<(int)(dh_units < ctx->sm_count ? dh_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
+               ctx->stream>>>(tmDZ_k, tmW_mn, gp);
+        gp.sync_ctr = f.sync_ctr + 8;
+        k_dw<<<(int)(dw_units < ctx->sm_count ? dw_units : ctx->sm_count), gemmbwd::THREADS, gemmbwd::SMEM_BYTES,
+               ctx->stream>>>(tmDZ_mn, rowscale ? tmHs_mn : tmH_mn, gp);
+      }
       ctx->launches += 4;
       AERO_CUDA_TRY(cudaGetLastError());
     }

@@ -111,9 +111,12 @@ def test_every_error_code_is_returned_for_its_argument_error(ctx):
     assert lib.aero_create(C.byref(h), 4096, None) == ERR_CUDA
     assert lib.aero_create(None, 0, None) == ERR_INVALID
     # tuning hook
-    assert lib.aero_set_tuning(ctx.h, 3, -1, -1, -1) == ERR_INVALID
-    assert lib.aero_set_tuning(ctx.h, 8, -1, -1, -1) == ERR_INVALID
-    assert lib.aero_set_tuning(ctx.h, 2, 4, 0, 2) == 0 and lib.aero_set_tuning(ctx.h, 0, -1, -1, -1) == 0
+    assert lib.aero_set_tuning(ctx.h, b"vsplit", 3) == ERR_INVALID
+    assert lib.aero_set_tuning(ctx.h, b"vsplit", 8) == ERR_INVALID
+    assert lib.aero_set_tuning(ctx.h, b"no_such_setting", 1) == ERR_INVALID
+    assert lib.aero_set_tuning(ctx.h, None, 1) == ERR_INVALID
+    assert lib.aero_set_tuning(ctx.h, b"vsplit", 2) == 0 and lib.aero_set_tuning(ctx.h, b"vsplit", 0) == 0
+    assert lib.aero_set_tuning(ctx.h, b"gemm_sync", 3) == 0 and lib.aero_set_tuning(ctx.h, b"gemm_sync", -1) == 0
     for code in (ERR_INVALID, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TOO_LARGE):
         assert lib.aero_error_string(code) not in (b"ok", b"unknown error")
     torch.cuda.synchronize()

@@ -413,10 +413,11 @@ def test_forward_and_backward_in_one_call(ctx, name):
     edge = (np.abs(rho - (1 + batch.ocfg.clip_hi)) < 1e-3) | (np.abs(rho - (1 - batch.ocfg.clip_lo)) < 1e-3)
     # (row factors in the backward GEMMs, with two splits sharing one shift per row; rowscale 0: the pass
     # that rewrites the block, with a shift per split)
-    # (the last entries also pace the producers of the backward products: same results, another schedule)
-    for chunk, vsplit, rowscale, gsync in ((None, 0, -1, -1), (128, 0, -1, -1), (128, 0, 0, 3), (128, 2, -1, 2), (128, 2, 0, -1),
-                                           (None, 0, -1, 5)):
-        ctx.set_tuning(vsplit=vsplit, rowscale=rowscale, gemm_sync=gsync)
+    # (the last entries also pace the producers of the backward products -- same results, another schedule --
+    # and run them on single CTAs instead of CTA pairs)
+    for chunk, vsplit, rowscale, gsync, pairs in ((None, 0, -1, -1, -1), (128, 0, -1, -1, -1), (128, 0, 0, 3, -1), (128, 2, -1, 2, -1),
+                                                  (128, 2, 0, -1, -1), (None, 0, -1, 5, 0), (128, 0, -1, 0, 0), (384, 2, 0, 2, 0)):
+        ctx.set_tuning(vsplit=vsplit, rowscale=rowscale, gemm_sync=gsync, gemm_pairs=pairs)
         try:
             ws = None
             if chunk:
@@ -613,6 +614,19 @@ def test_bwd_chunking_and_accumulation(ctx):
                                      ctx.bwd_workspace_bytes(batch.T, wl.d, wl.V, batch.R, 128), dtype=torch.uint8, device="cuda"))
     assert torch.equal(dH1, dH)
     assert TL.rel_l2(dW1.cpu().numpy(), dW.cpu().numpy()) < 1e-5
+    # the same products on single CTAs (the default runs them on CTA pairs: units of 256 rows, with an odd
+    # number of row tiles in the last pair of a chunk)
+    ctx.set_tuning(gemm_pairs=0)
+    try:
+        for chunk in (None, 128, 384):
+            ws = None if chunk is None else torch.empty(ctx.bwd_workspace_bytes(batch.T, wl.d, wl.V, batch.R, chunk),
+                                                        dtype=torch.uint8, device="cuda")
+            dHp, dWp = ctx.grpo_loss_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], dv["keep"], f["lse"], f["g"],
+                                         chunk_tokens=chunk, workspace=ws)
+            assert torch.equal(dHp, dH)
+            assert TL.rel_l2(dWp.cpu().numpy(), dW.cpu().numpy()) < 1e-5
+    finally:
+        ctx.set_tuning()
     # accumulate_dW adds to what is there
     dW2 = dW.clone()
     ctx.grpo_loss_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["cs"], dv["keep"], f["lse"], f["g"], dW=dW2, accumulate_dW=True)
