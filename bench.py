@@ -58,6 +58,8 @@ def parse_args():
     ap.add_argument("--only-main", action="store_true", help="only the timed steps of the headline workload")
     ap.add_argument("--gemm-sync", type=int, default=-1,
                     help="meeting points per unit of the backward products' producers (aero_set_tuning); -1: the library's default")
+    ap.add_argument("--gemm-pairs", type=int, default=-1,
+                    help="backward products on CTA pairs (1) or single CTAs (0) (aero_set_tuning); -1: the library's default")
     return ap.parse_args()
 
 
@@ -311,7 +313,7 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     pk = peaks()
     ctx = B.Context(local)
-    ctx.set_tuning(gemm_sync=args.gemm_sync)
+    ctx.set_tuning(gemm_sync=args.gemm_sync, gemm_pairs=args.gemm_pairs)
     if args.only_group_leg:
         print(json.dumps({"group_stage": group_stage_leg(ctx, pk, dev)}), flush=True)
         return
