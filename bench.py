@@ -38,6 +38,23 @@ NOMINAL_BF16_TFLOPS = 2250.0          # dense bf16 of the data sheet; the target
 TARGET_STAGE_B, TARGET_STAGE_A = 0.60, 0.70
 
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of lmhead_kernel<MODE_FWD_P> over a full
+# chunk of 592 token tiles at d = 3584, V = 152064: mean of four launches of a one-pass ncu capture of this program
+# (profiles/one_call_step_full_chunk_dram.md).  Valid for that launch shape and for the kernel as captured; any other
+# shape, or a change of the kernel, gets null.
+FWDP_TRAFFIC = {(3584, 152064, 592 * 128): 74.2e9}
+FWDP_TRAFFIC_NOTE = ("per launch over a full chunk (592 token tiles), from a one-pass ncu capture of "
+                     "`bench.py --config 2 --only-main --steps 1 --warmup 1 --no-e2e`, whose chunks have the launch shape of "
+                     "this workload's: 51.2 GB read (46-55 over four launches; 78-80 in a capture on another GPU of the "
+                     "pool) + 23.0 GB written, against 24.7 GB algorithmic; the excess is H tiles re-read after leaving L2 "
+                     "while a CTA walks the vocabulary, and how many of them miss varies between GPUs and runs; null for "
+                     "other launch shapes")
+
+
+def fwdp_traffic(wl, chunk_tokens):
+    return FWDP_TRAFFIC.get((wl.d, wl.V, int(chunk_tokens)))
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -58,6 +75,8 @@ def parse_args():
     ap.add_argument("--only-main", action="store_true", help="only the timed steps of the headline workload")
     ap.add_argument("--gemm-sync", type=int, default=-1,
                     help="meeting points per unit of the backward products' producers (aero_set_tuning); -1: the library's default")
+    ap.add_argument("--w-hint", type=int, default=-1,
+                    help="lm_head kernel loads W with the evict-first L2 priority (aero_set_tuning); -1: the library's default")
     ap.add_argument("--gemm-pairs", type=int, default=-1,
                     help="backward products on CTA pairs (1) or single CTAs (0) (aero_set_tuning); -1: the library's default")
     return ap.parse_args()
@@ -313,7 +332,7 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     pk = peaks()
     ctx = B.Context(local)
-    ctx.set_tuning(gemm_sync=args.gemm_sync, gemm_pairs=args.gemm_pairs)
+    ctx.set_tuning(gemm_sync=args.gemm_sync, gemm_pairs=args.gemm_pairs, w_hint=args.w_hint)
     if args.only_group_leg:
         print(json.dumps({"group_stage": group_stage_leg(ctx, pk, dev)}), flush=True)
         return
@@ -374,10 +393,9 @@ def run_ours(args):
                 "peak_source": pk["src"] + " sustained bf16 (kernel timed inside the step)",
                 "frac_of_burst": achieved / pk["burst"], "peak_burst": pk["burst"],
                 "frac_of_nominal_peak": achieved / NOMINAL_BF16_TFLOPS,
-                "traffic": None,
-                "traffic_note": "no DRAM counters for this kernel at this size: counters are taken on reduced cases only "
-                                "(profiles/); algorithmic_bytes = kept rows of H + W + the chunk blocks of exp(z - c_t) "
-                                "written, each once per step",
+                "traffic": fwdp_traffic(wl, main.chunk),
+                "traffic_note": FWDP_TRAFFIC_NOTE,
+                "algorithmic_bytes_per_full_launch": float(main.chunk * wl.d * 2 + wl.V * wl.d * 2 + main.chunk * ldz * 2),
                 "algorithmic_bytes": float(T_kept * wl.d * 2 + wl.V * wl.d * 2 + T_kept * ldz * 2),
                 "launches_per_step": fp_launches / n_kt, "ms_per_step_all_launches": fwdp_ms_step,
                 "share_of_step": fwdp_ms_step / (ms_local / args.steps),

@@ -159,6 +159,9 @@ int aero_last_status(aero_ctx* ctx, uint32_t* bits);
  *   "gemm_sync"  meeting points per unit of the two backward products' producers; 0 for none.
  *   "gemm_pairs" 1: the two backward products run on CTA pairs (units of 256 rows); 0: on
  *                single CTAs; by default pairs for d > 2048.
+ *   "w_hint"     1: the lm_head kernel loads W with the evict-first L2 priority, 0: plain loads;
+ *                by default 1 in the calls whose kernel stores per-row results only
+ *                (aero_grpo_loss_fwd, aero_logprob_fwd), 0 where it also stores a chunk block.
  * The workspace sizes the *_workspace_bytes functions return cover every setting.  Returns
  * AERO_ERR_INVALID for an unknown name or a value outside the ones listed. */
 int aero_set_tuning(aero_ctx* ctx, const char* name, int value);

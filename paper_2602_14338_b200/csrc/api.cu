@@ -82,6 +82,7 @@ int aero_create(aero_ctx** out, int device, void* cuda_stream) {
   ctx->n_timed = 0;
   ctx->tune_vsplit = 0;
   ctx->tune_nsync = -1;
+  ctx->tune_w_hint = -1;
   ctx->tune_rowscale = -1;
   ctx->tune_gemm_sync = -1;
   ctx->tune_gemm_pairs = -1;
@@ -156,6 +157,8 @@ int aero_set_tuning(aero_ctx* ctx, const char* name, int value) {
   } else if (n == "gemm_sync") {
     if (value > 4096) return AERO_ERR_INVALID;
     ctx->tune_gemm_sync = value < 0 ? -1 : value;
+  } else if (n == "w_hint") {
+    ctx->tune_w_hint = value < 0 ? -1 : (value ? 1 : 0);
   } else if (n == "gemm_pairs") {
     ctx->tune_gemm_pairs = value < 0 ? -1 : (value ? 1 : 0);
   } else {

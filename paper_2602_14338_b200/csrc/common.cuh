@@ -32,6 +32,7 @@ struct aero_ctx {
   int tune_nsync;         // < 0: the default number of meeting points; 0: no pacing; else that many
   int tune_rowscale;      // < 0 or 1: row factors in the backward GEMMs; 0: the pass that rewrites the block
   int tune_gemm_sync;     // < 0: the default number of meeting points per unit of the backward GEMMs; 0: none
+  int tune_w_hint;        // < 0: by kernel mode; 1: the lm_head kernel loads W with the evict-first L2 priority; 0: plain loads
   int tune_gemm_pairs;    // < 0: by d; 1: the backward GEMMs run on CTA pairs (256-row units); 0: on single CTAs
 };
 
@@ -140,6 +141,11 @@ static inline bool aero_rowscale(const aero_ctx* ctx) { return ctx->tune_rowscal
 // (a CTA stages a third fewer bytes per slab), at d = 1536 they change nothing or lose 1-2 %.
 static inline bool aero_gemm_pairs(const aero_ctx* ctx, int32_t d) {
   return ctx->tune_gemm_pairs < 0 ? d > 2048 : ctx->tune_gemm_pairs != 0;
+}
+// The hint pays where the kernel stores nothing but per-row results (measured: forward 1.5 % faster); where it
+// also streams a block of p~ or dz out with the same priority, the W lines lose against those stores (3 % slower).
+static inline int aero_w_hint(const aero_ctx* ctx, bool kernel_stores_block) {
+  return ctx->tune_w_hint < 0 ? (kernel_stores_block ? 0 : 1) : ctx->tune_w_hint;
 }
 static inline int aero_gemm_sync(const aero_ctx* ctx) { return ctx->tune_gemm_sync >= 0 ? ctx->tune_gemm_sync : 1; }
 size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t d, int32_t R);

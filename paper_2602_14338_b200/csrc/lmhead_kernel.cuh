@@ -86,6 +86,11 @@ struct Params {
   // is simply not waited for.
   unsigned int* sync_ctr;
   int nsync;
+  // W tiles are needed by all their sharers within microseconds of one another (pacing) and not
+  // again before the next wave of token tiles; a CTA's own H tile is needed again for every
+  // vocabulary tile.  With w_hint the W loads carry the evict-first priority, so that the stream
+  // of W lines is what L2 gives up first and the H tiles stay.
+  int w_hint;
   const int64_t* cs;
   const float* w;
   float ent_coef;
@@ -263,6 +268,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
       uint32_t it = 0;
       bool ok = true;
       unsigned int meetings = 0;
+      const uint64_t pol_w = tc::l2_policy_evict_first();
       // every CTA takes part in the same number of meetings: units of the longest schedule x nsync
       const int total_units = ((n_tiles - p.tile_begin + 1) / 2) * vsplit;
       const int max_units = total_units > 0 ? (total_units + npairs - 1) / npairs : 0;
@@ -291,7 +297,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
             const uint32_t full0 = tc::mapa_shared(tc::smem_u32(&ctl->full[s]), 0);
             if (rank == 0) tc::mbar_arrive_expect_tx(&ctl->full[s], 2 * STAGE_BYTES);
             tc::tma_load_2d_pair(a_s, &tmH, kb * BK, row0, full0);
-            tc::tma_load_2d_pair(a_s + A_BYTES, &tmW, kb * BK, j * BN + (int)rank * BNH, full0);
+            if (p.w_hint) tc::tma_load_2d_pair_hint(a_s + A_BYTES, &tmW, kb * BK, j * BN + (int)rank * BNH, full0, pol_w);
+            else tc::tma_load_2d_pair(a_s + A_BYTES, &tmW, kb * BK, j * BN + (int)rank * BNH, full0);
           }
         }
         // a unit whose range has fewer vocabulary tiles than meeting points still counts them all

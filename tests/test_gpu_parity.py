@@ -390,6 +390,22 @@ def test_vocabulary_split_between_cta_pairs(ctx, vsplit):
     # the split changes only the order in which a row's tiles are merged
     assert np.abs((split["logp"][:T] - plain["logp"][:T]).cpu().numpy()).max() < 1e-5
     assert np.abs((split["entropy"][:T] - plain["entropy"][:T]).cpu().numpy()).max() < 1e-4
+    # the L2 eviction priority of the W loads changes no arithmetic: same bits either way, in the
+    # forward (hint on by default) and in the one-call step (off by default)
+    outs = []
+    for hint in (0, 1):
+        ctx.set_tuning(w_hint=hint)
+        try:
+            lp = ctx.logprob_fwd(cfg, dv["H"], dv["W"], dv["y"], entropy=True)
+            f1, dH1, dW1 = ctx.grpo_loss_fwd_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"],
+                                                 dv["keep"])
+            torch.cuda.synchronize()
+        finally:
+            ctx.set_tuning()
+        outs.append((lp["logp"].clone(), f1["logp"].clone(), dH1.clone(), f1["loss"].clone()))
+    assert ctx.last_status() == 0
+    assert torch.equal(outs[0][0], plain["logp"]) and torch.equal(outs[1][0], plain["logp"])
+    assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2]) and torch.equal(outs[0][3], outs[1][3])
 
 
 @pytest.mark.parametrize("name", list(BF16_CASES) + ["tiny_fp32"])
