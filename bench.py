@@ -38,21 +38,21 @@ NOMINAL_BF16_TFLOPS = 2250.0          # dense bf16 of the data sheet; the target
 TARGET_STAGE_B, TARGET_STAGE_A = 0.60, 0.70
 
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of lmhead_kernel<MODE_FWD_P> over a full
-# chunk of 592 token tiles at d = 3584, V = 152064: mean of four launches of a one-pass ncu capture of this program
-# (profiles/one_call_step_full_chunk_dram.md).  Valid for that launch shape and for the kernel as captured; any other
-# shape, or a change of the kernel, gets null.
-FWDP_TRAFFIC = {(3584, 152064, 592 * 128): 74.2e9}
-FWDP_TRAFFIC_NOTE = ("per launch over a full chunk (592 token tiles), from a one-pass ncu capture of "
-                     "`bench.py --config 2 --only-main --steps 1 --warmup 1 --no-e2e`, whose chunks have the launch shape of "
-                     "this workload's: 51.2 GB read (46-55 over four launches; 78-80 in a capture on another GPU of the "
-                     "pool) + 23.0 GB written, against 24.7 GB algorithmic; the excess is H tiles re-read after leaving L2 "
-                     "while a CTA walks the vocabulary, and how many of them miss varies between GPUs and runs; null for "
-                     "other launch shapes")
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per token tile of a launch of lmhead_kernel<MODE_FWD_P> at
+# d = 3584, V = 152064, from an ncu capture of a reduced case of this program (one wave of 148 token tiles per launch:
+# 17.68 GB read + 5.74 GB written, mean of two launches; profiles/one_call_step_full_chunk_dram.md).  The traffic of a
+# launch grows with its token tiles (every wave of 74 tiles streams W once and re-reads its H tiles), so a full launch
+# is that figure times its tiles.  Valid for this shape and for the kernel as captured; otherwise null.
+FWDP_TRAFFIC_PER_TILE = {(3584, 152064): (17.68e9 + 5.74e9) / 148}
+FWDP_TRAFFIC_NOTE = ("per launch over a full chunk: the ncu counters of a reduced case (`bench.py --config 2 --prompts 10 "
+                     "--chunk-tokens 18944 --only-main --steps 1 --warmup 1`, 148 token tiles per launch, 23.4 GB) scaled by "
+                     "the token tiles of a launch; one-pass counters on full chunks gave 69-103 GB on two GPUs; algorithmic "
+                     "24.7 GB, the excess being H tiles re-read after leaving L2; null for other shapes")
 
 
 def fwdp_traffic(wl, chunk_tokens):
-    return FWDP_TRAFFIC.get((wl.d, wl.V, int(chunk_tokens)))
+    per_tile = FWDP_TRAFFIC_PER_TILE.get((wl.d, wl.V))
+    return None if per_tile is None else per_tile * (int(chunk_tokens) // 128)
 
 
 def parse_args():
