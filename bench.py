@@ -40,14 +40,14 @@ TARGET_STAGE_B, TARGET_STAGE_A = 0.60, 0.70
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per token tile of a launch of lmhead_kernel<MODE_FWD_P> at
 # d = 3584, V = 152064, from an ncu capture of a reduced case of this program (one wave of 148 token tiles per launch:
-# 17.68 GB read + 5.74 GB written, mean of two launches; profiles/one_call_step_full_chunk_dram.md).  The traffic of a
+# 6.78 GB read + 5.74 GB written, mean of two launches; profiles/one_call_step_full_chunk_dram.md).  The traffic of a
 # launch grows with its token tiles (every wave of 74 tiles streams W once and re-reads its H tiles), so a full launch
 # is that figure times its tiles.  Valid for this shape and for the kernel as captured; otherwise null.
-FWDP_TRAFFIC_PER_TILE = {(3584, 152064): (17.68e9 + 5.74e9) / 148}
+FWDP_TRAFFIC_PER_TILE = {(3584, 152064): (6.78e9 + 5.74e9) / 148}
 FWDP_TRAFFIC_NOTE = ("per launch over a full chunk: the ncu counters of a reduced case (`bench.py --config 2 --prompts 10 "
-                     "--chunk-tokens 18944 --only-main --steps 1 --warmup 1`, 148 token tiles per launch, 23.4 GB) scaled by "
-                     "the token tiles of a launch; one-pass counters on full chunks gave 69-103 GB on two GPUs; algorithmic "
-                     "24.7 GB, the excess being H tiles re-read after leaving L2; null for other shapes")
+                     "--chunk-tokens 18944 --only-main --steps 1 --warmup 1`, 148 token tiles per launch, 12.5 GB) scaled by "
+                     "the token tiles of a launch; algorithmic 24.7 GB per full launch, the excess being H tiles re-read "
+                     "after leaving L2; null for other shapes")
 
 
 def fwdp_traffic(wl, chunk_tokens):
@@ -77,6 +77,8 @@ def parse_args():
                     help="meeting points per unit of the backward products' producers (aero_set_tuning); -1: the library's default")
     ap.add_argument("--w-hint", type=int, default=-1,
                     help="lm_head kernel loads W with the evict-first L2 priority (aero_set_tuning); -1: the library's default")
+    ap.add_argument("--k-zigzag", type=int, default=-1,
+                    help="lm_head kernel walks d forwards and backwards in turn (aero_set_tuning); -1: the library's default")
     ap.add_argument("--gemm-pairs", type=int, default=-1,
                     help="backward products on CTA pairs (1) or single CTAs (0) (aero_set_tuning); -1: the library's default")
     return ap.parse_args()
@@ -332,7 +334,7 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     pk = peaks()
     ctx = B.Context(local)
-    ctx.set_tuning(gemm_sync=args.gemm_sync, gemm_pairs=args.gemm_pairs, w_hint=args.w_hint)
+    ctx.set_tuning(gemm_sync=args.gemm_sync, gemm_pairs=args.gemm_pairs, w_hint=args.w_hint, k_zigzag=args.k_zigzag)
     if args.only_group_leg:
         print(json.dumps({"group_stage": group_stage_leg(ctx, pk, dev)}), flush=True)
         return

@@ -162,6 +162,9 @@ int aero_last_status(aero_ctx* ctx, uint32_t* bits);
  *   "w_hint"     1: the lm_head kernel loads W with the evict-first L2 priority, 0: plain loads;
  *                by default 1 in the calls whose kernel stores per-row results only
  *                (aero_grpo_loss_fwd, aero_logprob_fwd), 0 where it also stores a chunk block.
+ *   "k_zigzag"   1 (the default): the lm_head kernel walks the reduction dimension d forwards for
+ *                even vocabulary tiles and backwards for odd ones (the H slabs used last are asked
+ *                for first); 0: always forwards.  Changes the order of the fp32 sums of a logit.
  * The workspace sizes the *_workspace_bytes functions return cover every setting.  Returns
  * AERO_ERR_INVALID for an unknown name or a value outside the ones listed. */
 int aero_set_tuning(aero_ctx* ctx, const char* name, int value);

@@ -195,10 +195,10 @@ class Context:
         self.stream = stream
         _check(self.lib.aero_set_stream(self.h, C.c_void_p(stream.cuda_stream)), "aero_set_stream")
 
-    def set_tuning(self, vsplit=0, nsync=-1, rowscale=-1, gemm_sync=-1, gemm_pairs=-1, w_hint=-1):
+    def set_tuning(self, vsplit=0, nsync=-1, rowscale=-1, gemm_sync=-1, gemm_pairs=-1, w_hint=-1, k_zigzag=-1):
         """aero_set_tuning for every setting: schedule choices of stage (b); the defaults let the library decide."""
         for name, value in (("vsplit", vsplit), ("nsync", nsync), ("rowscale", rowscale), ("gemm_sync", gemm_sync),
-                            ("gemm_pairs", gemm_pairs), ("w_hint", w_hint)):
+                            ("gemm_pairs", gemm_pairs), ("w_hint", w_hint), ("k_zigzag", k_zigzag)):
             _check(self.lib.aero_set_tuning(self.h, name.encode(), int(value)), f"aero_set_tuning({name})")
 
     def selftest_bounded_wait(self, limit_us=1000):

@@ -83,6 +83,7 @@ int aero_create(aero_ctx** out, int device, void* cuda_stream) {
   ctx->tune_vsplit = 0;
   ctx->tune_nsync = -1;
   ctx->tune_w_hint = -1;
+  ctx->tune_k_zigzag = -1;
   ctx->tune_rowscale = -1;
   ctx->tune_gemm_sync = -1;
   ctx->tune_gemm_pairs = -1;
@@ -159,6 +160,8 @@ int aero_set_tuning(aero_ctx* ctx, const char* name, int value) {
     ctx->tune_gemm_sync = value < 0 ? -1 : value;
   } else if (n == "w_hint") {
     ctx->tune_w_hint = value < 0 ? -1 : (value ? 1 : 0);
+  } else if (n == "k_zigzag") {
+    ctx->tune_k_zigzag = value < 0 ? -1 : (value ? 1 : 0);
   } else if (n == "gemm_pairs") {
     ctx->tune_gemm_pairs = value < 0 ? -1 : (value ? 1 : 0);
   } else {

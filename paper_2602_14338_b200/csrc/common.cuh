@@ -33,6 +33,7 @@ struct aero_ctx {
   int tune_rowscale;      // < 0 or 1: row factors in the backward GEMMs; 0: the pass that rewrites the block
   int tune_gemm_sync;     // < 0: the default number of meeting points per unit of the backward GEMMs; 0: none
   int tune_w_hint;        // < 0: by kernel mode; 1: the lm_head kernel loads W with the evict-first L2 priority; 0: plain loads
+  int tune_k_zigzag;      // < 0 or 1: the lm_head kernel walks d forwards and backwards in turn (the default); 0: always forwards
   int tune_gemm_pairs;    // < 0: by d; 1: the backward GEMMs run on CTA pairs (256-row units); 0: on single CTAs
 };
 
@@ -147,6 +148,7 @@ static inline bool aero_gemm_pairs(const aero_ctx* ctx, int32_t d) {
 static inline int aero_w_hint(const aero_ctx* ctx, bool kernel_stores_block) {
   return ctx->tune_w_hint < 0 ? (kernel_stores_block ? 0 : 1) : ctx->tune_w_hint;
 }
+static inline int aero_k_zigzag(const aero_ctx* ctx) { return ctx->tune_k_zigzag < 0 ? 1 : ctx->tune_k_zigzag; }
 static inline int aero_gemm_sync(const aero_ctx* ctx) { return ctx->tune_gemm_sync >= 0 ? ctx->tune_gemm_sync : 1; }
 size_t aero_fwd_ws_bytes_tc(int64_t T, int32_t d, int32_t R);
 int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,

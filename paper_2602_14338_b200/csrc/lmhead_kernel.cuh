@@ -91,6 +91,11 @@ struct Params {
   // vocabulary tile.  With w_hint the W loads carry the evict-first priority, so that the stream
   // of W lines is what L2 gives up first and the H tiles stay.
   int w_hint;
+  // With k_zigzag the producer walks the reduction dimension forwards for even vocabulary tiles and
+  // backwards for odd ones, so that the slabs of the CTA's own H tile it used last are the ones it
+  // asks for first: a cyclic walk is the worst case for a cache that gives up the oldest lines.  The
+  // order depends on the tile index alone, so a tile's sums are the same whichever CTA computes it.
+  int k_zigzag;
   const int64_t* cs;
   const float* w;
   float ent_coef;
@@ -296,9 +301,10 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
             uint8_t* a_s = smem + (size_t)s * STAGE_BYTES;
             const uint32_t full0 = tc::mapa_shared(tc::smem_u32(&ctl->full[s]), 0);
             if (rank == 0) tc::mbar_arrive_expect_tx(&ctl->full[s], 2 * STAGE_BYTES);
-            tc::tma_load_2d_pair(a_s, &tmH, kb * BK, row0, full0);
-            if (p.w_hint) tc::tma_load_2d_pair_hint(a_s + A_BYTES, &tmW, kb * BK, j * BN + (int)rank * BNH, full0, pol_w);
-            else tc::tma_load_2d_pair(a_s + A_BYTES, &tmW, kb * BK, j * BN + (int)rank * BNH, full0);
+            const int kx = (p.k_zigzag && (j & 1) ? nkb - 1 - kb : kb) * BK;
+            tc::tma_load_2d_pair(a_s, &tmH, kx, row0, full0);
+            if (p.w_hint) tc::tma_load_2d_pair_hint(a_s + A_BYTES, &tmW, kx, j * BN + (int)rank * BNH, full0, pol_w);
+            else tc::tma_load_2d_pair(a_s + A_BYTES, &tmW, kx, j * BN + (int)rank * BNH, full0);
           }
         }
         // a unit whose range has fewer vocabulary tiles than meeting points still counts them all

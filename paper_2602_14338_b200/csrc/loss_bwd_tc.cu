@@ -109,7 +109,7 @@ int aero_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     lp.lse_in = lse; lp.g_in = g; lp.logp_in = ex.logp; lp.grad_scale = grad_scale; lp.dz = dz; lp.ldz = ldz;
     lp.cs = cs; lp.w = ex.w; lp.ent_in = ex.entropy; lp.ent_coef = ex.ent_coef;
     lp.vsplit = aero_vsplit(ctx, d);
-    lp.sync_ctr = sync_ctr; lp.nsync = aero_nsync(ctx); lp.w_hint = aero_w_hint(ctx, true);
+    lp.sync_ctr = sync_ctr; lp.nsync = aero_nsync(ctx); lp.w_hint = aero_w_hint(ctx, true); lp.k_zigzag = aero_k_zigzag(ctx);
     AERO_CUDA_TRY(cudaMemsetAsync(sync_ctr, 0, 256, ctx->stream));
     const long long max_pairs = ctx->sm_count / 2 > 0 ? ctx->sm_count / 2 : 1;
     const long long dz_pairs = (tpc + 1) / 2 * lp.vsplit;

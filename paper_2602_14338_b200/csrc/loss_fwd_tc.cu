@@ -67,7 +67,7 @@ int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
     p.tile_row = f.tiles.tile_row; p.tile_valid = f.tiles.tile_valid; p.n_tiles = f.tiles.n_tiles;
     p.tile_begin = 0; p.tile_end = f.tiles.max_tiles;
     p.vsplit = aero_vsplit(ctx, d); p.xstate = f.xstate;
-    p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync(ctx); p.w_hint = aero_w_hint(ctx, false);
+    p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync(ctx); p.w_hint = aero_w_hint(ctx, false); p.k_zigzag = aero_k_zigzag(ctx);
     p.y = y; p.status = ctx->d_status;
     p.old_logp = ex.logprob_only ? nullptr : old_logp; p.cs = cs; p.adv = adv; p.w = w;
     p.ref_logp = ex.ref_logp; p.kl_beta = ex.kl_beta; p.ent_coef = ex.ent_coef; p.ent_out = ex.entropy;

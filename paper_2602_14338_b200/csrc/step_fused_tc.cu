@@ -391,7 +391,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
       p.tile_row = f.tiles.tile_row; p.tile_valid = f.tiles.tile_valid; p.n_tiles = f.tiles.n_tiles;
       p.tile_begin = (int)begin; p.tile_end = (int)(begin + tpc);
       p.y = y; p.status = ctx->d_status;
-      p.vsplit = vs; p.xstate = f.xstate; p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync(ctx); p.w_hint = aero_w_hint(ctx, true);
+      p.vsplit = vs; p.xstate = f.xstate; p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync(ctx); p.w_hint = aero_w_hint(ctx, true); p.k_zigzag = aero_k_zigzag(ctx);
       p.old_logp = old_logp; p.cs = cs; p.adv = adv; p.w = w;
       p.ref_logp = ref_logp; p.kl_beta = ref_logp ? kl_beta : 0.f;
       p.clip_lo = cfg->clip_lo; p.clip_hi = cfg->clip_hi;

@@ -406,6 +406,18 @@ def test_vocabulary_split_between_cta_pairs(ctx, vsplit):
     assert ctx.last_status() == 0
     assert torch.equal(outs[0][0], plain["logp"]) and torch.equal(outs[1][0], plain["logp"])
     assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2]) and torch.equal(outs[0][3], outs[1][3])
+    # walking d always forwards (instead of forwards and backwards in turn) only reorders a logit's fp32 sums
+    ctx.set_tuning(k_zigzag=0)
+    try:
+        fwd_only = ctx.logprob_fwd(cfg, dv["H"], dv["W"], dv["y"], entropy=True)
+        f2, dH2, dW2 = ctx.grpo_loss_fwd_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"], dv["keep"])
+        torch.cuda.synchronize()
+    finally:
+        ctx.set_tuning()
+    assert ctx.last_status() == 0
+    assert np.abs((fwd_only["logp"][:T] - plain["logp"][:T]).cpu().numpy()).max() < 1e-5
+    assert np.abs(f2["logp"][:T].cpu().numpy() - ref["logp"]).max() <= LOGP_ABS
+    assert TL.rel_l2(dH2.float().cpu().numpy(), outs[0][2].float().cpu().numpy()) < 5e-3    # bf16 roundings that flip
 
 
 @pytest.mark.parametrize("name", list(BF16_CASES) + ["tiny_fp32"])
