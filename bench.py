@@ -325,11 +325,17 @@ def run_ours(args):
     from paper_2602_14338_b200 import binding as B
     from paper_2602_14338_b200 import dist as D
 
-    rank, world, local = D.init_from_env()
+    # AERO_DIST_BACKEND=gloo lets the ranks share a GPU (NCCL wants one GPU per rank): a functional check of the
+    # data-parallel step where fewer GPUs than ranks are at hand, never a measurement
+    rank, world, local = D.init_from_env(os.environ.get("AERO_DIST_BACKEND"))
     if world != args.gpus:
         raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device (the library has no CPU path)")
+    if local >= torch.cuda.device_count():
+        if os.environ.get("AERO_DIST_BACKEND") != "gloo":
+            raise SystemExit(f"bench.py: rank {rank} has no GPU of its own ({torch.cuda.device_count()} visible)")
+        local = local % torch.cuda.device_count()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     pk = peaks()
@@ -587,6 +593,20 @@ def e2e_leg(ctx, pw, args, T_kept, world, dev):
 
     st, wl, cfg = pw.st, pw.wl, pw.cfg
     P, R, T = pw.P, pw.R, pw.T
+    # every rank pins its own copy of H: leave the leg out where the ranks' copies together would take more than
+    # half of the host memory that is free (all ranks decide alike)
+    need = float(pw.H.numel() * pw.H.element_size())
+    try:
+        import psutil
+        free = float(psutil.virtual_memory().available)
+    except Exception:
+        free = float("inf")
+    fits = torch.tensor([1.0 if need * world < 0.5 * free else 0.0], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(fits, op=torch.distributed.ReduceOp.MIN)
+    if fits.item() == 0.0:
+        return {"value": None, "unit": UNIT, "h2d_bytes_per_step": None, "d2h_bytes_per_step": None,
+                "skipped": f"{world} ranks x {need / 1e9:.1f} GB of pinned H against {free / 1e9:.0f} GB of free host memory"}
     pw.ws = None                                   # the host-buffer call has a workspace of its own
     gc.collect()
     torch.cuda.empty_cache()
