@@ -498,8 +498,8 @@ def k_sweep_leg(ctx, pw, pk):
 
 
 def variants_leg(ctx, pw, T_kept, pk):
-    """The step with Eq. 2's KL term and the entropy bonus (aero_grpo_loss_reg_fwd/_bwd), the one-call step
-    with the KL term (aero_grpo_loss_kl_fwd_bwd), the log-prob pass alone (aero_logprob_fwd) that produces old /
+    """The step with Eq. 2's KL term and the entropy bonus through the two calls (aero_grpo_loss_reg_fwd/_bwd) and
+    through one (aero_grpo_loss_reg_fwd_bwd), the one-call step with the KL term alone (aero_grpo_loss_kl_fwd_bwd), the log-prob pass alone (aero_logprob_fwd) that produces old /
     reference log-probs, and the allocation controller on simulated prompts; on the workload passed in."""
     import copy
     import torch
@@ -518,6 +518,9 @@ def variants_leg(ctx, pw, T_kept, pk):
                               dW=pw.dW, workspace=pw.ws, logp=f["logp"])
 
     ms_reg = timed(reg_step, 3)
+    ob = {}
+    ms_reg1 = timed(lambda: ctx.grpo_loss_fwd_bwd(rcfg, pw.H, pw.W, pw.y, pw.old, pw.cs, g["adv"], g["w"], g["keep"], out=ob,
+                                                  dH=pw.dH, dW=pw.dW, workspace=pw.ws, ref_logp=ref, entropy=True), 3)
     kcfg = copy.copy(pw.cfg)
     kcfg.kl_beta = 0.04
     ms_kl = timed(lambda: ctx.grpo_loss_fwd_bwd(kcfg, pw.H, pw.W, pw.y, pw.old, pw.cs, g["adv"], g["w"], g["keep"], out=kb,
@@ -542,6 +545,11 @@ def variants_leg(ctx, pw, T_kept, pk):
             "regularised_step": {"kl_beta": 0.04, "ent_coef": 1e-3, "ms": ms_reg, "tokens_per_s": T_kept / (ms_reg * 1e-3),
                                  "executed_tflops": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12,
                                  "frac_of_sustained": 4 * fl * T_kept / (ms_reg * 1e-3) / 1e12 / pk["sustained"]},
+            "regularised_step_one_call": {"kl_beta": 0.04, "ent_coef": 1e-3, "ms": ms_reg1,
+                                          "tokens_per_s": T_kept / (ms_reg1 * 1e-3),
+                                          "executed_tflops": 3 * fl * T_kept / (ms_reg1 * 1e-3) / 1e12,
+                                          "frac_of_sustained": 3 * fl * T_kept / (ms_reg1 * 1e-3) / 1e12 / pk["sustained"],
+                                          "api": "aero_grpo_loss_reg_fwd_bwd"},
             "kl_step_one_call": {"kl_beta": 0.04, "ms": ms_kl, "tokens_per_s": T_kept / (ms_kl * 1e-3),
                                  "executed_tflops": 3 * fl * T_kept / (ms_kl * 1e-3) / 1e12,
                                  "frac_of_sustained": 3 * fl * T_kept / (ms_kl * 1e-3) / 1e12 / pk["sustained"]},

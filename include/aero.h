@@ -363,8 +363,7 @@ int aero_grpo_loss_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_
 
 /* aero_grpo_loss_fwd_bwd with Eq. 2's KL term: ref_logp [T] f32 (NULL: no KL term, the call is
  * aero_grpo_loss_fwd_bwd) and cfg->kl_beta, defined as for aero_grpo_loss_reg_fwd below.  The term
- * only changes loss and g_t, so it costs nothing in the backward.  (The entropy bonus needs the
- * logits again in the backward and is available through aero_grpo_loss_reg_fwd / _reg_bwd only.) */
+ * only changes loss and g_t, so it costs nothing in the backward. */
 int aero_grpo_loss_kl_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                               const void* H, const void* W, const int32_t* y, const float* old_logp,
                               const float* ref_logp,
@@ -372,6 +371,23 @@ int aero_grpo_loss_kl_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int
                               float* logp, float* lse, float* g, float* loss, float* metrics,
                               float grad_scale, void* dH, float* dW, int accumulate_dW,
                               void* workspace, size_t workspace_bytes);
+
+/* aero_grpo_loss_fwd_bwd with both regularisers of Eq. 2 and Table 9 (defined with
+ * aero_grpo_loss_reg_fwd below): ref_logp [T] f32 or NULL as above, entropy [T] f32 out or NULL (NULL:
+ * no entropy term; with both NULL the call is aero_grpo_loss_fwd_bwd).  The entropy term of dz needs
+ * log p_tv per entry; the step takes it back from the stored block, log p_tv = log p~_tv + c_t - lse_t,
+ * in the pass that rewrites the block to dz (the row-factor form does not apply: the term is no
+ * multiple of p~ along a row).  The bf16 rounding of p~ moves that logarithm by at most 2^-9
+ * absolute; the target column uses the fp32 log-prob.  An entry whose p~ underflowed to 0 gets 0
+ * (p log p -> 0).  6 d V FLOP per token plus one pass over the chunk block, against 8 d V through
+ * aero_grpo_loss_reg_fwd + aero_grpo_loss_reg_bwd. */
+int aero_grpo_loss_reg_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                               const void* H, const void* W, const int32_t* y, const float* old_logp,
+                               const float* ref_logp,
+                               const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                               float* logp, float* lse, float* g, float* entropy, float* loss, float* metrics,
+                               float grad_scale, void* dH, float* dW, int accumulate_dW,
+                               void* workspace, size_t workspace_bytes);
 
 /* ------------------------------------------------------------------------------
  * Stage (b) with the regularisers of Eq. 2 and Table 9.

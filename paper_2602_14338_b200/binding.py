@@ -30,7 +30,8 @@ EXPORTS = [
     "aero_step_workspace_bytes", "aero_grpo_step_host", "aero_launch_count", "aero_group_stats_static",
     "aero_grpo_loss_reg_fwd", "aero_grpo_loss_reg_bwd", "aero_logprob_fwd",
     "aero_alloc_cfg_default", "aero_allocate_workspace_bytes", "aero_allocate_sim",
-    "aero_fwd_bwd_workspace_bytes", "aero_grpo_loss_fwd_bwd", "aero_grpo_loss_kl_fwd_bwd", "aero_enable_kernel_timing", "aero_kernel_timing_ms",
+    "aero_fwd_bwd_workspace_bytes", "aero_grpo_loss_fwd_bwd", "aero_grpo_loss_kl_fwd_bwd", "aero_grpo_loss_reg_fwd_bwd",
+    "aero_enable_kernel_timing", "aero_kernel_timing_ms",
     "aero_set_tuning", "aero_finalize_weights", "aero_selftest_bounded_wait",
 ]
 
@@ -106,6 +107,8 @@ def load_library():
                                            [vp, vp, C.c_int, vp, sz])
     lib.aero_grpo_loss_kl_fwd_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 14 + [f32] +
                                               [vp, vp, C.c_int, vp, sz])
+    lib.aero_grpo_loss_reg_fwd_bwd.argtypes = ([vp, C.POINTER(AeroCfg), i64, i32, i32, i32] + [vp] * 15 + [f32] +
+                                               [vp, vp, C.c_int, vp, sz])
     lib.aero_enable_kernel_timing.argtypes = [vp, C.c_int]
     lib.aero_kernel_timing_ms.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int)]
     lib.aero_step_workspace_bytes.restype = sz
@@ -387,9 +390,10 @@ class Context:
         return self.lib.aero_fwd_bwd_workspace_bytes(T, d, V, R, chunk_tokens)
 
     def grpo_loss_fwd_bwd(self, cfg, H, W, y, old_logp, cs, adv, w, keep, out=None, grad_scale=1.0, dH=None, dW=None,
-                          accumulate_dW=False, chunk_tokens=None, workspace=None, ref_logp=None):
-        """aero_grpo_loss_fwd_bwd (aero_grpo_loss_kl_fwd_bwd when ref_logp is given): forward and backward of
-        stage (b) in one call (no recompute of the logits).  Returns (forward outputs dict, dH, dW)."""
+                          accumulate_dW=False, chunk_tokens=None, workspace=None, ref_logp=None, entropy=False):
+        """aero_grpo_loss_fwd_bwd (aero_grpo_loss_kl_fwd_bwd when ref_logp is given, aero_grpo_loss_reg_fwd_bwd when
+        the entropy term is asked for): forward and backward of stage (b) in one call (no recompute of the
+        logits).  Returns (forward outputs dict, dH, dW)."""
         T, d = H.shape
         V = W.shape[0]
         R = cs.numel() - 1
@@ -416,7 +420,13 @@ class Context:
                 _ptr(keep, torch.uint8, R, "keep"), _ptr(o["logp"]), _ptr(o["lse"]), _ptr(o["g"]), _ptr(o["loss"]),
                 _ptr(o["metrics"]), C.c_float(grad_scale), _ptr(dH, dt, T * d, "dH"), _ptr(dW, torch.float32, V * d, "dW"),
                 1 if accumulate_dW else 0, workspace.data_ptr(), workspace.numel())
-        if ref_logp is None:
+        if entropy:
+            if "entropy" not in o:
+                o["entropy"] = torch.empty(max(T, 1), dtype=torch.float32, device=self.device)
+            ref = _ptr(ref_logp, torch.float32, T, "ref_logp") if ref_logp is not None else None
+            _check(self.lib.aero_grpo_loss_reg_fwd_bwd(*head, ref, *tail[:7], _ptr(o["entropy"]), *tail[7:]),
+                   "aero_grpo_loss_reg_fwd_bwd")
+        elif ref_logp is None:
             _check(self.lib.aero_grpo_loss_fwd_bwd(*head, *tail), "aero_grpo_loss_fwd_bwd")
         else:
             _check(self.lib.aero_grpo_loss_kl_fwd_bwd(*head, _ptr(ref_logp, torch.float32, T, "ref_logp"), *tail),

@@ -291,13 +291,13 @@ size_t aero_fwd_bwd_workspace_bytes(int64_t T, int32_t d, int32_t V, int32_t R, 
   return a > b ? a : b;
 }
 
-int aero_grpo_loss_kl_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
-                              const void* H, const void* W, const int32_t* y, const float* old_logp,
-                              const float* ref_logp,
-                              const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
-                              float* logp, float* lse, float* g, float* loss, float* metrics,
-                              float grad_scale, void* dH, float* dW, int accumulate_dW,
-                              void* workspace, size_t workspace_bytes) {
+int aero_grpo_loss_reg_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                               const void* H, const void* W, const int32_t* y, const float* old_logp,
+                               const float* ref_logp,
+                               const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                               float* logp, float* lse, float* g, float* entropy, float* loss, float* metrics,
+                               float grad_scale, void* dH, float* dW, int accumulate_dW,
+                               void* workspace, size_t workspace_bytes) {
   Range nv("aero_grpo_loss_fwd_bwd");
   if (!ctx || !cfg || T < 0 || d <= 0 || V <= 0 || R < 0 || T >= (int64_t)1 << 31) return AERO_ERR_INVALID;
   if (!W || !cs || !loss || !dW) return AERO_ERR_INVALID;
@@ -306,8 +306,11 @@ int aero_grpo_loss_kl_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int
   if (!workspace || !aligned256(workspace)) return AERO_ERR_INVALID;
   if (cfg->dtype == AERO_FP32) {
     int rc = aero_grpo_loss_reg_fwd(ctx, cfg, T, d, V, R, H, W, y, old_logp, ref_logp, cs, adv, w, keep, logp, lse, g,
-                                    nullptr, loss, metrics, 0, workspace, workspace_bytes);
+                                    entropy, loss, metrics, 0, workspace, workspace_bytes);
     if (rc) return rc;
+    if (entropy)
+      return aero_grpo_loss_reg_bwd(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, logp, entropy, w, grad_scale, dH, dW,
+                                    accumulate_dW, workspace, workspace_bytes);
     return aero_grpo_loss_bwd(ctx, cfg, T, d, V, R, H, W, y, cs, keep, lse, g, logp, grad_scale, dH, dW, accumulate_dW,
                               workspace, workspace_bytes);
   }
@@ -317,8 +320,19 @@ int aero_grpo_loss_kl_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int
   if (workspace_bytes < aero_fwd_bwd_ws_bytes_tc(T, d, V, R, 128)) return AERO_ERR_WORKSPACE;
   const int rc = check_ctx(ctx);
   if (rc) return rc;
-  return aero_fwd_bwd_tc(ctx, cfg, T, d, V, R, H, W, y, old_logp, ref_logp, cfg->kl_beta, cs, adv, w, keep, logp, lse, g,
-                         loss, metrics, grad_scale, dH, dW, accumulate_dW, workspace, workspace_bytes);
+  return aero_fwd_bwd_tc(ctx, cfg, T, d, V, R, H, W, y, old_logp, ref_logp, cfg->kl_beta, entropy, cfg->ent_coef, cs, adv, w,
+                         keep, logp, lse, g, loss, metrics, grad_scale, dH, dW, accumulate_dW, workspace, workspace_bytes);
+}
+
+int aero_grpo_loss_kl_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
+                              const void* H, const void* W, const int32_t* y, const float* old_logp,
+                              const float* ref_logp,
+                              const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
+                              float* logp, float* lse, float* g, float* loss, float* metrics,
+                              float grad_scale, void* dH, float* dW, int accumulate_dW,
+                              void* workspace, size_t workspace_bytes) {
+  return aero_grpo_loss_reg_fwd_bwd(ctx, cfg, T, d, V, R, H, W, y, old_logp, ref_logp, cs, adv, w, keep, logp, lse, g,
+                                    nullptr, loss, metrics, grad_scale, dH, dW, accumulate_dW, workspace, workspace_bytes);
 }
 
 int aero_grpo_loss_fwd_bwd(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,

@@ -159,7 +159,7 @@ int aero_fwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_
 size_t aero_fwd_bwd_ws_bytes_tc(int64_t T, int32_t d, int32_t V, int32_t R, int64_t chunk_tokens);
 int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                     const void* H, const void* W, const int32_t* y, const float* old_logp,
-                    const float* ref_logp, float kl_beta,
+                    const float* ref_logp, float kl_beta, float* entropy, float ent_coef,
                     const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
                     float* logp, float* lse, float* g, float* loss, float* metrics,
                     float grad_scale, void* dH, float* dW, int accumulate_dW, void* ws, size_t ws_bytes);

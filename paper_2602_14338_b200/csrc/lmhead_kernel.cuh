@@ -50,7 +50,7 @@ constexpr int BM = 128, BN = 256, BNH = BN / 2, BK = 64, STAGES = AERO_TC_STAGES
 constexpr uint32_t A_BYTES = BM * BK * 2, B_BYTES = BNH * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
 // bit 0: dz mode, bit 1: entropy term, bit 2: the forward also stores exp(z - c_t) of the chunk (see MODE_FWD_P)
-constexpr int MODE_FWD = 0, MODE_DZ = 1, MODE_FWD_ENT = 2, MODE_DZ_ENT = 3, MODE_FWD_P = 4;
+constexpr int MODE_FWD = 0, MODE_DZ = 1, MODE_FWD_ENT = 2, MODE_DZ_ENT = 3, MODE_FWD_P = 4, MODE_FWD_P_ENT = 6;
 constexpr float kShiftMargin = 40.f;   // c_t = (largest logit of the row's first 32 columns) + this margin
 constexpr float kMasked = -1e30f;   // stands for -inf in columns past V (finite, so that 0 * z stays 0)
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
@@ -108,6 +108,7 @@ struct Params {
   float* lse_out;
   float* g_out;
   float* ent_out;               // entropy per row (entropy modes)
+  float* zmax_out;              // largest logit of the row outside the target's column, or NULL (-inf if there is none)
   float* shift_out;             // MODE_FWD_P: c_t * log2(e) per split and row, [vsplit][T]
   int common_shift;             // MODE_FWD_P with vsplit > 1: every split takes c_t from the row's first 32 logits
                                 // of the whole vocabulary (the later splits compute that tile once more for it)
@@ -165,6 +166,7 @@ __device__ __forceinline__ void finish_rows(const Params& p, bool ent_mode, bool
     p.logp[row] = lp;
     p.lse_out[row] = ls;
     if (ent_mode) p.ent_out[row] = ent;
+    if (p.zmax_out != nullptr) p.zmax_out[row] = l > 0.f ? m2 * kLn2 : -INFINITY;
     if (p.old_logp != nullptr) {
       const int i = aero_owner(p.cs, p.R, row);
       const float old = p.old_logp[row];
@@ -265,7 +267,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
   auto unit_j0 = [&](int k) { return (int)((long long)((pair + k * npairs) % vsplit) * nvt / vsplit); };
   auto unit_j1 = [&](int k) { return (int)((long long)((pair + k * npairs) % vsplit + 1) * nvt / vsplit); };
   // with a common shift, a unit of a later split starts with vocabulary tile 0, used for the shift alone
-  auto unit_pre = [&](int k) { return (MODE == MODE_FWD_P && p.common_shift && (pair + k * npairs) % vsplit != 0) ? 1 : 0; };
+  auto unit_pre = [&](int k) { return (STORE_P && p.common_shift && (pair + k * npairs) % vsplit != 0) ? 1 : 0; };
 
   if (warp == 4) {
     // ---------------- TMA producer ----------------
@@ -493,6 +495,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ C
               for (int q = 0; q < 32; q += 2) {
                 const float e0 = ex2(fmaf(z[q], kLog2e, -m2n)), e1 = ex2(fmaf(z[q + 1], kLog2e, -m2n));
                 acc += e0 + e1;
+                if (ENT) accz = fmaf(e0, z[q], fmaf(e1, z[q + 1], accz));
                 pk[q >> 1] = pack_bf16(e0 * sc, e1 * sc);
               }
               stage_store(pk, c, col0);

@@ -45,12 +45,24 @@ struct ScaleArgs {
   const float* logp;
   const float* shift;       // [vsplit][T], log2 domain
   float grad_scale;
+  const float* ent;         // entropy term: H_t per row,
+  const float* row_et;      // ... ent_coef * w_i per row,
+  const float* zmax;        // ... and the row's largest logit outside the target's column (all NULL without the term)
 };
 
 constexpr int kBlocksPerCta = 8;     // 64-column blocks one CTA rescales for its token tile
 
 // One CTA: one token tile x kBlocksPerCta column blocks of the chunk's block, 16 bytes per thread
 // and step.  Rows past the tile's run, or whose g is 0, come out as zeros (p~ is 0 or g is).
+// With the entropy term (Table 9's bonus) an entry gets e_t p (log p + H_t) more, e_t = ent_coef w_i
+// grad_scale, where log p comes back from the stored value: log p = log p~ + c_t - lse_t.  The
+// rounding of p~ to bf16 moves that logarithm by up to 2^-8 absolute, which is nothing for the many
+// small entries (the error of the entry is that times p) but would be all of the entry where one
+// column holds nearly the whole probability (log p + H_t close to 0).  The two columns that can do
+// so take exact logarithms: the target's from the fp32 log-prob, the largest other logit's from
+// its fp32 value, kept by the forward; an entry is taken for the latter when its stored value is
+// within bf16 rounding of it.
+template <bool ENT>
 __global__ void __launch_bounds__(256) scale_dz_kernel(ScaleArgs a) {
   const int n_tiles = min(*a.n_tiles, a.tile_end);
   const int tile = a.tile_begin + blockIdx.y;
@@ -65,27 +77,49 @@ __global__ void __launch_bounds__(256) scale_dz_kernel(ScaleArgs a) {
     const long long row = (long long)row0 + r;
     uint4* ptr = reinterpret_cast<uint4*>(a.dz + (((size_t)blockIdx.y * a.nblk + b) * 128 + r) * 64 + seg * 8);
     float coef = 0.f, sc = 0.f, tgt = 0.f;
+    float et = 0.f, e2 = 0.f, pe = 0.f, hent = 0.f;   // entropy term: e_t, log2 of p / p~, p / p~, H_t
+    float lpm = 0.f, ptm_lo = INFINITY, ptm_hi = -INFINITY;   // ... log p of the largest other column, its p~ +- rounding
     int yt = -1;
     if (r < valid && row < a.T) {
       coef = a.g[row] * a.grad_scale;
       yt = a.y[row];
-      if (coef != 0.f) {
-        tgt = -coef * expm1f(a.logp[row]);          // coef (1 - p_y), exact for p_y close to 1
+      if (ENT) et = a.row_et[row] * a.grad_scale;
+      if (coef != 0.f || et != 0.f) {
+        const float lp = a.logp[row];
+        tgt = -coef * expm1f(lp);                   // coef (1 - p_y), exact for p_y close to 1
         // the vocabulary split that produced this column block, and its shift
         const int j = b / (lmhead::BN / 64);
         int s = 0;
         while (s + 1 < a.vsplit && j >= (int)((long long)(s + 1) * a.nvt / a.vsplit)) ++s;
-        sc = -coef * exp2f(a.shift[(size_t)s * a.T + row] - a.lse[row] * kLog2e);
+        e2 = a.shift[(size_t)s * a.T + row] - a.lse[row] * kLog2e;
+        pe = exp2f(e2);
+        sc = -coef * pe;
+        if (ENT) {
+          hent = a.ent[row];
+          tgt = fmaf(et * __expf(lp), lp + hent, tgt);
+          lpm = a.zmax[row] - a.lse[row];
+          const float ptm = exp2f(lpm * kLog2e - e2);          // what the forward stored for that column, before rounding
+          ptm_lo = ptm * (1.f - 0.0059f);                      // 1.5 bf16 steps either way
+          ptm_hi = ptm * (1.f + 0.0059f);
+        }
       }
     }
     uint4 v = *ptr;
     __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
     const int col0 = b * 64 + seg * 8;
+    constexpr float kLn2 = 0.6931471805599453f;
+    // dz = p (-coef + e_t (log p + H_t)) with p = p~ pe; an entry that underflowed to 0 stays 0
+    auto entry = [&](float pt) {
+      if (!ENT) return sc * pt;
+      if (pt <= 0.f) return 0.f;
+      const float lpv = (pt >= ptm_lo && pt <= ptm_hi) ? lpm : (__log2f(pt) + e2) * kLn2;
+      return pt * fmaf(et * pe, lpv + hent, sc);
+    };
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       float2 f = __bfloat1622float2(h[q]);
-      f.x = col0 + 2 * q == yt ? tgt : sc * f.x;
-      f.y = col0 + 2 * q + 1 == yt ? tgt : sc * f.y;
+      f.x = col0 + 2 * q == yt ? tgt : entry(f.x);
+      f.y = col0 + 2 * q + 1 == yt ? tgt : entry(f.y);
       h[q] = __floats2bfloat162_rn(f.x, f.y);
     }
     *ptr = v;
@@ -183,6 +217,8 @@ struct RangeArgs {
   const __nv_bfloat16* W;   // [V, d]
   __nv_bfloat16* Hs;        // row-factor form: the row's copy of H (unscaled here); NULL otherwise
   float* row_scale;         // row-factor form: set to 1 for a redone row
+  const float* ent;         // entropy term: H_t and ent_coef * w_i per row; both NULL without the term
+  const float* row_et;
 };
 
 // The forward could not hold exp(z - c_t) of these rows in bf16: write their dz rows from the
@@ -202,8 +238,9 @@ __global__ void __launch_bounds__(256) range_fix_kernel(RangeArgs a) {
     const long long row = (long long)a.tile_row[a.tile_begin + lt] + r;
     if (row >= a.T) continue;
     const float coef = a.g[row] * a.grad_scale;
+    const float et = a.row_et != nullptr ? a.row_et[row] * a.grad_scale : 0.f;
     float val = 0.f;
-    if (v < a.V && coef != 0.f) {
+    if (v < a.V && (coef != 0.f || et != 0.f)) {
       const uint4* h = reinterpret_cast<const uint4*>(a.H + row * a.d);
       const uint4* w = reinterpret_cast<const uint4*>(a.W + (long long)v * a.d);
       float acc = 0.f;
@@ -220,7 +257,9 @@ __global__ void __launch_bounds__(256) range_fix_kernel(RangeArgs a) {
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      val = v == a.y[row] ? -coef * expm1f(a.logp[row]) : -coef * __expf(acc - a.lse[row]);
+      const float lpv = v == a.y[row] ? a.logp[row] : acc - a.lse[row];
+      val = v == a.y[row] ? -coef * expm1f(lpv) : -coef * __expf(lpv);
+      if (et != 0.f) val = fmaf(et * __expf(lpv), lpv + a.ent[row], val);
     }
     if (lane == 0) a.dz[(((size_t)lt * a.nblk + v / 64) * 128 + r) * 64 + v % 64] = __float2bfloat16_rn(val);
     if (a.Hs != nullptr && v == 0) {
@@ -230,6 +269,23 @@ __global__ void __launch_bounds__(256) range_fix_kernel(RangeArgs a) {
       uint4* dst = reinterpret_cast<uint4*>(a.Hs + ((size_t)lt * 128 + r) * a.d);
       for (int k = lane; k < a.d / 8; k += 32) dst[k] = src[k];
     }
+  }
+}
+
+// Entropy term: ent_coef * w_i for every token row of a kept rollout (one warp per rollout), so
+// that the per-row kernels need no search for the row's owner.
+__global__ void __launch_bounds__(256) row_entropy_weights_kernel(int R, const int64_t* __restrict__ cs,
+                                                                  const uint8_t* __restrict__ keep,
+                                                                  const float* __restrict__ w, float ent_coef,
+                                                                  long long T, float* __restrict__ row_et) {
+  const int lane = threadIdx.x & 31;
+  const int warp0 = blockIdx.x * 8 + (threadIdx.x >> 5), nwarps = gridDim.x * 8;
+  for (int i = warp0; i < R; i += nwarps) {
+    const float v = keep[i] ? ent_coef * w[i] : 0.f;
+    long long t1 = cs[i + 1];
+    if (t1 > T) t1 = T;
+    for (long long t = cs[i] + lane; t < t1; t += 32)
+      if (t >= 0) row_et[t] = v;
   }
 }
 
@@ -256,6 +312,7 @@ struct FusedWs {
   float4* xstate;
   float* shift;
   float* row_scale;
+  float* zmax;
   int* range_count;
   int* range_rows;
   __nv_bfloat16* dz;
@@ -282,6 +339,7 @@ FusedWs carve(void* ws, int64_t T, int32_t d, int32_t R) {
   f.xstate = reinterpret_cast<float4*>(p + off);               off += aero_align_up(vs * Tn * sizeof(float4), 256);
   f.shift = reinterpret_cast<float*>(p + off);                 off += aero_align_up(vs * Tn * sizeof(float), 256);
   f.row_scale = reinterpret_cast<float*>(p + off);             off += aero_align_up(Tn * sizeof(float), 256);
+  f.zmax = reinterpret_cast<float*>(p + off);                  off += aero_align_up(Tn * sizeof(float), 256);
   f.dz = reinterpret_cast<__nv_bfloat16*>(p + off);
   f.head_bytes = off;
   return f;
@@ -297,16 +355,18 @@ size_t aero_fwd_bwd_ws_bytes_tc(int64_t T, int32_t d, int32_t V, int32_t R, int6
 
 int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, int32_t V, int32_t R,
                     const void* H, const void* W, const int32_t* y, const float* old_logp,
-                    const float* ref_logp, float kl_beta,
+                    const float* ref_logp, float kl_beta, float* entropy, float ent_coef,
                     const int64_t* cs, const float* adv, const float* w, const uint8_t* keep,
                     float* logp, float* lse, float* g, float* loss, float* metrics,
                     float grad_scale, void* dH, float* dW, int accumulate_dW, void* ws, size_t ws_bytes) {
   FusedWs f = carve(ws, T, d, R);
+  const bool with_ent = entropy != nullptr;
   AERO_CUDA_TRY(cudaMemsetAsync(f.partials, 0, f.n_partials * kPartialStride * sizeof(double), ctx->stream));
   if (T > 0) {
     AERO_CUDA_TRY(cudaMemsetAsync(logp, 0, (size_t)T * sizeof(float), ctx->stream));
     AERO_CUDA_TRY(cudaMemsetAsync(lse, 0, (size_t)T * sizeof(float), ctx->stream));
     AERO_CUDA_TRY(cudaMemsetAsync(g, 0, (size_t)T * sizeof(float), ctx->stream));
+    if (with_ent) AERO_CUDA_TRY(cudaMemsetAsync(entropy, 0, (size_t)T * sizeof(float), ctx->stream));
   }
   if (!accumulate_dW) AERO_CUDA_TRY(cudaMemsetAsync(dW, 0, (size_t)V * d * sizeof(float), ctx->stream));
   int rc = aero_build_tiles(ctx, T, R, cs, keep, lmhead::BM, f.tiles);
@@ -345,7 +405,15 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
     if ((rc = aero_make_tmap_dz(ctx, &tmDZ_mn, f.dz, (uint64_t)tpc, nblk, 64, gemmbwd::BM / 64))) return rc;
     if ((rc = aero_make_tmap_blocked(ctx, &tmW_mn, W, V, d, d, 64, gemmbwd::BN / 64))) return rc;
     if ((rc = aero_make_tmap_blocked(ctx, &tmH_mn, H, T, d, d, 64, gemmbwd::BN / 64))) return rc;
-    const bool rowscale = aero_rowscale(ctx);
+    // the entropy term is no multiple of p~ along a row: it takes the pass that rewrites the block, and
+    // the array of row factors then holds ent_coef * w_i per row
+    const bool rowscale = aero_rowscale(ctx) && !with_ent;
+    if (with_ent) {
+      const int blocks = (R + 7) / 8;
+      row_entropy_weights_kernel<<<blocks < 4096 ? (blocks > 0 ? blocks : 1) : 4096, 256, 0, ctx->stream>>>(
+          R, cs, keep, w, ent_coef, T, f.row_scale);
+      ctx->launches += 1;
+    }
     __nv_bfloat16* Hs = f.dz + (size_t)tpc * lmhead::BM * (size_t)ldz;      // after the chunk's p~ block
     CUtensorMap tmHs_mn;
     if (rowscale && (rc = aero_make_tmap_blocked(ctx, &tmHs_mn, Hs, tpc * lmhead::BM, d, d, 64, gemmbwd::BN / 64))) return rc;
@@ -359,7 +427,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
       if (rc) return rc;
     }
 
-    auto k_fwd = lmhead::lmhead_kernel<lmhead::MODE_FWD_P>;
+    auto k_fwd = with_ent ? lmhead::lmhead_kernel<lmhead::MODE_FWD_P_ENT> : lmhead::lmhead_kernel<lmhead::MODE_FWD_P>;
     auto k_dh = gemmbwd::gemm_kernel<gemmbwd::KIND_DH>;
     auto k_dw = gemmbwd::gemm_kernel<gemmbwd::KIND_DW>;
     AERO_CUDA_TRY(cudaFuncSetAttribute(k_fwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lmhead::SMEM_BYTES));
@@ -394,6 +462,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
       p.vsplit = vs; p.xstate = f.xstate; p.sync_ctr = f.sync_ctr; p.nsync = aero_nsync(ctx); p.w_hint = aero_w_hint(ctx, true); p.k_zigzag = aero_k_zigzag(ctx);
       p.old_logp = old_logp; p.cs = cs; p.adv = adv; p.w = w;
       p.ref_logp = ref_logp; p.kl_beta = ref_logp ? kl_beta : 0.f;
+      p.ent_out = entropy; p.ent_coef = with_ent ? ent_coef : 0.f; p.zmax_out = with_ent ? f.zmax : nullptr;
       p.clip_lo = cfg->clip_lo; p.clip_hi = cfg->clip_hi;
       p.logp = logp; p.lse_out = lse; p.g_out = g; p.partials = f.partials;
       p.shift_out = f.shift; p.dz = f.dz; p.ldz = ldz;
@@ -417,7 +486,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
       }
       ctx->launches += 1;
       if (vs > 1) {
-        lmhead::merge_kernel<<<(int)(tpc < 8 * ctx->sm_count ? tpc : 8 * ctx->sm_count), lmhead::BM, 0, ctx->stream>>>(p, 0);
+        lmhead::merge_kernel<<<(int)(tpc < 8 * ctx->sm_count ? tpc : 8 * ctx->sm_count), lmhead::BM, 0, ctx->stream>>>(p, with_ent ? 1 : 0);
         ctx->launches += 1;
       }
       if (rowscale) {
@@ -433,7 +502,10 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
         sa.n_tiles = f.tiles.n_tiles; sa.tile_begin = (int)begin; sa.tile_end = (int)(begin + tpc);
         sa.T = T; sa.V = V; sa.vsplit = vs; sa.nvt = nvt; sa.y = y; sa.lse = lse; sa.g = g; sa.logp = logp; sa.shift = f.shift;
         sa.grad_scale = grad_scale;
-        scale_dz_kernel<<<dim3((unsigned)((nblk + kBlocksPerCta - 1) / kBlocksPerCta), (unsigned)tpc), 256, 0, ctx->stream>>>(sa);
+        sa.ent = entropy; sa.row_et = with_ent ? f.row_scale : nullptr; sa.zmax = with_ent ? f.zmax : nullptr;
+        const dim3 sgrid((unsigned)((nblk + kBlocksPerCta - 1) / kBlocksPerCta), (unsigned)tpc);
+        if (with_ent) scale_dz_kernel<true><<<sgrid, 256, 0, ctx->stream>>>(sa);
+        else scale_dz_kernel<false><<<sgrid, 256, 0, ctx->stream>>>(sa);
       }
       {
         RangeArgs fa;
@@ -442,6 +514,7 @@ int aero_fwd_bwd_tc(aero_ctx* ctx, const aero_cfg* cfg, int64_t T, int32_t d, in
         fa.lse = lse; fa.g = g; fa.logp = logp; fa.grad_scale = grad_scale;
         fa.H = static_cast<const __nv_bfloat16*>(H); fa.W = static_cast<const __nv_bfloat16*>(W);
         fa.Hs = rowscale ? Hs : nullptr; fa.row_scale = rowscale ? f.row_scale : nullptr;
+        fa.ent = entropy; fa.row_et = with_ent ? f.row_scale : nullptr;
         range_fix_kernel<<<2 * ctx->sm_count, 256, 0, ctx->stream>>>(fa);
       }
 

@@ -513,6 +513,27 @@ def test_one_call_step_redoes_rows_with_a_logit_out_of_range(ctx):
         err = np.linalg.norm(a - b, axis=1)[live] / np.linalg.norm(b, axis=1)[live]
         assert err.max() < GRAD_L2
         assert TL.rel_l2(dW.cpu().numpy(), dW2.cpu().numpy()) < GRAD_L2
+    # the same with the entropy term, whose part of a redone row's dz is recomputed from the logits too
+    ecfg = TL.lib_cfg(O.Cfg(seed=wl.seed, ent_coef=0.5), "bf16")
+    fe = ctx.grpo_loss_reg_fwd(ecfg, H, W, y, old, None, dv["cs"], dv["adv"], dv["w"], dv["keep"], entropy=True)
+    dHe, dWe = ctx.grpo_loss_reg_bwd(ecfg, H, W, y, dv["cs"], dv["keep"], fe["lse"], fe["g"], fe["entropy"], dv["w"],
+                                     logp=fe["logp"])
+    f, dH, dW = ctx.grpo_loss_fwd_bwd(ecfg, H, W, y, old, dv["cs"], dv["adv"], dv["w"], dv["keep"], entropy=True)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    assert torch.isfinite(dH.float()).all() and torch.isfinite(dW).all()
+    np.testing.assert_allclose(f["entropy"][:batch.T].cpu().numpy(), fe["entropy"][:batch.T].cpu().numpy(), atol=2e-5)
+    a, b = dH.float().cpu().numpy(), dHe.float().cpu().numpy()
+    nb = np.linalg.norm(b, axis=1)
+    live = nb > 0
+    # (rows where one column holds all of the probability have H_t = 0 and a gradient of rounding size on both
+    # paths, each with its own noise: a row is compared against its own norm or a twentieth of the typical row's,
+    # whichever is larger -- an entropy term taken from a rounded logarithm would miss that by a factor of 500)
+    err = np.linalg.norm(a - b, axis=1)[live] / np.maximum(nb[live], 0.05 * np.median(nb[live]))
+    assert err.max() < GRAD_L2
+    assert nb[rows[0]] > 0.05 * np.median(nb[live])
+    assert TL.rel_l2(dW.cpu().numpy(), dWe.cpu().numpy()) < GRAD_L2
+    assert TL.rel_l2(dHe.float().cpu().numpy(), dH2.float().cpu().numpy()) > 5 * GRAD_L2      # the term carries weight
 
 
 def _row_err(a, b, rows):
@@ -783,6 +804,32 @@ def test_regularised_objective(ctx, name):
     plain = O.grpo_loss_fwd(ocfg, batch.H, batch.W, batch.st.y, batch.old, batch.st.cs, adv32, w32, rg["keep"])
     pdH, _ = O.grpo_loss_bwd(batch.H, batch.W, batch.st.y, batch.st.cs, rg["keep"], plain["lse"], plain["g"])
     assert TL.rel_l2(pdH, rdH) > 5 * tol[2]
+    # the same objective through the one-call step (aero_grpo_loss_reg_fwd_bwd): the entropy term of dz
+    # takes log p back from the stored exp(z - c_t); unsplit and with the vocabulary split in two
+    for vsplit in ((0,) if dtype == "fp32" else (0, 2)):
+        ctx.set_tuning(vsplit=vsplit)
+        try:
+            f1, dH1, dW1 = ctx.grpo_loss_fwd_bwd(cfg, dv["H"], dv["W"], dv["y"], dv["old"], dv["cs"], dv["adv"], dv["w"],
+                                                 dv["keep"], ref_logp=TL.dev(ref_lp) if use_ref else None,
+                                                 entropy=want_ent)
+            torch.cuda.synchronize()
+        finally:
+            ctx.set_tuning()
+        assert ctx.last_status() == 0
+        assert np.abs(f1["logp"][:batch.T].cpu().numpy() - ref["logp"]).max() <= tol[0]
+        if want_ent:
+            ent1 = f1["entropy"][:batch.T].cpu().numpy()
+            assert np.abs(ent1 - ref["entropy"]).max() <= tol[0] and not ent1[~kept].any()
+        assert abs(f1["loss"].item() - ref["loss"]) <= tol[1] * abs(ref["loss"]) + 1e-7
+        np.testing.assert_allclose(f1["g"][:batch.T].cpu().numpy()[~edge], ref["g"][~edge], rtol=2e-2, atol=1e-9)
+        assert TL.rel_l2(dH1.float().cpu().numpy()[~edge], rdH[~edge]) < tol[2]
+        if not edge.any():
+            assert TL.rel_l2(dW1.cpu().numpy(), rdW) < tol[2]
+            if want_ent:
+                # the entropy part on its own: rows of dW that no token has as its target
+                never_hit = np.setdiff1d(np.arange(wl.V), batch.st.y)
+                if never_hit.size:
+                    assert TL.rel_l2(dW1.cpu().numpy()[never_hit], rdW[never_hit]) < 2 * tol[2]
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
