@@ -28,7 +28,7 @@ int check_ctx(aero_ctx* ctx) {
 
 extern "C" {
 
-int aero_version(void) { return 101; }
+int aero_version(void) { return 102; }
 
 const char* aero_error_string(int code) {
   switch (code) {
